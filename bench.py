@@ -1,0 +1,485 @@
+#!/usr/bin/env python3
+"""Benchmark of the integrity-verification hot path on B200.
+
+One step = one pass of the whole path over one synthetic weight blob: SHA-256 chunk digests,
+Merkle root, comparison with the manifest (`iv_verify_manifest`; for the ragged workload
+`iv_hash_ragged` + `iv_merkle_root`).  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
+
+Multi-GPU runs are launched with torch.distributed.run, one rank per GPU; every rank verifies
+its own blob (independent problems, weak scaling, no data-path collective).
+`--impl reference` times the CPU oracle (the plain restatement of the method) on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+GIB = 1 << 30
+MIB = 1 << 20
+
+# Integer roofline of the path: 1400 INT32 lane-operations per 64-byte block (64 rounds of
+# 6 SHF + 4 LOP3 + 4 IADD3, 48 schedule steps of 6 SHF + 2 LOP3 + 2 IADD3, 16 PRMT, 8 adds)
+# against 148 SMs x 64 INT32 lanes x the maximum SM clock.
+INT_OPS_PER_BYTE = 1400.0 / 64.0
+INT_LANES_PER_SM = 64
+SM_COUNT = 148
+
+CONFIGS = {
+    1: dict(name="config1: 64 MiB uniform random bytes, 64 KiB chunks, 1024 leaves", kind="uniform",
+            nbytes=64 * MIB, chunk=64 << 10),
+    2: dict(name="config2: 2.6 GB 1.3B-parameter bf16 weight file (header + 194 tensors), 1 MiB chunks",
+            kind="file", model="gpt_1p3b", chunk=1 * MIB),
+    3: dict(name="config3: 16 GB 8B-parameter bf16 weight file (header + 291 tensors), 4 MiB chunks",
+            kind="file", model="llama_8b", chunk=4 * MIB),
+    4: dict(name="config4: 112 GiB (120 GB) bf16 weight blob ~N(0,0.02), 4 MiB chunks, 28672 leaves, device-resident",
+            kind="bf16", nbytes=28 * 4 * GIB, chunk=4 * MIB),
+    5: dict(name="config5: 10000 ragged tensors, log-uniform 4 KiB..64 MiB (~69 GB), one SHA-256 each + Merkle root",
+            kind="ragged"),
+}
+
+
+def _env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def _physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# --------------------------------------------------------------------------------------------
+# workloads
+
+def build_workload(cfg_id: int, device, seed: int):
+    from paper_2510_23938_b200 import inputs
+    cfg = dict(CONFIGS[cfg_id])
+    if cfg["kind"] == "uniform":
+        data = inputs.uniform_bytes(cfg["nbytes"], seed, device)
+    elif cfg["kind"] == "bf16":
+        data = torch.empty(cfg["nbytes"], dtype=torch.uint8, device=device)
+        step = 1 * GIB
+        for off in range(0, cfg["nbytes"], step):
+            inputs.fill_bf16_normal(data[off:off + step], seed, first_elem=off // 2)
+    elif cfg["kind"] == "file":
+        tensors = inputs.gpt_1p3b_tensors() if cfg["model"] == "gpt_1p3b" else inputs.llama_8b_tensors()
+        data, table = inputs.weight_file(tensors, seed, device)
+        cfg["table"] = table
+    elif cfg["kind"] == "ragged":
+        sizes = inputs.ragged_sizes(seed=5)
+        offs = inputs.packed_offsets(sizes, first=0)
+        total = int(offs[-1] + sizes[-1])
+        data = torch.empty(total + (-total % 2), dtype=torch.uint8, device=device)
+        step = 1 * GIB
+        for off in range(0, data.numel(), step):
+            inputs.fill_bf16_normal(data[off:off + step], seed, first_elem=off // 2)
+        cfg["offsets"], cfg["lengths"] = offs, sizes
+        cfg["chunk"] = None
+    cfg["nbytes"] = int(data.numel()) if cfg["kind"] != "ragged" else int(cfg["lengths"].sum())
+    cfg["data"] = data
+    return cfg
+
+
+def pick_config(requested: int | None, device) -> tuple[int, str | None]:
+    """The default workload is the largest single-GPU configuration (config 4); it needs ~125 GiB free."""
+    if requested is not None:
+        return requested, None
+    free, _ = torch.cuda.mem_get_info(device)
+    need = CONFIGS[4]["nbytes"] + 14 * GIB
+    if free >= need:
+        return 4, None
+    return 3, f"config4 needs {need / GIB:.0f} GiB free, device has {free / GIB:.0f} GiB"
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+
+def run_ours(args):
+    from paper_2510_23938_b200 import binding, build as iv_build
+    import oracle
+
+    world = _env_int("WORLD_SIZE", 1)
+    rank = _env_int("RANK", 0)
+    local_rank = _env_int("LOCAL_RANK", 0)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    if rank == 0 and iv_build.is_stale():
+        iv_build.build()
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+        dist.barrier()
+
+    cfg_id, fallback = pick_config(args.config, device)
+    ctx = binding.Context(local_rank)
+    t_setup = time.time()
+    wl = build_workload(cfg_id, device, seed=1000 + rank)
+    data, nbytes, chunk = wl["data"], wl["nbytes"], wl["chunk"]
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    ragged = wl["kind"] == "ragged"
+    if ragged:
+        d_off = torch.from_numpy(wl["offsets"]).to(device)
+        d_len = torch.from_numpy(wl["lengths"]).to(device)
+        n_units = int(d_off.numel())
+        digests = torch.empty((n_units, 32), dtype=torch.uint8, device=device)
+        root = torch.empty(32, dtype=torch.uint8, device=device)
+
+        def step():
+            ctx.hash_ragged(data, d_off, d_len, out=digests)
+            ctx.merkle_root(digests, out=root)
+    else:
+        n_units = binding.n_chunks(nbytes, chunk)
+        man_digests = ctx.hash_chunks(data, chunk)
+        man_root = bytes(ctx.merkle_root(man_digests).cpu().numpy().tobytes())
+        manifest = ctx.make_manifest(nbytes, chunk, man_digests, man_root)
+        result = binding.new_result(device)
+        idx = torch.zeros(64, dtype=torch.int64, device=device)
+
+        def step():
+            ctx.verify_manifest(data, manifest, result, idx)
+    torch.cuda.synchronize()
+    setup_s = time.time() - t_setup
+
+    # L2 (126 MB): every workload but config 1 is far larger than L2; config 1 gets a flush between steps.
+    flush = torch.empty(256 * MIB, dtype=torch.uint8, device=device) if nbytes < 512 * MIB else None
+
+    ctx.set_timing(True)
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    launches0 = ctx.kernel_launches
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    with ClockSampler(_physical_gpu_index(local_rank)) as clocks:
+        for k in range(args.steps):
+            if flush is not None:
+                flush.fill_(k & 0xFF)
+            starts[k].record(stream)
+            step()
+            ends[k].record(stream)
+        torch.cuda.synchronize()
+    launches = ctx.kernel_launches - launches0
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    total_ms = float(sum(step_ms)) if flush is not None else float(starts[0].elapsed_time(ends[-1]))
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        dist.barrier()
+    ctx.set_timing(False)
+
+    # dominant kernel: the leaf-hashing launch, timed by the library's own events inside the timed steps
+    if ragged:
+        hash_ms = None
+    else:
+        hash_ms = float(np.mean([ctx.phase_times(k)[0] for k in range(min(args.steps, 64))]))
+        tree_ms = float(np.mean([ctx.phase_times(k)[1] for k in range(min(args.steps, 64))]))
+        cmp_ms = float(np.mean([ctx.phase_times(k)[2] for k in range(min(args.steps, 64))]))
+
+    if ragged:
+        # time the hashing launch alone, same launch configuration, for the roofline line
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ctx.hash_ragged(data, d_off, d_len, out=digests)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        hash_ms, tree_ms, cmp_ms = float(e0.elapsed_time(e1)), None, None
+
+    ms_per_step = total_ms / args.steps
+    value = world * nbytes / (ms_per_step * 1e-3) / 1e9
+
+    peak_gbs = SM_COUNT * INT_LANES_PER_SM * 1.965e9 / INT_OPS_PER_BYTE / 1e9
+    achieved = nbytes / (hash_ms * 1e-3) / 1e9
+    roofline = {
+        "bound": "alu", "kernel": "hash_ragged_kernel" if ragged else "hash_chunks_kernel",
+        "achieved": round(achieved, 2), "peak": round(peak_gbs, 1), "unit": "GB/s",
+        "frac": round(achieved / peak_gbs, 4), "traffic": None,
+        "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1.965 GHz / 21.875 INT32 ops per byte",
+        "hbm_peak_gbs_measured": _measured_peak("hbm_gbs"),
+        "launch_ms": round(hash_ms, 4), "tree_ms": tree_ms, "compare_ms": cmp_ms,
+        "chains": n_units,
+    }
+
+    out = {
+        "metric": "GB/s verified (SHA-256 chunks + Merkle root + manifest compare) at 1 B200",
+        "value": round(value, 3), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u32", "data": "synthetic",
+        "config": {"workload": wl["name"], "bytes_per_gpu": nbytes, "chunk_bytes": chunk, "units": n_units,
+                   "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps (256 MiB write)",
+                   "parallelism": f"independent blob per GPU x{world}", "setup_s": round(setup_s, 1)},
+        "clocks": clocks.summary(), "gpu_launches": int(launches), "roofline": roofline,
+    }
+    if fallback:
+        out["config"]["fallback"] = fallback
+
+    if rank == 0 and not ragged and not args.no_e2e:
+        out["e2e"] = measure_e2e(ctx, wl, device, args)
+    elif rank == 0:
+        out["e2e"] = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        out["cpu_baseline"] = measure_cpu_baseline(ctx, wl, device, oracle, ragged,
+                                                   None if ragged else man_digests,
+                                                   (d_off, d_len, digests) if ragged else None)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    ctx.close()
+
+
+def _measured_peak(key):
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f).get(key)
+    except Exception:
+        return None
+
+
+def measure_e2e(ctx, wl, device, args):
+    """Same metric through iv_verify_streamed: the blob starts in pinned HOST memory, every step copies it
+    to the device in 4 GiB windows (overlapped with hashing) and reads the verification result back."""
+    from paper_2510_23938_b200 import binding
+    data, nbytes, chunk = wl["data"], wl["nbytes"], wl["chunk"]
+    window = min(4 * GIB, -(-nbytes // chunk) * chunk)
+    n_win = -(-nbytes // window)
+    ring = None
+    for r in (min(4, n_win), 2, 1):
+        if r > n_win:
+            continue
+        try:
+            ring = [torch.empty(min(window, nbytes - w * window) if n_win <= r else window,
+                                dtype=torch.uint8, pin_memory=True) for w in range(r)]
+            break
+        except RuntimeError:
+            ring = None
+    if ring is None:
+        return {"value": None, "unit": "GB/s", "note": "could not pin host memory"}
+    r = len(ring)
+    for w in range(r):
+        ring[w].copy_(data[w * window:w * window + ring[w].numel()])
+    torch.cuda.synchronize()
+    windows = [ring[w % r] for w in range(n_win)]
+    periodic = n_win > r
+    if periodic:
+        # the streamed blob is window (w mod r) of the resident blob; its manifest follows from the ring's digests
+        per = [ctx.hash_chunks(data[w * window:(w + 1) * window], chunk) for w in range(r)]
+        man_digests = torch.cat([per[w % r] for w in range(n_win)])
+        e_nbytes = n_win * window
+    else:
+        man_digests = ctx.hash_chunks(data, chunk)
+        e_nbytes = nbytes
+    man_root = bytes(ctx.merkle_root(man_digests).cpu().numpy().tobytes())
+    manifest = ctx.make_manifest(e_nbytes, chunk, man_digests, man_root)
+    result = binding.new_result(device)
+    idx = torch.zeros(64, dtype=torch.int64, device=device)
+    stream = torch.cuda.current_stream()
+    steps = max(1, min(args.steps, 3))
+    ok = True
+    for _ in range(1):
+        ctx.verify_streamed(windows, window, e_nbytes, manifest, result, idx)
+        ok &= binding.read_result(result)["root_ok"]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(steps):
+        ctx.verify_streamed(windows, window, e_nbytes, manifest, result, idx)
+        host_result = binding.read_result(result)          # device -> host read of the step's result
+        ok &= host_result["root_ok"] and host_result["n_mismatch"] == 0
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return {"value": round(e_nbytes / (ms * 1e-3) / 1e9, 3), "unit": "GB/s", "ms_per_step": round(ms, 3),
+            "steps": steps, "h2d_bytes_per_step": int(e_nbytes), "d2h_bytes_per_step": 48,
+            "api": "iv_verify_streamed, pinned host windows of %d MiB, two device windows" % (window // MIB),
+            "host_ring_windows": r, "periodic_blob": periodic, "verified_ok": bool(ok)}
+
+
+def measure_cpu_baseline(ctx, wl, device, oracle, ragged, man_digests, ragged_state):
+    """The oracle, as it stands, on the host cores, on a bounded sample of the same bytes; also a parity check
+    of the GPU digests for that sample."""
+    cores = oracle.host_threads()
+    data, chunk = wl["data"], wl["chunk"]
+    if ragged:
+        d_off, d_len, digests = ragged_state
+        lens = wl["lengths"]
+        budget, pick, acc = 3 * GIB, [], 0
+        for k in range(len(lens)):
+            if acc + int(lens[k]) > budget:
+                break
+            pick.append(k)
+            acc += int(lens[k])
+        hi = int(wl["offsets"][pick[-1]] + lens[pick[-1]])
+        host = data[:hi].cpu().numpy()
+        t0 = time.perf_counter()
+        want = oracle.hash_ragged(host, wl["offsets"][:len(pick)], lens[:len(pick)], nthreads=cores)
+        root = oracle.merkle_root(want)
+        dt = time.perf_counter() - t0
+        got = digests[:len(pick)].cpu().numpy()
+        parity = bool(np.array_equal(got, want))
+        sample = f"first {len(pick)} tensors ({acc / 1e9:.2f} GB) of the same set"
+        nb = acc
+    else:
+        n = man_digests.shape[0]
+        ns = min(n, max(1, (4 * GIB) // chunk))
+        nb = min(wl["nbytes"], ns * chunk)
+        host = data[:nb].cpu().numpy()
+        gpu_d = man_digests[:ns].cpu().numpy()
+        gpu_root = bytes(ctx.merkle_root(man_digests[:ns].contiguous()).cpu().numpy().tobytes())
+        t0 = time.perf_counter()
+        ok, bad, _, root = oracle.verify(host, chunk, gpu_d, gpu_root, nthreads=cores)
+        dt = time.perf_counter() - t0
+        parity = bool(ok and bad == 0)
+        sample = f"first {ns} chunks ({nb / 1e9:.2f} GB) of the same blob, verified against the GPU's digests and root"
+    return {"value": round(nb / dt / 1e9, 3), "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample,
+            "seconds": round(dt, 2), "gpu_matches_oracle_on_sample": parity}
+
+
+# --------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle
+
+def run_reference(args):
+    rank = _env_int("RANK", 0)
+    if rank != 0:
+        return
+    import oracle
+    from paper_2510_23938_b200 import inputs
+    cfg_id = args.config if args.config is not None else 4
+    cfg = CONFIGS[cfg_id]
+    cores = oracle.host_threads()
+    chunk = cfg.get("chunk") or 4 * MIB
+    sample_bytes = min(cfg.get("nbytes", 1 * GIB), 1 * GIB)
+    sample_bytes -= sample_bytes % chunk
+    sample_bytes = max(sample_bytes, chunk)
+    if cfg["kind"] == "uniform":
+        host = inputs.uniform_bytes(sample_bytes, 1000).numpy()
+    else:
+        host = inputs.bf16_normal_bytes(sample_bytes // 2, 1000).numpy()
+    digests = oracle.hash_chunks(host, chunk, nthreads=cores)
+    root = oracle.merkle_root(digests)
+    times = []
+    for k in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        ok, bad, _, _ = oracle.verify(host, chunk, digests, root, nthreads=cores)
+        dt = time.perf_counter() - t0
+        assert ok and bad == 0
+        if k >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = sample_bytes / (ms * 1e-3) / 1e9
+    sample = f"{sample_bytes / MIB:.0f} MiB of the workload's bytes per step ({sample_bytes // chunk} chunks of {chunk // 1024} KiB)"
+    print(json.dumps({
+        "impl": "reference",
+        "metric": "GB/s verified (SHA-256 chunks + Merkle root + manifest compare) at 1 B200",
+        "value": round(value, 4), "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(ms, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u32", "data": "synthetic",
+        "config": {"workload": cfg["name"], "sample": sample},
+        "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=None, choices=sorted(CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

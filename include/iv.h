@@ -1,0 +1,222 @@
+/*
+ * iv.h -- C ABI of libiv: GPU-resident integrity verification of model-weight
+ * bytes on NVIDIA B200 (sm_100a).
+ *
+ * The library computes, entirely in CUDA kernels, the data-parallel path of the
+ * paper "Scalable GPU-Based Integrity Verification for Large Machine Learning
+ * Models": FIPS 180-4 SHA-256 digests of fixed-size chunks of a byte blob, a
+ * binary Merkle reduction of those digests to a root, and the comparison of
+ * digests and root with an expected manifest (Algorithm 1, "Streaming Model
+ * Verification", and the section "Memory Scalability Considerations").
+ *
+ * Conventions
+ *  - Pointers named d_* are DEVICE pointers owned by the caller; the library
+ *    neither frees nor keeps them beyond the work it enqueues.  Pointers named
+ *    h_* are HOST pointers.  Everything else is passed by value.
+ *  - A digest is 32 bytes: the eight 32-bit words H0..H7 of FIPS 180-4
+ *    section 6.2.2, each stored big-endian.  Digest arrays are contiguous
+ *    records in index order.
+ *  - Every call enqueues its GPU work on `cuda_stream` (a cudaStream_t passed
+ *    as void*, NULL = the legacy default stream) and returns without waiting,
+ *    except where stated.  Results in device memory are valid once the stream
+ *    has reached that point.
+ *  - Return value: IV_OK (0) or a negative iv_status.  Finding a mismatch is
+ *    NOT an error: verification calls return IV_OK and report it in the result.
+ *  - There is no CPU fallback: without a usable CUDA device iv_create fails.
+ *  - A context may be used by one host thread at a time.  Calls on the same
+ *    context that overlap on the GPU (different streams) share its scratch
+ *    memory and therefore race; serialise them or use one context per stream.
+ */
+#ifndef IV_H
+#define IV_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum iv_status {
+    IV_OK = 0,
+    IV_ERR_INVALID_ARG = -1, /* null pointer, zero chunk size, capacity too small, inconsistent manifest */
+    IV_ERR_NOMEM = -2,       /* a device or host allocation for scratch failed */
+    IV_ERR_CUDA = -3,        /* a CUDA runtime call failed; see iv_last_cuda_error */
+    IV_ERR_NO_DEVICE = -4    /* no CUDA device, or not a compute-capability-10.x device */
+} iv_status;
+
+/* Opaque context.  Owns scratch memory (Merkle level buffers, tickets, the
+ * digest array used by verification, streaming windows), sized lazily. */
+typedef struct iv_ctx iv_ctx;
+
+/* Creates a context on CUDA device `cuda_device`.  Synchronous.  *out is set
+ * to NULL on failure. */
+int iv_create(iv_ctx **out, int cuda_device);
+
+/* Waits for the device, frees all scratch, destroys the context.  NULL is allowed. */
+int iv_destroy(iv_ctx *ctx);
+
+/* Static, human-readable text for a status code. */
+const char *iv_strerror(int code);
+
+/* The cudaError_t (as int) of the last failed CUDA call on this context, 0 if none. */
+int iv_last_cuda_error(const iv_ctx *ctx);
+
+/* Number of kernels this context has launched so far (a host-side counter). */
+uint64_t iv_kernel_launches(const iv_ctx *ctx);
+
+/* ---------------------------------------------------------------------------
+ * Leaf hashing -- Algorithm 1, "chunk_count <- ceil(|M| / C)" and
+ * "H_i = GPU_HASH(M_i)" with GPU_HASH = SHA-256 (FIPS 180-4 section 6.2).
+ *
+ *   d_data        nbytes bytes of device memory, any alignment
+ *   chunk_bytes   C > 0; chunk i covers bytes [i*C, min((i+1)*C, nbytes)); the
+ *                 last chunk is hashed at its true length (no zero fill)
+ *   d_digests     receives n = ceil(nbytes / C) records of 32 bytes
+ *   digests_cap   capacity of d_digests in records; n > digests_cap is an error
+ *   h_n_chunks    optional host pointer, receives n (written before returning)
+ *
+ * nbytes == 0 gives n == 0 and launches nothing.  Streaming (the loop of
+ * Algorithm 1) needs no other entry point: call once per resident window,
+ * each window a multiple of C except the last, with d_digests advanced by
+ * 32 * (chunks before the window).
+ */
+int iv_hash_chunks(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                   uint8_t *d_digests, uint64_t digests_cap, uint64_t *h_n_chunks,
+                   void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Merkle reduction -- Algorithm 1, "Construct Merkle tree from leaf_hashes
+ * using GPU".  Binary tree over n_leaves digests in index order; a parent is
+ * SHA-256(left || right) of exactly 64 bytes (no domain-separation prefix); an
+ * unpaired last node of a level moves up unchanged; one leaf is its own root;
+ * zero leaves give SHA-256 of the empty string.
+ *
+ *   d_leaves   n_leaves * 32 bytes (may be NULL when n_leaves == 0)
+ *   d_root     receives 32 bytes
+ */
+int iv_merkle_root(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
+                   void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Verification -- Algorithm 1, "Compare root hash with expected value", plus
+ * the per-chunk comparison that locates the damage.
+ *
+ * The manifest is the publisher's expected value: the blob's size, the chunk
+ * size, the chunk digests and their Merkle root.
+ */
+typedef struct iv_manifest {
+    uint64_t total_bytes;     /* must equal nbytes of the call */
+    uint64_t chunk_bytes;     /* C */
+    uint64_t n_chunks;        /* must equal ceil(total_bytes / chunk_bytes) */
+    const uint8_t *d_digests; /* DEVICE: n_chunks * 32 bytes (may be NULL when n_chunks == 0) */
+    uint8_t root[32];         /* expected Merkle root (host bytes inside this struct) */
+} iv_manifest;
+
+/* Written by the GPU into DEVICE memory supplied by the caller. */
+typedef struct iv_verify_result {
+    uint32_t status;     /* device-side status: 0 = completed */
+    uint32_t root_ok;    /* 1 iff the recomputed root equals manifest root */
+    uint64_t n_mismatch; /* exact number of chunks whose digest differs, even if > idx_cap */
+    uint8_t root[32];    /* the recomputed root */
+} iv_verify_result;
+
+/*   d_data, nbytes    the blob to verify (device)
+ *   h_manifest        host struct (read before returning), digests on the device
+ *   d_result          device memory for one iv_verify_result
+ *   d_mismatch_idx    device array of idx_cap uint64: the indices of mismatching
+ *                     chunks in ASCENDING order, the first min(n_mismatch, idx_cap)
+ *                     of them; may be NULL when idx_cap == 0
+ * The recomputed chunk digests stay in the context (iv_ctx_digests). */
+int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
+                       const iv_manifest *h_manifest, iv_verify_result *d_result,
+                       uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream);
+
+/* Device pointer of the digest array the last iv_verify_manifest /
+ * iv_verify_streamed on this context wrote (n_chunks * 32 bytes), NULL if none. */
+const uint8_t *iv_ctx_digests(const iv_ctx *ctx);
+
+/* ---------------------------------------------------------------------------
+ * Streamed verification -- the whole of Algorithm 1 for a blob that lives in
+ * HOST memory ("Load model chunk M_i into GPU memory ... Free GPU memory"):
+ * the blob is copied window by window into two device windows owned by the
+ * context, the copy of window w+1 overlapping the hashing of window w on a
+ * second stream, then the tree is built and compared as in iv_verify_manifest.
+ *
+ *   h_windows      host array of n_windows HOST pointers; window w holds bytes
+ *                  [w*window_bytes, min((w+1)*window_bytes, nbytes)) of the blob.
+ *                  The windows need not be adjacent in memory (file shards,
+ *                  mapped pieces) and may repeat.  Page-locked memory is needed
+ *                  for the copies to overlap (pageable memory works, slowly).
+ *   n_windows      must equal ceil(nbytes / window_bytes)
+ *   window_bytes   > 0, a multiple of h_manifest->chunk_bytes
+ * The pointer array is read before the call returns; the window contents must
+ * stay valid until the enqueued copies have run.  The call returns when all
+ * work is ENQUEUED on cuda_stream and the context's copy stream; cuda_stream
+ * reaches completion only after both are done.
+ */
+int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_windows,
+                       uint64_t window_bytes, uint64_t nbytes, const iv_manifest *h_manifest,
+                       iv_verify_result *d_result, uint64_t *d_mismatch_idx, uint64_t idx_cap,
+                       void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Phase timing (the paper's result record carries a verification time).  When
+ * switched on, iv_verify_manifest and iv_verify_streamed bracket their three
+ * phases -- leaf hashing, tree reduction, comparison -- with CUDA events on
+ * cuda_stream.  The context keeps the events of the most recent
+ * IV_TIMING_RING verification calls.
+ *
+ * iv_phase_times waits for the events of the call made `calls_back` calls ago
+ * (0 = the most recent) and writes the three durations in milliseconds to
+ * h_ms[0..2].  Returns IV_ERR_INVALID_ARG if timing was off for that call or
+ * calls_back >= IV_TIMING_RING.
+ */
+#define IV_TIMING_RING 64
+int iv_set_timing(iv_ctx *ctx, int enabled);
+int iv_phase_times(iv_ctx *ctx, uint32_t calls_back, float *h_ms);
+
+/* ---------------------------------------------------------------------------
+ * Per-tensor digests -- the paper's batch verification ("verification of
+ * dozens of models concurrently", one digest per payload): digest k =
+ * SHA-256(d_base[offset_k .. offset_k + length_k)).
+ *
+ *   d_offsets, d_lengths   n uint64 each, DEVICE memory; any byte alignment of
+ *                          offsets, any length including 0
+ *   d_digests              receives n * 32 bytes
+ * The caller guarantees that every range lies inside the d_base allocation.
+ */
+int iv_hash_ragged(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets,
+                   const uint64_t *d_lengths, uint64_t n, uint8_t *d_digests,
+                   void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Roofline probe (a measurement aid; the paper has no counterpart).  Runs a
+ * register-only microbenchmark on every SM and reports, from the SM cycle
+ * counter, how many lane-operations of one instruction kind an SM retires per
+ * clock -- the denominator of the integer roofline -- or, for IV_PROBE_SHA256,
+ * how many message bytes per clock per SM the compression function alone
+ * sustains.  Synchronous; allocates and frees a few KB of device memory.
+ *
+ *   warps_per_block, blocks_per_sm   launch shape (blocks = blocks_per_sm * SM count)
+ *   active_lanes                     1..32 lanes of each warp that do work
+ *   iters                            loop trips (128 operations each; one compression
+ *                                    each for IV_PROBE_SHA256)
+ *   h_out[0]                         lane-ops (or bytes) per clock per SM
+ *   h_out[1]                         mean cycles per block
+ */
+typedef enum iv_probe_kind {
+    IV_PROBE_IADD3 = 0,  /* three-input integer add */
+    IV_PROBE_LOP3 = 1,   /* three-input logic op */
+    IV_PROBE_SHF = 2,    /* funnel shift (rotate) */
+    IV_PROBE_PRMT = 3,   /* byte permute */
+    IV_PROBE_IMAD = 4,   /* integer multiply-add */
+    IV_PROBE_MIXED = 5,  /* LOP3 and IMAD interleaved 1:1 */
+    IV_PROBE_SHA256 = 6  /* full SHA-256 compressions, registers only */
+} iv_probe_kind;
+int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t blocks_per_sm,
+                 uint32_t active_lanes, uint32_t iters, double *h_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IV_H */

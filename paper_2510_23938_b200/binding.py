@@ -1,0 +1,285 @@
+"""ctypes binding of libiv.so: the same entry points as include/iv.h.
+
+Argument marshalling only.  Tensors are torch CUDA tensors (torch supplies
+device memory and streams); every step of the path runs inside the library's
+kernels.  There is no fallback: if the shared library is missing, loading
+raises with the build command.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libiv.so")
+
+IV_OK = 0
+IV_ERR_INVALID_ARG = -1
+IV_ERR_NOMEM = -2
+IV_ERR_CUDA = -3
+IV_ERR_NO_DEVICE = -4
+
+EXPORTS = (
+    "iv_create", "iv_destroy", "iv_strerror", "iv_last_cuda_error", "iv_kernel_launches",
+    "iv_hash_chunks", "iv_merkle_root", "iv_verify_manifest", "iv_ctx_digests",
+    "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu",
+)
+
+
+class IvError(RuntimeError):
+    def __init__(self, code: int, what: str, cuda_error: int = 0):
+        self.code = code
+        self.cuda_error = cuda_error
+        extra = f" (cudaError {cuda_error})" if cuda_error else ""
+        super().__init__(f"{what}: {_strerror(code)}{extra}")
+
+
+class Manifest(ctypes.Structure):
+    """iv_manifest: host struct, digest array on the device."""
+    _fields_ = [("total_bytes", ctypes.c_uint64), ("chunk_bytes", ctypes.c_uint64),
+                ("n_chunks", ctypes.c_uint64), ("d_digests", ctypes.c_void_p),
+                ("root", ctypes.c_uint8 * 32)]
+
+
+class VerifyResult(ctypes.Structure):
+    """iv_verify_result as laid out in device memory (48 bytes)."""
+    _fields_ = [("status", ctypes.c_uint32), ("root_ok", ctypes.c_uint32),
+                ("n_mismatch", ctypes.c_uint64), ("root", ctypes.c_uint8 * 32)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libiv.so from the package directory; raises if it was not built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2510_23938_b200.build` "
+            "(needs nvcc; there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, u64, i32 = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int
+    lib.iv_create.argtypes = [ctypes.POINTER(vp), i32]
+    lib.iv_create.restype = i32
+    lib.iv_destroy.argtypes = [vp]
+    lib.iv_destroy.restype = i32
+    lib.iv_strerror.argtypes = [i32]
+    lib.iv_strerror.restype = ctypes.c_char_p
+    lib.iv_last_cuda_error.argtypes = [vp]
+    lib.iv_last_cuda_error.restype = i32
+    lib.iv_kernel_launches.argtypes = [vp]
+    lib.iv_kernel_launches.restype = u64
+    lib.iv_hash_chunks.argtypes = [vp, vp, u64, u64, vp, u64, ctypes.POINTER(u64), vp]
+    lib.iv_hash_chunks.restype = i32
+    lib.iv_merkle_root.argtypes = [vp, vp, u64, vp, vp]
+    lib.iv_merkle_root.restype = i32
+    lib.iv_verify_manifest.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
+    lib.iv_verify_manifest.restype = i32
+    lib.iv_ctx_digests.argtypes = [vp]
+    lib.iv_ctx_digests.restype = vp
+    lib.iv_verify_streamed.argtypes = [vp, ctypes.POINTER(vp), u64, u64, u64, ctypes.POINTER(Manifest),
+                                       vp, vp, u64, vp]
+    lib.iv_verify_streamed.restype = i32
+    lib.iv_set_timing.argtypes = [vp, i32]
+    lib.iv_set_timing.restype = i32
+    lib.iv_phase_times.argtypes = [vp, ctypes.c_uint32, ctypes.POINTER(ctypes.c_float)]
+    lib.iv_phase_times.restype = i32
+    lib.iv_hash_ragged.argtypes = [vp, vp, vp, vp, u64, vp, vp]
+    lib.iv_hash_ragged.restype = i32
+    lib.iv_probe_alu.argtypes = [vp, i32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
+                                 ctypes.POINTER(ctypes.c_double)]
+    lib.iv_probe_alu.restype = i32
+    _lib = lib
+    return lib
+
+
+def _strerror(code: int) -> str:
+    try:
+        return load_library().iv_strerror(code).decode()
+    except Exception:  # pragma: no cover
+        return f"status {code}"
+
+
+def n_chunks(nbytes: int, chunk_bytes: int) -> int:
+    return 0 if nbytes == 0 else (nbytes - 1) // chunk_bytes + 1
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _dev_ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None or t.numel() == 0:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _nbytes(t: torch.Tensor) -> int:
+    return t.numel() * t.element_size()
+
+
+class Context:
+    """iv_ctx: scratch memory and streams of one verifier on one device."""
+
+    def __init__(self, device: int | None = None):
+        lib = load_library()
+        if device is None:
+            device = torch.cuda.current_device() if torch.cuda.is_available() else 0
+        self.device = int(device)
+        handle = ctypes.c_void_p()
+        rc = lib.iv_create(ctypes.byref(handle), self.device)
+        if rc != IV_OK:
+            raise IvError(rc, "iv_create")
+        self._h = handle
+        self._lib = lib
+
+    # -- plumbing ---------------------------------------------------------------------------
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.iv_destroy(self._h)
+            self._h = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def _check(self, rc: int, what: str):
+        if rc != IV_OK:
+            raise IvError(rc, what, self._lib.iv_last_cuda_error(self._h))
+
+    @property
+    def kernel_launches(self) -> int:
+        return int(self._lib.iv_kernel_launches(self._h))
+
+    # -- entry points -----------------------------------------------------------------------
+    def hash_chunks(self, data: torch.Tensor, chunk_bytes: int, out: torch.Tensor | None = None,
+                    nbytes: int | None = None, stream=None) -> torch.Tensor:
+        """iv_hash_chunks: (n, 32) uint8 digests of the chunks of `data` (any dtype, read as bytes)."""
+        nb = _nbytes(data) if nbytes is None else int(nbytes)
+        n = n_chunks(nb, chunk_bytes) if chunk_bytes > 0 else 0
+        if out is None:
+            out = torch.empty((n, 32), dtype=torch.uint8, device=data.device)
+        got = ctypes.c_uint64(0)
+        rc = self._lib.iv_hash_chunks(self._h, _dev_ptr(data), nb, chunk_bytes, _dev_ptr(out),
+                                      out.numel() // 32, ctypes.byref(got), _stream_ptr(stream))
+        self._check(rc, "iv_hash_chunks")
+        return out[:got.value]
+
+    def merkle_root(self, leaves: torch.Tensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+        """iv_merkle_root: 32-byte root (uint8 tensor on the device) of (n, 32) leaf digests."""
+        n = leaves.numel() // 32
+        if out is None:
+            out = torch.empty(32, dtype=torch.uint8, device=leaves.device)
+        rc = self._lib.iv_merkle_root(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
+        self._check(rc, "iv_merkle_root")
+        return out
+
+    def make_manifest(self, total_bytes: int, chunk_bytes: int, digests: torch.Tensor, root: bytes) -> Manifest:
+        m = Manifest()
+        m.total_bytes = total_bytes
+        m.chunk_bytes = chunk_bytes
+        m.n_chunks = digests.numel() // 32
+        m.d_digests = _dev_ptr(digests)
+        m.root = (ctypes.c_uint8 * 32).from_buffer_copy(root)
+        m._keepalive = digests
+        return m
+
+    def verify_manifest(self, data: torch.Tensor, manifest: Manifest, result: torch.Tensor,
+                        mismatch_idx: torch.Tensor | None, nbytes: int | None = None, stream=None) -> None:
+        """iv_verify_manifest (asynchronous): `result` is a 48-byte uint8 device tensor,
+        `mismatch_idx` an int64 device tensor whose length is the index capacity."""
+        nb = _nbytes(data) if nbytes is None else int(nbytes)
+        cap = 0 if mismatch_idx is None else mismatch_idx.numel()
+        rc = self._lib.iv_verify_manifest(self._h, _dev_ptr(data), nb, ctypes.byref(manifest),
+                                          _dev_ptr(result), _dev_ptr(mismatch_idx), cap, _stream_ptr(stream))
+        self._check(rc, "iv_verify_manifest")
+
+    def verify_streamed(self, host_windows, window_bytes: int, nbytes: int, manifest: Manifest,
+                        result: torch.Tensor, mismatch_idx: torch.Tensor | None, stream=None) -> None:
+        """iv_verify_streamed (asynchronous).  `host_windows` is a CPU uint8 tensor holding the whole
+        blob, or a list of CPU tensors, one per window (pinned for overlap; entries may repeat)."""
+        if isinstance(host_windows, torch.Tensor):
+            flat = host_windows.view(torch.uint8).reshape(-1)
+            assert not flat.is_cuda and flat.is_contiguous() and flat.numel() >= nbytes
+            host_windows = [flat[o:o + window_bytes] for o in range(0, nbytes, window_bytes)] if window_bytes > 0 else []
+        n_win = len(host_windows)
+        ptrs = (ctypes.c_void_p * max(n_win, 1))()
+        for w, t in enumerate(host_windows):
+            assert not t.is_cuda and t.is_contiguous()
+            ptrs[w] = t.data_ptr()
+        cap = 0 if mismatch_idx is None else mismatch_idx.numel()
+        rc = self._lib.iv_verify_streamed(self._h, ptrs, n_win, window_bytes, nbytes, ctypes.byref(manifest),
+                                          _dev_ptr(result), _dev_ptr(mismatch_idx), cap, _stream_ptr(stream))
+        self._check(rc, "iv_verify_streamed")
+
+    def set_timing(self, enabled: bool) -> None:
+        self._check(self._lib.iv_set_timing(self._h, int(enabled)), "iv_set_timing")
+
+    def phase_times(self, calls_back: int = 0) -> tuple[float, float, float]:
+        """iv_phase_times: (hash, tree, compare) milliseconds of a recent verification call."""
+        ms = (ctypes.c_float * 3)()
+        self._check(self._lib.iv_phase_times(self._h, calls_back, ms), "iv_phase_times")
+        return float(ms[0]), float(ms[1]), float(ms[2])
+
+    def hash_ragged(self, base: torch.Tensor, offsets: torch.Tensor, lengths: torch.Tensor,
+                    out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+        """iv_hash_ragged: (n, 32) digests of base[offset_k : offset_k + length_k) (offsets/lengths int64 on device)."""
+        n = offsets.numel()
+        assert lengths.numel() == n and offsets.dtype == torch.int64 and lengths.dtype == torch.int64
+        if out is None:
+            out = torch.empty((n, 32), dtype=torch.uint8, device=base.device)
+        rc = self._lib.iv_hash_ragged(self._h, _dev_ptr(base), _dev_ptr(offsets), _dev_ptr(lengths), n,
+                                      _dev_ptr(out), _stream_ptr(stream))
+        self._check(rc, "iv_hash_ragged")
+        return out
+
+    PROBE_KINDS = {"iadd3": 0, "lop3": 1, "shf": 2, "prmt": 3, "imad": 4, "mixed": 5, "sha256": 6}
+
+    def probe_alu(self, kind: str, warps_per_block: int = 4, blocks_per_sm: int = 1, active_lanes: int = 32,
+                  iters: int = 2000) -> tuple[float, float]:
+        """iv_probe_alu: (lane-ops or bytes per clock per SM, mean cycles per block)."""
+        out = (ctypes.c_double * 2)()
+        rc = self._lib.iv_probe_alu(self._h, self.PROBE_KINDS[kind], warps_per_block, blocks_per_sm,
+                                    active_lanes, iters, out)
+        self._check(rc, "iv_probe_alu")
+        return float(out[0]), float(out[1])
+
+    def last_digests(self, n: int) -> torch.Tensor:
+        """Copy of the chunk digests the last verification on this context computed."""
+        ptr = self._lib.iv_ctx_digests(self._h)
+        if not ptr:
+            raise RuntimeError("no verification has run on this context")
+        out = torch.empty((n, 32), dtype=torch.uint8, device=f"cuda:{self.device}")
+        if n:
+            cudart = torch.cuda.cudart()
+            err = cudart.cudaMemcpy(out.data_ptr(), ptr, 32 * n, 3)  # device to device
+            if int(err) != 0:
+                raise RuntimeError(f"cudaMemcpy failed: {err}")
+        return out
+
+
+def read_result(result: torch.Tensor) -> dict:
+    """Decodes a 48-byte iv_verify_result tensor (synchronises on the copy to the host)."""
+    raw = bytes(result.cpu().numpy().tobytes())
+    r = VerifyResult.from_buffer_copy(raw)
+    return {"status": int(r.status), "root_ok": bool(r.root_ok), "n_mismatch": int(r.n_mismatch),
+            "root": bytes(r.root)}
+
+
+def new_result(device) -> torch.Tensor:
+    return torch.zeros(ctypes.sizeof(VerifyResult), dtype=torch.uint8, device=device)

@@ -1,0 +1,396 @@
+// C ABI of libiv (see include/iv.h): argument checks, scratch management,
+// stream plumbing.  All arithmetic of the path runs in the kernels.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "iv_internal.h"
+
+struct iv_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int last_cuda_error = 0;
+    uint64_t launches = 0;
+
+    // small fixed block: tickets, work-queue counter, root
+    uint32_t *d_tickets = nullptr;            // kMerkleMaxPasses + 1 words
+    unsigned long long *d_queue = nullptr;
+    uint8_t *d_root = nullptr;                // 32 bytes
+    void *d_small = nullptr;
+
+    // lazily sized scratch
+    uint8_t *d_merkle_a = nullptr, *d_merkle_b = nullptr;
+    uint64_t merkle_cap = 0;                  // in digests, each buffer
+    uint8_t *d_digests = nullptr;
+    uint64_t digests_cap = 0;                 // in digests
+    uint64_t digests_valid = 0;
+    uint32_t *d_words = nullptr;
+    uint64_t words_cap = 0;
+
+    // streaming windows
+    uint8_t *d_window[2] = {nullptr, nullptr};
+    uint64_t window_cap = 0;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_entry = nullptr, ev_copied[2] = {nullptr, nullptr}, ev_hashed[2] = {nullptr, nullptr};
+
+    // phase timing: four events (start, hashed, reduced, compared) per recent call
+    bool timing = false;
+    uint64_t timed_calls = 0;                          // verification calls made so far
+    cudaEvent_t ev_phase[IV_TIMING_RING][4] = {};
+    bool slot_timed[IV_TIMING_RING] = {};
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) cudaSetDevice(dev);
+        else prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+int fail_cuda(iv_ctx *ctx, cudaError_t e) {
+    if (ctx) ctx->last_cuda_error = (int)e;
+    (void)cudaGetLastError();   // clear the sticky-free error state
+    return e == cudaErrorMemoryAllocation ? IV_ERR_NOMEM : IV_ERR_CUDA;
+}
+
+#define IV_TRY(ctx, call)                                   \
+    do {                                                    \
+        cudaError_t e_ = (call);                            \
+        if (e_ != cudaSuccess) return fail_cuda((ctx), e_); \
+    } while (0)
+
+uint64_t chunk_count(uint64_t nbytes, uint64_t chunk_bytes) {
+    return nbytes == 0 ? 0 : (nbytes - 1) / chunk_bytes + 1;
+}
+
+// Grows a device buffer to at least `need` bytes (contents are not preserved).
+template <typename T>
+int grow(iv_ctx *ctx, T **buf, uint64_t *cap_items, uint64_t need_items, uint64_t item_bytes) {
+    if (need_items <= *cap_items) return IV_OK;
+    if (*buf) {
+        IV_TRY(ctx, cudaDeviceSynchronize());
+        IV_TRY(ctx, cudaFree(*buf));
+        *buf = nullptr;
+        *cap_items = 0;
+    }
+    uint64_t items = need_items + need_items / 4 + 64;
+    void *p = nullptr;
+    IV_TRY(ctx, cudaMalloc(&p, items * item_bytes));
+    *buf = static_cast<T *>(p);
+    *cap_items = items;
+    return IV_OK;
+}
+
+int ensure_merkle_scratch(iv_ctx *ctx, uint64_t n_leaves) {
+    const uint64_t need = (n_leaves + ivk::kMerkleRun - 1) / ivk::kMerkleRun + 1;
+    if (need <= ctx->merkle_cap) return IV_OK;
+    uint64_t cap_a = ctx->merkle_cap, cap_b = ctx->merkle_cap;
+    int rc = grow(ctx, &ctx->d_merkle_a, &cap_a, need, 32);
+    if (rc != IV_OK) return rc;
+    rc = grow(ctx, &ctx->d_merkle_b, &cap_b, need, 32);
+    if (rc != IV_OK) return rc;
+    ctx->merkle_cap = cap_a < cap_b ? cap_a : cap_b;
+    return IV_OK;
+}
+
+int check_manifest(const iv_manifest *m, uint64_t nbytes) {
+    if (!m || m->chunk_bytes == 0) return IV_ERR_INVALID_ARG;
+    if (m->total_bytes != nbytes) return IV_ERR_INVALID_ARG;
+    if (m->n_chunks != chunk_count(nbytes, m->chunk_bytes)) return IV_ERR_INVALID_ARG;
+    if (m->n_chunks && !m->d_digests) return IV_ERR_INVALID_ARG;
+    return IV_OK;
+}
+
+// Records phase event `which` (0..3) of the current verification call when timing is on.
+int mark_phase(iv_ctx *ctx, int which, cudaStream_t stream) {
+    if (!ctx->timing) return IV_OK;
+    const uint32_t slot = (uint32_t)(ctx->timed_calls % IV_TIMING_RING);
+    for (int k = 0; k < 4; ++k)
+        if (!ctx->ev_phase[slot][k]) IV_TRY(ctx, cudaEventCreate(&ctx->ev_phase[slot][k]));
+    IV_TRY(ctx, cudaEventRecord(ctx->ev_phase[slot][which], stream));
+    return IV_OK;
+}
+
+// Root + compare, shared by the resident and the streamed verification.
+int finish_verification(iv_ctx *ctx, const iv_manifest *m, iv_verify_result *d_result,
+                        uint64_t *d_mismatch_idx, uint64_t idx_cap, cudaStream_t stream) {
+    const uint64_t n = m->n_chunks;
+    int rc = ensure_merkle_scratch(ctx, n);
+    if (rc != IV_OK) return rc;
+    rc = grow(ctx, &ctx->d_words, &ctx->words_cap, (n + 31) / 32 + 1, sizeof(uint32_t));
+    if (rc != IV_OK) return rc;
+    if ((rc = mark_phase(ctx, 1, stream)) != IV_OK) return rc;
+    IV_TRY(ctx, ivk::launch_merkle_root(ctx->d_digests, n, ctx->d_root, ctx->d_merkle_a, ctx->d_merkle_b,
+                                        ctx->d_tickets, stream, &ctx->launches));
+    if ((rc = mark_phase(ctx, 2, stream)) != IV_OK) return rc;
+    ivk::RootBytes expect;
+    std::memcpy(expect.b, m->root, 32);
+    IV_TRY(ctx, ivk::launch_verify_compare(ctx->d_digests, m->d_digests, n, ctx->d_root, expect, d_result,
+                                           d_mismatch_idx, idx_cap, ctx->d_words,
+                                           ctx->d_tickets + ivk::kMerkleMaxPasses, stream, &ctx->launches));
+    if ((rc = mark_phase(ctx, 3, stream)) != IV_OK) return rc;
+    ctx->slot_timed[ctx->timed_calls % IV_TIMING_RING] = ctx->timing;
+    ++ctx->timed_calls;
+    ctx->digests_valid = n;
+    return IV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *iv_strerror(int code) {
+    switch (code) {
+        case IV_OK: return "ok";
+        case IV_ERR_INVALID_ARG: return "invalid argument";
+        case IV_ERR_NOMEM: return "out of memory";
+        case IV_ERR_CUDA: return "CUDA runtime error";
+        case IV_ERR_NO_DEVICE: return "no usable CUDA device (compute capability 10.x required)";
+        default: return "unknown status";
+    }
+}
+
+int iv_create(iv_ctx **out, int cuda_device) {
+    if (!out) return IV_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || cuda_device < 0 || cuda_device >= count) {
+        (void)cudaGetLastError();
+        return IV_ERR_NO_DEVICE;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cuda_device) != cudaSuccess || prop.major != 10) {
+        (void)cudaGetLastError();
+        return IV_ERR_NO_DEVICE;   // the kernels are built for sm_100a only
+    }
+    iv_ctx *ctx = new (std::nothrow) iv_ctx();
+    if (!ctx) return IV_ERR_NOMEM;
+    ctx->device = cuda_device;
+    ctx->sm_count = prop.multiProcessorCount;
+    DeviceGuard guard(cuda_device);
+
+    const size_t small_bytes = 256;
+    cudaError_t e = cudaMalloc(&ctx->d_small, small_bytes);
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_small, 0, small_bytes);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_hashed[i], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) {
+        int rc = fail_cuda(nullptr, e);
+        iv_destroy(ctx);
+        return rc;
+    }
+    uint8_t *base = static_cast<uint8_t *>(ctx->d_small);
+    ctx->d_root = base;                                                   // 32 bytes
+    ctx->d_queue = reinterpret_cast<unsigned long long *>(base + 64);     // 8 bytes
+    ctx->d_tickets = reinterpret_cast<uint32_t *>(base + 128);            // kMerkleMaxPasses + 1 words
+    *out = ctx;
+    return IV_OK;
+}
+
+int iv_destroy(iv_ctx *ctx) {
+    if (!ctx) return IV_OK;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    cudaFree(ctx->d_small);
+    cudaFree(ctx->d_merkle_a);
+    cudaFree(ctx->d_merkle_b);
+    cudaFree(ctx->d_digests);
+    cudaFree(ctx->d_words);
+    cudaFree(ctx->d_window[0]);
+    cudaFree(ctx->d_window[1]);
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
+        if (ctx->ev_hashed[i]) cudaEventDestroy(ctx->ev_hashed[i]);
+    }
+    for (int r = 0; r < IV_TIMING_RING; ++r)
+        for (int k = 0; k < 4; ++k)
+            if (ctx->ev_phase[r][k]) cudaEventDestroy(ctx->ev_phase[r][k]);
+    (void)cudaGetLastError();
+    delete ctx;
+    return IV_OK;
+}
+
+int iv_last_cuda_error(const iv_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+uint64_t iv_kernel_launches(const iv_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+const uint8_t *iv_ctx_digests(const iv_ctx *ctx) {
+    return (ctx && ctx->digests_valid) ? ctx->d_digests : nullptr;
+}
+
+int iv_hash_chunks(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                   uint8_t *d_digests, uint64_t digests_cap, uint64_t *h_n_chunks, void *cuda_stream) {
+    if (!ctx || chunk_bytes == 0) return IV_ERR_INVALID_ARG;
+    const uint64_t n = chunk_count(nbytes, chunk_bytes);
+    if (n > digests_cap) return IV_ERR_INVALID_ARG;
+    if (n && (!d_data || !d_digests)) return IV_ERR_INVALID_ARG;
+    if (h_n_chunks) *h_n_chunks = n;
+    if (n == 0) return IV_OK;
+    DeviceGuard guard(ctx->device);
+    IV_TRY(ctx, ivk::launch_hash_chunks(static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
+                                        ctx->sm_count, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+    return IV_OK;
+}
+
+int iv_merkle_root(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
+    if (!ctx || !d_root || (n_leaves && !d_leaves)) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    int rc = ensure_merkle_scratch(ctx, n_leaves);
+    if (rc != IV_OK) return rc;
+    IV_TRY(ctx, ivk::launch_merkle_root(d_leaves, n_leaves, d_root, ctx->d_merkle_a, ctx->d_merkle_b,
+                                        ctx->d_tickets, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+    return IV_OK;
+}
+
+int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest *h_manifest,
+                       iv_verify_result *d_result, uint64_t *d_mismatch_idx, uint64_t idx_cap,
+                       void *cuda_stream) {
+    if (!ctx || !d_result || (idx_cap && !d_mismatch_idx)) return IV_ERR_INVALID_ARG;
+    int rc = check_manifest(h_manifest, nbytes);
+    if (rc != IV_OK) return rc;
+    if (nbytes && !d_data) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint64_t n = h_manifest->n_chunks;
+    rc = grow(ctx, &ctx->d_digests, &ctx->digests_cap, n + 1, 32);
+    if (rc != IV_OK) return rc;
+    if ((rc = mark_phase(ctx, 0, stream)) != IV_OK) return rc;
+    IV_TRY(ctx, ivk::launch_hash_chunks(static_cast<const uint8_t *>(d_data), nbytes, h_manifest->chunk_bytes, n,
+                                        ctx->d_digests, ctx->sm_count, stream, &ctx->launches));
+    return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream);
+}
+
+int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_windows, uint64_t window_bytes,
+                       uint64_t nbytes, const iv_manifest *h_manifest, iv_verify_result *d_result,
+                       uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream) {
+    if (!ctx || !d_result || (idx_cap && !d_mismatch_idx)) return IV_ERR_INVALID_ARG;
+    int rc = check_manifest(h_manifest, nbytes);
+    if (rc != IV_OK) return rc;
+    const uint64_t chunk = h_manifest->chunk_bytes;
+    if (window_bytes == 0 || window_bytes % chunk != 0) return IV_ERR_INVALID_ARG;
+    if (n_windows != chunk_count(nbytes, window_bytes)) return IV_ERR_INVALID_ARG;
+    if (n_windows && !h_windows) return IV_ERR_INVALID_ARG;
+    for (uint64_t w = 0; w < n_windows; ++w)
+        if (!h_windows[w]) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint64_t n = h_manifest->n_chunks;
+    rc = grow(ctx, &ctx->d_digests, &ctx->digests_cap, n + 1, 32);
+    if (rc != IV_OK) return rc;
+
+    const uint64_t win = window_bytes < nbytes ? window_bytes : nbytes;
+    if (win > ctx->window_cap) {
+        IV_TRY(ctx, cudaDeviceSynchronize());
+        for (int i = 0; i < 2; ++i) {
+            if (ctx->d_window[i]) IV_TRY(ctx, cudaFree(ctx->d_window[i]));
+            ctx->d_window[i] = nullptr;
+        }
+        ctx->window_cap = 0;
+        for (int i = 0; i < 2; ++i) {
+            void *p = nullptr;
+            IV_TRY(ctx, cudaMalloc(&p, win));
+            ctx->d_window[i] = static_cast<uint8_t *>(p);
+        }
+        ctx->window_cap = win;
+    }
+
+    if ((rc = mark_phase(ctx, 0, stream)) != IV_OK) return rc;
+    // The copy stream starts after everything already enqueued on the caller's
+    // stream (which includes the previous call's use of the windows).
+    IV_TRY(ctx, cudaEventRecord(ctx->ev_entry, stream));
+    IV_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_entry, 0));
+    const uint64_t chunks_per_window = window_bytes / chunk;
+    for (uint64_t w = 0; w < n_windows; ++w) {
+        const int b = (int)(w & 1u);
+        const uint64_t off = w * window_bytes;
+        const uint64_t bytes = nbytes - off < window_bytes ? nbytes - off : window_bytes;
+        if (w >= 2) IV_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_hashed[b], 0));
+        IV_TRY(ctx, cudaMemcpyAsync(ctx->d_window[b], h_windows[w], bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+        IV_TRY(ctx, cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
+        IV_TRY(ctx, cudaStreamWaitEvent(stream, ctx->ev_copied[b], 0));
+        IV_TRY(ctx, ivk::launch_hash_chunks(ctx->d_window[b], bytes, chunk, chunk_count(bytes, chunk),
+                                            ctx->d_digests + 32 * w * chunks_per_window, ctx->sm_count, stream,
+                                            &ctx->launches));
+        IV_TRY(ctx, cudaEventRecord(ctx->ev_hashed[b], stream));
+    }
+    return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream);
+}
+
+int iv_set_timing(iv_ctx *ctx, int enabled) {
+    if (!ctx) return IV_ERR_INVALID_ARG;
+    ctx->timing = enabled != 0;
+    return IV_OK;
+}
+
+int iv_phase_times(iv_ctx *ctx, uint32_t calls_back, float *h_ms) {
+    if (!ctx || !h_ms || calls_back >= IV_TIMING_RING || calls_back >= ctx->timed_calls) return IV_ERR_INVALID_ARG;
+    const uint32_t slot = (uint32_t)((ctx->timed_calls - 1 - calls_back) % IV_TIMING_RING);
+    if (!ctx->slot_timed[slot]) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    IV_TRY(ctx, cudaEventSynchronize(ctx->ev_phase[slot][3]));
+    for (int k = 0; k < 3; ++k)
+        IV_TRY(ctx, cudaEventElapsedTime(&h_ms[k], ctx->ev_phase[slot][k], ctx->ev_phase[slot][k + 1]));
+    return IV_OK;
+}
+
+int iv_hash_ragged(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
+                   uint64_t n, uint8_t *d_digests, void *cuda_stream) {
+    if (!ctx) return IV_ERR_INVALID_ARG;
+    if (n == 0) return IV_OK;
+    if (!d_base || !d_offsets || !d_lengths || !d_digests) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    IV_TRY(ctx, ivk::launch_hash_ragged(static_cast<const uint8_t *>(d_base), d_offsets, d_lengths, n, d_digests,
+                                        ctx->d_queue, ctx->sm_count, static_cast<cudaStream_t>(cuda_stream),
+                                        &ctx->launches));
+    return IV_OK;
+}
+
+int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t blocks_per_sm, uint32_t active_lanes,
+                 uint32_t iters, double *h_out) {
+    if (!ctx || !h_out || warps_per_block == 0 || warps_per_block > 32 || blocks_per_sm == 0 ||
+        blocks_per_sm > 32 || active_lanes == 0 || active_lanes > 32 || iters == 0)
+        return IV_ERR_INVALID_ARG;
+    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_SHA256) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    const unsigned blocks = blocks_per_sm * (unsigned)ctx->sm_count;
+    unsigned long long *d_cycles = nullptr;
+    IV_TRY(ctx, cudaMalloc(&d_cycles, sizeof(unsigned long long) * blocks + 64));
+    uint32_t *d_sink = reinterpret_cast<uint32_t *>(d_cycles + blocks);
+    unsigned long long *h_cycles = static_cast<unsigned long long *>(std::malloc(sizeof(unsigned long long) * blocks));
+    int rc = IV_OK;
+    cudaError_t e = h_cycles ? cudaSuccess : cudaErrorMemoryAllocation;
+    for (int rep = 0; rep < 2 && e == cudaSuccess; ++rep) {   // first launch warms the instruction cache
+        e = ivk::launch_probe(kind, blocks, 32u * warps_per_block, iters, active_lanes, d_cycles, d_sink, nullptr);
+        ++ctx->launches;
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    }
+    if (e == cudaSuccess)
+        e = cudaMemcpy(h_cycles, d_cycles, sizeof(unsigned long long) * blocks, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) {
+        double sum = 0.0;
+        for (unsigned b = 0; b < blocks; ++b) sum += (double)h_cycles[b];
+        const double mean = sum / blocks;
+        double per_thread = (double)ivk::probe_ops_per_thread(kind, iters);
+        if (kind == IV_PROBE_SHA256) per_thread *= 64.0;       // bytes per compression
+        h_out[0] = (double)blocks_per_sm * warps_per_block * active_lanes * per_thread / mean;
+        h_out[1] = mean;
+    } else {
+        rc = fail_cuda(ctx, e);
+    }
+    std::free(h_cycles);
+    cudaFree(d_cycles);
+    return rc;
+}
+
+}  // extern "C"

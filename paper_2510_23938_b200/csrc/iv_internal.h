@@ -1,0 +1,52 @@
+// Internal interfaces between the C-ABI layer (iv_api.cu) and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+#include "../../include/iv.h"
+
+namespace ivk {
+
+// Device-side status values written to iv_verify_result::status.
+enum : uint32_t { IVK_DEV_OK = 0, IVK_DEV_TIMEOUT = 1, IVK_DEV_BOUNDS = 2 };
+
+// Leaves reduced by one CTA of the Merkle kernel (2^9): nine tree levels per pass.
+constexpr uint32_t kMerkleRun = 512;
+
+// hash_chunks.cu -----------------------------------------------------------
+// One SHA-256 per chunk: digest i <- SHA-256(data[i*C .. min((i+1)*C, nbytes))).
+cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                               uint64_t n_chunks, uint8_t *d_digests, int sm_count,
+                               cudaStream_t stream, uint64_t *launches);
+
+// hash_ragged.cu -----------------------------------------------------------
+// One SHA-256 per (offset, length); d_queue is one zeroed uint64 work counter.
+cudaError_t launch_hash_ragged(const uint8_t *d_base, const uint64_t *d_offsets,
+                               const uint64_t *d_lengths, uint64_t n, uint8_t *d_digests,
+                               unsigned long long *d_queue, int sm_count, cudaStream_t stream,
+                               uint64_t *launches);
+
+// merkle.cu ----------------------------------------------------------------
+// Root of n leaves.  d_scratch_a / d_scratch_b each hold ceil(n / kMerkleRun)
+// digests; d_ticket is one zeroed uint32 per pass (kMerkleMaxPasses of them).
+constexpr int kMerkleMaxPasses = 8;
+cudaError_t launch_merkle_root(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root,
+                               uint8_t *d_scratch_a, uint8_t *d_scratch_b, uint32_t *d_tickets,
+                               cudaStream_t stream, uint64_t *launches);
+
+// Compare n computed digests with the manifest's, compact the mismatching
+// indices in ascending order, compare the root.  d_words holds ceil(n/32)
+// uint32 mask words; d_ticket one zeroed uint32.
+struct RootBytes { uint8_t b[32]; };
+cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_manifest_digests,
+                                  uint64_t n, const uint8_t *d_root, RootBytes manifest_root,
+                                  iv_verify_result *d_result, uint64_t *d_mismatch_idx,
+                                  uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
+                                  cudaStream_t stream, uint64_t *launches);
+
+// probe_alu.cu -------------------------------------------------------------
+cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t iters, uint32_t active_lanes,
+                         unsigned long long *d_cycles, uint32_t *d_sink, cudaStream_t stream);
+uint64_t probe_ops_per_thread(int kind, uint32_t iters);
+
+}  // namespace ivk

@@ -1,0 +1,259 @@
+// Merkle reduction of leaf digests to a root, and the comparison of computed
+// digests and root with the manifest (Algorithm 1: "Construct Merkle tree from
+// leaf_hashes using GPU", "Compare root hash with expected value").
+//
+// Tree rule: parent = SHA-256(left || right) over exactly 64 bytes, an unpaired
+// last node moves up unchanged.  Because pairing is index-aligned, any aligned
+// run of 2^k leaves reduces to one node of the global tree on its own, so each
+// CTA reduces a run of 512 leaves through nine levels in shared memory, and the
+// CTA that finishes last (a ticket, no spinning) reduces the run roots.
+#include "iv_internal.h"
+#include "sha256_dev.cuh"
+
+namespace ivk {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// Parent of two nodes held as eight native words each: the first block is the
+// 64 message bytes, the second block is the constant padding of a 64-byte message.
+__device__ __forceinline__ void merkle_parent(const uint32_t *left_right /* 16 words */, uint32_t *out /* 8 words */) {
+    uint32_t st[8], w[16];
+    sha256_init(st);
+    const uint4 *s = reinterpret_cast<const uint4 *>(left_right);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 q = s[i];
+        w[4 * i + 0] = q.x; w[4 * i + 1] = q.y; w[4 * i + 2] = q.z; w[4 * i + 3] = q.w;
+    }
+    sha256_compress(st, w);
+    sha256_pad_only_block(w, 64);
+    sha256_compress(st, w);
+    uint4 *d = reinterpret_cast<uint4 *>(out);
+    d[0] = make_uint4(st[0], st[1], st[2], st[3]);
+    d[1] = make_uint4(st[4], st[5], st[6], st[7]);
+}
+
+// Level-by-level reduction of `count` nodes (8 words each) that sit in buffer a;
+// b is the other half of the ping-pong.  Returns the buffer holding the single root.
+__device__ uint32_t *reduce_in_shared(uint32_t *a, uint32_t *b, uint32_t count) {
+    while (count > 1) {
+        const uint32_t parents = count >> 1;
+        for (uint32_t j = threadIdx.x; j < parents; j += blockDim.x) merkle_parent(a + 16 * j, b + 8 * j);
+        if ((count & 1u) && threadIdx.x < 8) b[8 * parents + threadIdx.x] = a[8 * (count - 1) + threadIdx.x];
+        __syncthreads();
+        uint32_t *t = a; a = b; b = t;
+        count = parents + (count & 1u);
+    }
+    return a;
+}
+
+// Copies `count` digests (byte records, big-endian words) from global memory
+// into shared memory as native words.  `coherent` = the records were written
+// by other CTAs of this launch, so the loads must bypass L1.
+__device__ void load_nodes(const uint8_t *src, uint32_t count, uint32_t *dst, bool coherent) {
+    if ((reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+        const uint4 *s = reinterpret_cast<const uint4 *>(src);
+        for (uint32_t q = threadIdx.x; q < 2 * count; q += blockDim.x) {
+            const uint4 v = coherent ? __ldcg(s + q) : __ldg(s + q);
+            reinterpret_cast<uint4 *>(dst)[q] = make_uint4(bswap32(v.x), bswap32(v.y), bswap32(v.z), bswap32(v.w));
+        }
+    } else {
+        for (uint32_t q = threadIdx.x; q < 8 * count; q += blockDim.x) {
+            const uint8_t *p = src + 4 * (uint64_t)q;
+            dst[q] = ((uint32_t)p[0] << 24) | ((uint32_t)p[1] << 16) | ((uint32_t)p[2] << 8) | (uint32_t)p[3];
+        }
+    }
+    __syncthreads();
+}
+
+__device__ void store_node(uint8_t *dst, const uint32_t *node) {
+    if (threadIdx.x == 0) {
+        uint32_t st[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) st[i] = node[i];
+        store_digest(dst, st);
+    }
+}
+
+// One pass: nodes_in[n] -> nodes_out[ceil(n/512)].  When fuse_top is set (at most
+// 512 run roots) the CTA that takes the last ticket reduces them to d_root too.
+__global__ void __launch_bounds__(kThreads)
+merkle_pass_kernel(const uint8_t *__restrict__ nodes_in, uint64_t n, uint8_t *__restrict__ nodes_out,
+                   uint8_t *__restrict__ d_root, uint32_t *ticket, int fuse_top) {
+    __shared__ __align__(16) uint32_t buf_a[kMerkleRun * 8];
+    __shared__ __align__(16) uint32_t buf_b[kMerkleRun * 4];
+    __shared__ uint32_t s_last;
+
+    const uint64_t runs = (n + kMerkleRun - 1) / kMerkleRun;
+    for (uint64_t r = blockIdx.x; r < runs; r += gridDim.x) {
+        const uint64_t first = r * kMerkleRun;
+        const uint32_t count = (uint32_t)((n - first < kMerkleRun) ? (n - first) : kMerkleRun);
+        load_nodes(nodes_in + 32 * first, count, buf_a, false);
+        const uint32_t *root = reduce_in_shared(buf_a, buf_b, count);
+        // a lone run with fuse_top is already the root of the whole tree
+        store_node((runs == 1 && fuse_top) ? d_root : nodes_out + 32 * r, root);
+        __syncthreads();
+    }
+    if (!fuse_top || runs == 1) return;
+
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    load_nodes(nodes_out, (uint32_t)runs, buf_a, true);
+    const uint32_t *root = reduce_in_shared(buf_a, buf_b, (uint32_t)runs);
+    store_node(d_root, root);
+    if (threadIdx.x == 0) *ticket = 0u;   // ready for the next call
+}
+
+// Root of zero leaves: SHA-256 of the empty string, computed here rather than typed in.
+__global__ void empty_root_kernel(uint8_t *d_root) {
+    uint32_t st[8], w[16];
+    sha256_init(st);
+    sha256_pad_only_block(w, 0);
+    sha256_compress(st, w);
+    store_digest(d_root, st);
+}
+
+// ---------------------------------------------------------------------------
+// Compare + ordered compaction.
+// Each warp compares 32 chunk digests with the manifest and publishes the
+// ballot as one mask word; the CTA that takes the last ticket turns the mask
+// words into the ascending index list with a block-wide exclusive scan.
+// ---------------------------------------------------------------------------
+
+__device__ __forceinline__ bool digest_differs(const uint8_t *a, const uint8_t *b, bool aligned) {
+    if (aligned) {
+        const uint4 a0 = __ldg(reinterpret_cast<const uint4 *>(a)), a1 = __ldg(reinterpret_cast<const uint4 *>(a) + 1);
+        const uint4 b0 = __ldg(reinterpret_cast<const uint4 *>(b)), b1 = __ldg(reinterpret_cast<const uint4 *>(b) + 1);
+        return ((a0.x ^ b0.x) | (a0.y ^ b0.y) | (a0.z ^ b0.z) | (a0.w ^ b0.w) |
+                (a1.x ^ b1.x) | (a1.y ^ b1.y) | (a1.z ^ b1.z) | (a1.w ^ b1.w)) != 0u;
+    }
+    uint32_t diff = 0;
+    for (int i = 0; i < 32; ++i) diff |= (uint32_t)(a[i] ^ b[i]);
+    return diff != 0u;
+}
+
+__global__ void __launch_bounds__(kThreads)
+verify_compare_kernel(const uint8_t *__restrict__ digests, const uint8_t *__restrict__ manifest, uint64_t n,
+                      const uint8_t *__restrict__ d_root, RootBytes manifest_root,
+                      iv_verify_result *__restrict__ result, uint64_t *__restrict__ idx_out, uint64_t idx_cap,
+                      uint32_t *__restrict__ words, uint32_t *ticket) {
+    __shared__ uint32_t s_last;
+    __shared__ uint32_t s_warp_sum[kThreads / 32];
+    __shared__ unsigned long long s_base;
+
+    const bool aligned = (((reinterpret_cast<uintptr_t>(digests) | reinterpret_cast<uintptr_t>(manifest)) & 15u) == 0);
+    const uint64_t n_words = (n + 31) / 32;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t warps_total = (uint64_t)gridDim.x * (kThreads / 32);
+    for (uint64_t wi = (uint64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); wi < n_words; wi += warps_total) {
+        const uint64_t i = wi * 32 + lane;
+        const bool bad = (i < n) && digest_differs(digests + 32 * i, manifest + 32 * i, aligned);
+        const uint32_t mask = __ballot_sync(0xffffffffu, bad);
+        if (lane == 0) words[wi] = mask;
+    }
+
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    if (threadIdx.x == 0) s_base = 0ull;
+    __syncthreads();
+    for (uint64_t tile = 0; tile < n_words; tile += kThreads) {
+        const uint64_t wi = tile + threadIdx.x;
+        const uint32_t mask = (wi < n_words) ? __ldcg(words + wi) : 0u;
+        const uint32_t cnt = __popc(mask);
+        // exclusive scan of cnt across the CTA
+        uint32_t incl = cnt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= (uint32_t)d) incl += up;
+        }
+        if (lane == 31) s_warp_sum[threadIdx.x >> 5] = incl;
+        __syncthreads();
+        uint32_t warp_off = 0, tile_total = 0;
+#pragma unroll
+        for (int k = 0; k < kThreads / 32; ++k) {
+            const uint32_t s = s_warp_sum[k];
+            if (k < (int)(threadIdx.x >> 5)) warp_off += s;
+            tile_total += s;
+        }
+        unsigned long long pos = s_base + warp_off + (incl - cnt);
+        uint32_t m = mask;
+        while (m) {
+            const uint32_t b = __ffs(m) - 1;
+            m &= m - 1;
+            if (pos < idx_cap) idx_out[pos] = wi * 32 + b;
+            ++pos;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) s_base += tile_total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        uint32_t diff = 0;
+        for (int i = 0; i < 32; ++i) {
+            const uint8_t r = d_root[i];
+            result->root[i] = r;
+            diff |= (uint32_t)(r ^ manifest_root.b[i]);
+        }
+        result->status = IVK_DEV_OK;
+        result->root_ok = diff == 0u ? 1u : 0u;
+        result->n_mismatch = s_base;
+        *ticket = 0u;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_merkle_root(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root,
+                               uint8_t *d_scratch_a, uint8_t *d_scratch_b, uint32_t *d_tickets,
+                               cudaStream_t stream, uint64_t *launches) {
+    if (n == 0) {
+        empty_root_kernel<<<1, 1, 0, stream>>>(d_root);
+        if (launches) ++*launches;
+        return cudaGetLastError();
+    }
+    const uint8_t *in = d_leaves;
+    uint8_t *out = d_scratch_a, *other = d_scratch_b;
+    for (int pass = 0; pass < kMerkleMaxPasses; ++pass) {
+        const uint64_t runs = (n + kMerkleRun - 1) / kMerkleRun;
+        const int fuse_top = runs <= kMerkleRun ? 1 : 0;
+        const unsigned grid = (unsigned)(runs < 4096 ? runs : 4096);
+        merkle_pass_kernel<<<grid, kThreads, 0, stream>>>(in, n, out, d_root, d_tickets + pass, fuse_top);
+        if (launches) ++*launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess || fuse_top) return e;
+        in = out;
+        uint8_t *t = out; out = other; other = t;
+        n = runs;
+    }
+    return cudaErrorInvalidValue;   // more than 512^8 leaves cannot be addressed
+}
+
+cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_manifest_digests,
+                                  uint64_t n, const uint8_t *d_root, RootBytes manifest_root,
+                                  iv_verify_result *d_result, uint64_t *d_mismatch_idx,
+                                  uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
+                                  cudaStream_t stream, uint64_t *launches) {
+    const uint64_t n_words = (n + 31) / 32;
+    uint64_t blocks = (n_words + (kThreads / 32) - 1) / (kThreads / 32);
+    if (blocks == 0) blocks = 1;
+    if (blocks > 1184) blocks = 1184;
+    verify_compare_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(
+        d_digests, d_manifest_digests, n, d_root, manifest_root, d_result, d_mismatch_idx, idx_cap,
+        d_words, d_ticket);
+    if (launches) ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace ivk

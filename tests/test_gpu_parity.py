@@ -1,0 +1,288 @@
+"""GPU parity: every digest, root, count and index from the CUDA library equals the CPU oracle's
+on the same seeded bytes (bit-exact: the path is integer and byte work only).  All calls go
+through the C ABI via the ctypes binding."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_23938_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu-marked tests need a CUDA device")
+    c = binding.Context(0)
+    yield c
+    c.close()
+
+
+def _host(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy()
+
+
+def _root_bytes(t: torch.Tensor) -> bytes:
+    return _host(t).tobytes()
+
+
+# ------------------------------------------------------------------------------------------ a2
+
+@pytest.mark.parametrize("nbytes,chunk", [
+    (64 << 20, 64 << 10),            # the small configuration: 1024 leaves
+    (1 << 20, 4096), (1 << 20, 64), (1 << 20, 1 << 20), (1 << 20, 2 << 20),
+    ((1 << 20) + 77, 4096),          # ragged last chunk
+    (100_003, 1000), (100_003, 1001), (100_003, 7), (65, 64), (64, 64), (63, 64), (1, 1), (1, 4096),
+    (5 * 4096 + 56, 4096), (5 * 4096 + 55, 4096), (5 * 4096 + 119, 4096), (5 * 4096 + 120, 4096),
+    (37 * 48 + 16, 48),              # chunk size multiple of 16 but not 64
+])
+def test_hash_chunks_equals_oracle(ctx, nbytes, chunk):
+    data = inputs.uniform_bytes(nbytes, seed=1, device="cuda")
+    got = ctx.hash_chunks(data, chunk)
+    want = oracle.hash_chunks(_host(data), chunk, nthreads=oracle.host_threads())
+    assert got.shape == want.shape
+    assert np.array_equal(_host(got), want)
+
+
+@pytest.mark.parametrize("shift", [1, 2, 3, 4, 5, 8, 13, 15])
+@pytest.mark.parametrize("chunk", [256, 1000, 4096 + 3])
+def test_hash_chunks_any_base_alignment(ctx, shift, chunk):
+    buf = inputs.uniform_bytes(300_000 + 16, seed=11, device="cuda")
+    data = buf[shift:shift + 300_000]
+    got = ctx.hash_chunks(data, chunk)
+    assert np.array_equal(_host(got), oracle.hash_chunks(_host(data), chunk))
+
+
+def test_hash_chunks_empty_and_argument_errors(ctx):
+    data = inputs.uniform_bytes(4096, seed=2, device="cuda")
+    assert ctx.hash_chunks(data[:0], 64).shape == (0, 32)
+    with pytest.raises(binding.IvError) as e:
+        ctx.hash_chunks(data, 0)
+    assert e.value.code == binding.IV_ERR_INVALID_ARG
+    small = torch.empty((3, 32), dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.IvError):
+        ctx.hash_chunks(data, 1024, out=small)      # needs 4 records
+
+
+def test_hash_chunks_window_split_invariance(ctx):
+    """Algorithm 1's loop: hashing window by window into one digest array equals one call."""
+    c, n = 4096, 37
+    data = inputs.uniform_bytes(n * c - 100, seed=3, device="cuda")
+    whole = ctx.hash_chunks(data, c)
+    out = torch.zeros((n, 32), dtype=torch.uint8, device="cuda")
+    win = 8 * c
+    for w, off in enumerate(range(0, data.numel(), win)):
+        ctx.hash_chunks(data[off:off + win], c, out=out[8 * w:])
+    assert torch.equal(out, whole)
+
+
+# ------------------------------------------------------------------------------------------ a3
+
+@pytest.mark.parametrize("n", [0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 31, 32, 33, 255, 256, 257, 511, 512, 513, 1023, 1024, 1025,
+                               2510, 3830, 10_000, 28_672, 512 * 512, 512 * 512 + 5, 300_001])
+def test_merkle_root_equals_oracle(ctx, n):
+    leaves = inputs.uniform_bytes(32 * n, seed=100 + n, device="cuda").view(n, 32)
+    got = _root_bytes(ctx.merkle_root(leaves))
+    assert got == oracle.merkle_root(_host(leaves))
+
+
+def test_merkle_root_unaligned_leaf_pointer(ctx):
+    buf = inputs.uniform_bytes(32 * 700 + 8, seed=5, device="cuda")
+    leaves = buf[3:3 + 32 * 700]
+    assert _root_bytes(ctx.merkle_root(leaves)) == oracle.merkle_root(_host(leaves))
+
+
+def test_merkle_root_repeated_calls_reuse_scratch(ctx):
+    for n in (70_000, 5, 70_000, 1300):
+        leaves = inputs.uniform_bytes(32 * n, seed=n, device="cuda")
+        assert _root_bytes(ctx.merkle_root(leaves)) == oracle.merkle_root(_host(leaves))
+
+
+# ------------------------------------------------------------------------------------------ a4
+
+def _manifest_from_oracle(ctx, host_blob: np.ndarray, chunk: int):
+    digests = oracle.hash_chunks(host_blob, chunk, nthreads=oracle.host_threads())
+    root = oracle.merkle_root(digests)
+    d_dig = torch.from_numpy(digests).cuda()
+    return ctx.make_manifest(host_blob.size, chunk, d_dig, root), digests, root
+
+
+def _verify(ctx, data, manifest, cap):
+    res = binding.new_result("cuda")
+    idx = torch.full((max(cap, 1),), -1, dtype=torch.int64, device="cuda")
+    ctx.verify_manifest(data, manifest, res, idx if cap else None)
+    torch.cuda.synchronize()
+    r = binding.read_result(res)
+    return r, [int(v) for v in idx[:min(cap, r["n_mismatch"])].cpu()]
+
+
+def test_verify_small_configuration_with_three_tampered_copies(ctx):
+    """64 MiB, 64 KiB chunks, manifest from the oracle; three copies with one flipped bit each."""
+    nbytes, chunk = 64 << 20, 64 << 10
+    data = inputs.uniform_bytes(nbytes, seed=1, device="cuda")
+    manifest, digests, root = _manifest_from_oracle(ctx, _host(data), chunk)
+    r, idx = _verify(ctx, data, manifest, 16)
+    assert r == {"status": 0, "root_ok": True, "n_mismatch": 0, "root": root} and idx == []
+    assert np.array_equal(_host(ctx.last_digests(1024)), digests)
+    for seed in (2, 3, 4):
+        off, bit = inputs.flip_position(seed, nbytes)
+        bad = data.clone()
+        bad[off] ^= (1 << bit)
+        r, idx = _verify(ctx, bad, manifest, 16)
+        o_ok, o_bad, o_idx, o_root = oracle.verify(_host(bad), chunk, digests, root, nthreads=oracle.host_threads())
+        assert (r["root_ok"], r["n_mismatch"], idx, r["root"]) == (o_ok, o_bad, o_idx, o_root)
+        assert idx == [off // chunk] and not r["root_ok"]
+
+
+def test_verify_many_mismatches_ascending_exact_count_and_truncation(ctx):
+    chunk, n = 512, 5000
+    data = inputs.uniform_bytes(chunk * n - 17, seed=8, device="cuda")
+    manifest, digests, root = _manifest_from_oracle(ctx, _host(data), chunk)
+    rng = np.random.default_rng(9)
+    hit = np.sort(rng.choice(n, size=777, replace=False))
+    bad = data.clone()
+    bad[torch.from_numpy(hit * chunk + 5).cuda()] ^= 0x40
+    want = oracle.verify(_host(bad), chunk, digests, root, nthreads=oracle.host_threads())
+    r, idx = _verify(ctx, bad, manifest, n)
+    assert (r["root_ok"], r["n_mismatch"], idx, r["root"]) == want
+    assert idx == [int(v) for v in hit]
+    r, idx = _verify(ctx, bad, manifest, 100)
+    assert r["n_mismatch"] == 777 and idx == [int(v) for v in hit[:100]]
+    r, idx = _verify(ctx, bad, manifest, 0)
+    assert r["n_mismatch"] == 777 and idx == []
+    # every chunk wrong
+    allbad = data ^ 0xFF
+    r, idx = _verify(ctx, allbad, manifest, n)
+    assert r["n_mismatch"] == n and idx == list(range(n))
+
+
+def test_verify_manifest_side_tampering_and_argument_checks(ctx):
+    chunk = 1024
+    data = inputs.uniform_bytes(chunk * 70 + 1, seed=12, device="cuda")
+    manifest, digests, root = _manifest_from_oracle(ctx, _host(data), chunk)
+    man2 = digests.copy()
+    man2[33, 0] ^= 1
+    m2 = ctx.make_manifest(data.numel(), chunk, torch.from_numpy(man2).cuda(), root)
+    r, idx = _verify(ctx, data, m2, 8)
+    assert r["root_ok"] and r["n_mismatch"] == 1 and idx == [33]
+    wrong_root = bytes([root[0] ^ 0x80]) + root[1:]
+    m3 = ctx.make_manifest(data.numel(), chunk, torch.from_numpy(digests).cuda(), wrong_root)
+    r, idx = _verify(ctx, data, m3, 8)
+    assert (not r["root_ok"]) and r["n_mismatch"] == 0 and r["root"] == root
+    res = binding.new_result("cuda")
+    with pytest.raises(binding.IvError):                 # manifest for a different size
+        ctx.verify_manifest(data[:-1], manifest, res, None)
+    bad = ctx.make_manifest(data.numel(), chunk, torch.from_numpy(digests[:-1]).cuda(), root)
+    with pytest.raises(binding.IvError):                 # wrong chunk count
+        ctx.verify_manifest(data, bad, res, None)
+
+
+def test_verify_empty_blob(ctx):
+    empty = torch.empty(0, dtype=torch.uint8, device="cuda")
+    root = oracle.merkle_root(b"")
+    m = ctx.make_manifest(0, 4096, empty, root)
+    r, idx = _verify(ctx, empty, m, 4)
+    assert r["root_ok"] and r["n_mismatch"] == 0 and r["root"] == root
+
+
+# ------------------------------------------------------------------------------------------ a5
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_streamed_verification_equals_resident(ctx, pinned):
+    chunk, n = 4096, 301
+    host = inputs.uniform_bytes(chunk * n - 1000, seed=21)
+    if pinned:
+        host = host.pin_memory()
+    manifest, digests, root = _manifest_from_oracle(ctx, host.numpy(), chunk)
+    for window_chunks in (1, 7, 64, 1000):
+        res = binding.new_result("cuda")
+        idx = torch.zeros(8, dtype=torch.int64, device="cuda")
+        ctx.verify_streamed(host, window_chunks * chunk, host.numel(), manifest, res, idx)
+        torch.cuda.synchronize()
+        r = binding.read_result(res)
+        assert r["root_ok"] and r["n_mismatch"] == 0 and r["root"] == root
+        assert np.array_equal(_host(ctx.last_digests(n)), digests)
+    bad = host.clone()
+    bad[chunk * 200 + 9] ^= 2
+    res = binding.new_result("cuda")
+    idx = torch.zeros(8, dtype=torch.int64, device="cuda")
+    ctx.verify_streamed(bad.pin_memory() if pinned else bad, 16 * chunk, bad.numel(), manifest, res, idx)
+    torch.cuda.synchronize()
+    r = binding.read_result(res)
+    assert (not r["root_ok"]) and r["n_mismatch"] == 1 and int(idx[0]) == 200
+    with pytest.raises(binding.IvError):                 # window not a multiple of the chunk size
+        ctx.verify_streamed(host, chunk + 1, host.numel(), manifest, res, idx)
+
+
+# ------------------------------------------------------------------------------------------ a6
+
+def test_hash_ragged_edge_lengths_and_alignments(ctx):
+    base = inputs.uniform_bytes(200_000, seed=31, device="cuda")
+    lengths, offsets = [], []
+    for ln in (0, 1, 2, 3, 4, 55, 56, 57, 63, 64, 65, 119, 120, 121, 127, 128, 129, 1000, 4096, 4097):
+        for o in (0, 1, 2, 3, 5, 6, 7, 9, 13, 15, 16, 17):
+            lengths.append(ln)
+            offsets.append(o + 37 * len(lengths))
+    got = ctx.hash_ragged(base, torch.tensor(offsets, device="cuda"), torch.tensor(lengths, device="cuda"))
+    want = oracle.hash_ragged(_host(base), offsets, lengths, nthreads=oracle.host_threads())
+    assert np.array_equal(_host(got), want)
+
+
+def test_hash_ragged_log_uniform_set_and_root(ctx):
+    """The ragged configuration scaled down: 3000 tensors, log-uniform 64 B .. 256 KiB, packed at 2-byte alignment."""
+    sizes = inputs.ragged_sizes(3000, 64, 256 << 10, seed=5)
+    offs = inputs.packed_offsets(sizes, first=6)
+    total = int(offs[-1] + sizes[-1])
+    base = inputs.uniform_bytes(total + 10, seed=32, device="cuda")
+    got = ctx.hash_ragged(base, torch.from_numpy(offs).cuda(), torch.from_numpy(sizes).cuda())
+    want = oracle.hash_ragged(_host(base), offs, sizes, nthreads=oracle.host_threads())
+    assert np.array_equal(_host(got), want)
+    assert _root_bytes(ctx.merkle_root(got)) == oracle.merkle_root(want)
+
+
+def test_hash_ragged_per_tensor_digests_of_a_weight_file(ctx):
+    blob, table = inputs.weight_file(inputs.tiny_tensors(), seed=7, device="cuda")
+    offs = np.array([o for _, o, _ in table], dtype=np.int64)
+    lens = np.array([n for _, _, n in table], dtype=np.int64)
+    got = ctx.hash_ragged(blob, torch.from_numpy(offs).cuda(), torch.from_numpy(lens).cuda())
+    assert np.array_equal(_host(got), oracle.hash_ragged(_host(blob), offs, lens))
+    # chunk digests of the same file, header included, 4 KiB chunks
+    chunks = ctx.hash_chunks(blob, 4096)
+    assert np.array_equal(_host(chunks), oracle.hash_chunks(_host(blob), 4096))
+
+
+def test_hash_ragged_empty_set(ctx):
+    base = inputs.uniform_bytes(64, seed=1, device="cuda")
+    e = torch.empty(0, dtype=torch.int64, device="cuda")
+    assert ctx.hash_ragged(base, e, e).shape == (0, 32)
+
+
+def test_streamed_windows_may_repeat_and_phase_times_are_reported(ctx):
+    """A ring of two host windows read three times each: the blob is periodic; timing brackets the phases."""
+    chunk, per_win = 4096, 16
+    ring = [inputs.uniform_bytes(chunk * per_win, seed=40 + k).pin_memory() for k in range(2)]
+    windows = [ring[w % 2] for w in range(6)]
+    whole = torch.cat(windows).numpy()
+    manifest, digests, root = _manifest_from_oracle(ctx, whole, chunk)
+    res = binding.new_result("cuda")
+    ctx.set_timing(True)
+    ctx.verify_streamed(windows, chunk * per_win, whole.size, manifest, res, None)
+    torch.cuda.synchronize()
+    ms = ctx.phase_times(0)
+    ctx.set_timing(False)
+    r = binding.read_result(res)
+    assert r["root_ok"] and r["n_mismatch"] == 0 and r["root"] == root
+    assert all(t >= 0.0 for t in ms) and ms[0] > 0.0
+    ctx.verify_manifest(torch.from_numpy(whole).cuda(), manifest, res, None)
+    with pytest.raises(binding.IvError):
+        ctx.phase_times(0)                       # timing was off for that call
+
+
+def test_launch_counter_counts_kernels(ctx):
+    before = ctx.kernel_launches
+    data = inputs.uniform_bytes(1 << 16, seed=1, device="cuda")
+    d = ctx.hash_chunks(data, 1024)
+    ctx.merkle_root(d)
+    assert ctx.kernel_launches == before + 2
