@@ -43,39 +43,75 @@ __device__ __forceinline__ void sha256_init(uint32_t (&st)[8]) {
     st[4] = IV_H0_4; st[5] = IV_H0_5; st[6] = IV_H0_6; st[7] = IV_H0_7;
 }
 
-// One round: T1 = h + S1(e) + Ch(e,f,g) + K + W;  d += T1;  h = T1 + S0(a) + Maj(a,b,c).
+// Two-input add on a chosen pipe.  The INT32 ALU pipe (SHF, LOP3, PRMT, IADD3) is what bounds
+// SHA-256; an integer multiply-add runs on the FMA pipe, which is otherwise idle here, so
+// "a * one + b" with a multiplier the compiler cannot see (a kernel argument equal to 1)
+// moves the add off the ALU pipe.  FMA = false gives the plain add.
+template <bool FMA>
+__device__ __forceinline__ uint32_t padd(uint32_t a, uint32_t b, uint32_t one) {
+    if (FMA) {
+        uint32_t r;
+        asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(one), "r"(b));
+        return r;
+    }
+    return a + b;
+}
+
+// One round (FIPS 180-4 section 6.2.2 step 3):
+//   T1 = h + S1(e) + Ch(e,f,g) + K + W;  d += T1;  h = T1 + S0(a) + Maj(a,b,c).
 // The caller rotates the variable names instead of moving values.
-#define IV_ROUND(a, b, c, d, e, f, g, h, kw)                          \
-    do {                                                              \
-        uint32_t t1_ = (h) + ivk::big_s1(e) + ivk::f_ch(e, f, g) + (kw); \
-        (d) += t1_;                                                   \
-        (h) = t1_ + ivk::big_s0(a) + ivk::f_maj(a, b, c);             \
-    } while (0)
+template <bool FMA>
+__device__ __forceinline__ void sha_round(uint32_t a, uint32_t b, uint32_t c, uint32_t &d, uint32_t e, uint32_t f,
+                                          uint32_t g, uint32_t &h, uint32_t k, uint32_t w, uint32_t one) {
+    if (FMA) {
+        const uint32_t kw = padd<true>(w, k, one);
+        const uint32_t x = padd<true>(h, kw, one);
+        const uint32_t y = padd<true>(x, f_ch(e, f, g), one);
+        const uint32_t t1 = padd<true>(y, big_s1(e), one);
+        const uint32_t q = padd<true>(big_s0(a), f_maj(a, b, c), one);
+        d = padd<true>(d, t1, one);
+        h = padd<true>(t1, q, one);
+    } else {
+        const uint32_t t1 = h + big_s1(e) + f_ch(e, f, g) + (k + w);
+        d += t1;
+        h = t1 + big_s0(a) + f_maj(a, b, c);
+    }
+}
 
 // Message-schedule step in the rolling 16-word window (i = t mod 16):
 // W[t] = s1(W[t-2]) + W[t-7] + s0(W[t-15]) + W[t-16].
-#define IV_SCHED(w, i) \
-    ((w)[(i) & 15] += ivk::small_s1((w)[((i) + 14) & 15]) + (w)[((i) + 9) & 15] + ivk::small_s0((w)[((i) + 1) & 15]))
+template <bool FMA>
+__device__ __forceinline__ void sha_sched(uint32_t (&w)[16], int i, uint32_t one) {
+    const uint32_t s = padd<FMA>(small_s1(w[(i + 14) & 15]), w[(i + 9) & 15], one);
+    const uint32_t t = padd<FMA>(small_s0(w[(i + 1) & 15]), w[i & 15], one);
+    w[i & 15] = padd<FMA>(s, t, one);
+}
+
+#define IV_ROUND(a, b, c, d, e, f, g, h, k, wv) ivk::sha_round<FMA>(a, b, c, d, e, f, g, h, k, wv, one)
 
 // Eight rounds starting at a round index that is a multiple of 8 (so the
 // variable rotation returns to a..h), constants k0..k7 from FIPS 180-4 4.2.2.
-#define IV_ROUNDS8(v, w, i, k0, k1, k2, k3, k4, k5, k6, k7)                                  \
-    IV_ROUND(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], (k0) + (w)[((i) + 0) & 15]);   \
-    IV_ROUND(v[7], v[0], v[1], v[2], v[3], v[4], v[5], v[6], (k1) + (w)[((i) + 1) & 15]);   \
-    IV_ROUND(v[6], v[7], v[0], v[1], v[2], v[3], v[4], v[5], (k2) + (w)[((i) + 2) & 15]);   \
-    IV_ROUND(v[5], v[6], v[7], v[0], v[1], v[2], v[3], v[4], (k3) + (w)[((i) + 3) & 15]);   \
-    IV_ROUND(v[4], v[5], v[6], v[7], v[0], v[1], v[2], v[3], (k4) + (w)[((i) + 4) & 15]);   \
-    IV_ROUND(v[3], v[4], v[5], v[6], v[7], v[0], v[1], v[2], (k5) + (w)[((i) + 5) & 15]);   \
-    IV_ROUND(v[2], v[3], v[4], v[5], v[6], v[7], v[0], v[1], (k6) + (w)[((i) + 6) & 15]);   \
-    IV_ROUND(v[1], v[2], v[3], v[4], v[5], v[6], v[7], v[0], (k7) + (w)[((i) + 7) & 15])
+#define IV_ROUNDS8(v, w, i, k0, k1, k2, k3, k4, k5, k6, k7)                           \
+    IV_ROUND(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], k0, (w)[((i) + 0) & 15]); \
+    IV_ROUND(v[7], v[0], v[1], v[2], v[3], v[4], v[5], v[6], k1, (w)[((i) + 1) & 15]); \
+    IV_ROUND(v[6], v[7], v[0], v[1], v[2], v[3], v[4], v[5], k2, (w)[((i) + 2) & 15]); \
+    IV_ROUND(v[5], v[6], v[7], v[0], v[1], v[2], v[3], v[4], k3, (w)[((i) + 3) & 15]); \
+    IV_ROUND(v[4], v[5], v[6], v[7], v[0], v[1], v[2], v[3], k4, (w)[((i) + 4) & 15]); \
+    IV_ROUND(v[3], v[4], v[5], v[6], v[7], v[0], v[1], v[2], k5, (w)[((i) + 5) & 15]); \
+    IV_ROUND(v[2], v[3], v[4], v[5], v[6], v[7], v[0], v[1], k6, (w)[((i) + 6) & 15]); \
+    IV_ROUND(v[1], v[2], v[3], v[4], v[5], v[6], v[7], v[0], k7, (w)[((i) + 7) & 15])
 
-#define IV_SCHED8(w, i)                                                          \
-    IV_SCHED(w, (i) + 0); IV_SCHED(w, (i) + 1); IV_SCHED(w, (i) + 2); IV_SCHED(w, (i) + 3); \
-    IV_SCHED(w, (i) + 4); IV_SCHED(w, (i) + 5); IV_SCHED(w, (i) + 6); IV_SCHED(w, (i) + 7)
+#define IV_SCHED8(w, i)                                                                      \
+    ivk::sha_sched<FMA>(w, (i) + 0, one); ivk::sha_sched<FMA>(w, (i) + 1, one);               \
+    ivk::sha_sched<FMA>(w, (i) + 2, one); ivk::sha_sched<FMA>(w, (i) + 3, one);               \
+    ivk::sha_sched<FMA>(w, (i) + 4, one); ivk::sha_sched<FMA>(w, (i) + 5, one);               \
+    ivk::sha_sched<FMA>(w, (i) + 6, one); ivk::sha_sched<FMA>(w, (i) + 7, one)
 
 // st <- compress(st, block) where w[0..15] holds the block as big-endian words.
-// w is destroyed (it is the rolling schedule window).
-__device__ __forceinline__ void sha256_compress(uint32_t (&st)[8], uint32_t (&w)[16]) {
+// w is destroyed (it is the rolling schedule window).  With FMA = true every
+// addition is issued on the FMA pipe; `one` must then hold the value 1.
+template <bool FMA = false>
+__device__ __forceinline__ void sha256_compress(uint32_t (&st)[8], uint32_t (&w)[16], uint32_t one = 1u) {
     uint32_t v[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = st[i];
@@ -96,7 +132,7 @@ __device__ __forceinline__ void sha256_compress(uint32_t (&st)[8], uint32_t (&w)
     IV_ROUNDS8(v, w, 8, 0x748f82eeu, 0x78a5636fu, 0x84c87814u, 0x8cc70208u, 0x90befffau, 0xa4506cebu, 0xbef9a3f7u, 0xc67178f2u);
 
 #pragma unroll
-    for (int i = 0; i < 8; ++i) st[i] += v[i];
+    for (int i = 0; i < 8; ++i) st[i] = padd<FMA>(st[i], v[i], one);
 }
 
 // The last block of a message whose length is a multiple of 64 bytes holds no
