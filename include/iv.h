@@ -61,6 +61,13 @@ const char *iv_strerror(int code);
 /* The cudaError_t (as int) of the last failed CUDA call on this context, 0 if none. */
 int iv_last_cuda_error(const iv_ctx *ctx);
 
+/* Device-side status of the kernels this context has run: 0 = all completed,
+ * 1 = a kernel gave up on a bounded wait for a bulk copy (its outputs are then
+ * invalid), 2 = an index check failed.  Waits for the device (synchronous),
+ * writes the word to *h_status and clears it.  Verification calls also copy it
+ * into iv_verify_result::status. */
+int iv_device_status(iv_ctx *ctx, uint32_t *h_status);
+
 /* Number of kernels this context has launched so far (a host-side counter). */
 uint64_t iv_kernel_launches(const iv_ctx *ctx);
 
@@ -211,7 +218,8 @@ typedef enum iv_probe_kind {
     IV_PROBE_PRMT = 3,   /* byte permute */
     IV_PROBE_IMAD = 4,   /* integer multiply-add */
     IV_PROBE_MIXED = 5,  /* LOP3 and IMAD interleaved 1:1 */
-    IV_PROBE_SHA256 = 6  /* full SHA-256 compressions, registers only */
+    IV_PROBE_SHA256 = 6,     /* full SHA-256 compressions, registers only */
+    IV_PROBE_SHA256_FMA = 7  /* the same with every addition issued as a multiply-add (FMA pipe) */
 } iv_probe_kind;
 int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t blocks_per_sm,
                  uint32_t active_lanes, uint32_t iters, double *h_out);

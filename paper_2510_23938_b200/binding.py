@@ -25,7 +25,7 @@ IV_ERR_NO_DEVICE = -4
 EXPORTS = (
     "iv_create", "iv_destroy", "iv_strerror", "iv_last_cuda_error", "iv_kernel_launches",
     "iv_hash_chunks", "iv_merkle_root", "iv_verify_manifest", "iv_ctx_digests",
-    "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu",
+    "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
 )
 
 
@@ -91,6 +91,8 @@ def load_library() -> ctypes.CDLL:
     lib.iv_phase_times.restype = i32
     lib.iv_hash_ragged.argtypes = [vp, vp, vp, vp, u64, vp, vp]
     lib.iv_hash_ragged.restype = i32
+    lib.iv_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.iv_device_status.restype = i32
     lib.iv_probe_alu.argtypes = [vp, i32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
                                  ctypes.POINTER(ctypes.c_double)]
     lib.iv_probe_alu.restype = i32
@@ -248,7 +250,13 @@ class Context:
         self._check(rc, "iv_hash_ragged")
         return out
 
-    PROBE_KINDS = {"iadd3": 0, "lop3": 1, "shf": 2, "prmt": 3, "imad": 4, "mixed": 5, "sha256": 6}
+    def device_status(self) -> int:
+        """iv_device_status: waits for the device, returns and clears the device-side status word."""
+        st = ctypes.c_uint32(0)
+        self._check(self._lib.iv_device_status(self._h, ctypes.byref(st)), "iv_device_status")
+        return int(st.value)
+
+    PROBE_KINDS = {"iadd3": 0, "lop3": 1, "shf": 2, "prmt": 3, "imad": 4, "mixed": 5, "sha256": 6, "sha256_fma": 7}
 
     def probe_alu(self, kind: str, warps_per_block: int = 4, blocks_per_sm: int = 1, active_lanes: int = 32,
                   iters: int = 2000) -> tuple[float, float]:

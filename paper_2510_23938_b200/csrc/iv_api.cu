@@ -16,6 +16,7 @@ struct iv_ctx {
     uint32_t *d_tickets = nullptr;            // kMerkleMaxPasses + 1 words
     unsigned long long *d_queue = nullptr;
     uint8_t *d_root = nullptr;                // 32 bytes
+    uint32_t *d_status = nullptr;             // device-side status word (0 = ok), sticky until read
     void *d_small = nullptr;
 
     // lazily sized scratch
@@ -132,7 +133,8 @@ int finish_verification(iv_ctx *ctx, const iv_manifest *m, iv_verify_result *d_r
     std::memcpy(expect.b, m->root, 32);
     IV_TRY(ctx, ivk::launch_verify_compare(ctx->d_digests, m->d_digests, n, ctx->d_root, expect, d_result,
                                            d_mismatch_idx, idx_cap, ctx->d_words,
-                                           ctx->d_tickets + ivk::kMerkleMaxPasses, stream, &ctx->launches));
+                                           ctx->d_tickets + ivk::kMerkleMaxPasses, ctx->d_status, stream,
+                                           &ctx->launches));
     if ((rc = mark_phase(ctx, 3, stream)) != IV_OK) return rc;
     ctx->slot_timed[ctx->timed_calls % IV_TIMING_RING] = ctx->timing;
     ++ctx->timed_calls;
@@ -192,6 +194,7 @@ int iv_create(iv_ctx **out, int cuda_device) {
     ctx->d_root = base;                                                   // 32 bytes
     ctx->d_queue = reinterpret_cast<unsigned long long *>(base + 64);     // 8 bytes
     ctx->d_tickets = reinterpret_cast<uint32_t *>(base + 128);            // kMerkleMaxPasses + 1 words
+    ctx->d_status = reinterpret_cast<uint32_t *>(base + 192);
     *out = ctx;
     return IV_OK;
 }
@@ -225,6 +228,15 @@ int iv_last_cuda_error(const iv_ctx *ctx) { return ctx ? ctx->last_cuda_error : 
 
 uint64_t iv_kernel_launches(const iv_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
+int iv_device_status(iv_ctx *ctx, uint32_t *h_status) {
+    if (!ctx || !h_status) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    IV_TRY(ctx, cudaDeviceSynchronize());
+    IV_TRY(ctx, cudaMemcpy(h_status, ctx->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (*h_status != 0) IV_TRY(ctx, cudaMemset(ctx->d_status, 0, sizeof(uint32_t)));
+    return IV_OK;
+}
+
 const uint8_t *iv_ctx_digests(const iv_ctx *ctx) {
     return (ctx && ctx->digests_valid) ? ctx->d_digests : nullptr;
 }
@@ -239,7 +251,7 @@ int iv_hash_chunks(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t ch
     if (n == 0) return IV_OK;
     DeviceGuard guard(ctx->device);
     IV_TRY(ctx, ivk::launch_hash_chunks(static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
-                                        ctx->sm_count, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+                                        ctx->sm_count, ctx->d_status, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
     return IV_OK;
 }
 
@@ -267,7 +279,7 @@ int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const i
     if (rc != IV_OK) return rc;
     if ((rc = mark_phase(ctx, 0, stream)) != IV_OK) return rc;
     IV_TRY(ctx, ivk::launch_hash_chunks(static_cast<const uint8_t *>(d_data), nbytes, h_manifest->chunk_bytes, n,
-                                        ctx->d_digests, ctx->sm_count, stream, &ctx->launches));
+                                        ctx->d_digests, ctx->sm_count, ctx->d_status, stream, &ctx->launches));
     return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream);
 }
 
@@ -320,7 +332,7 @@ int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_win
         IV_TRY(ctx, cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
         IV_TRY(ctx, cudaStreamWaitEvent(stream, ctx->ev_copied[b], 0));
         IV_TRY(ctx, ivk::launch_hash_chunks(ctx->d_window[b], bytes, chunk, chunk_count(bytes, chunk),
-                                            ctx->d_digests + 32 * w * chunks_per_window, ctx->sm_count, stream,
+                                            ctx->d_digests + 32 * w * chunks_per_window, ctx->sm_count, ctx->d_status, stream,
                                             &ctx->launches));
         IV_TRY(ctx, cudaEventRecord(ctx->ev_hashed[b], stream));
     }
@@ -361,7 +373,7 @@ int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t block
     if (!ctx || !h_out || warps_per_block == 0 || warps_per_block > 32 || blocks_per_sm == 0 ||
         blocks_per_sm > 32 || active_lanes == 0 || active_lanes > 32 || iters == 0)
         return IV_ERR_INVALID_ARG;
-    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_SHA256) return IV_ERR_INVALID_ARG;
+    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_SHA256_FMA) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     const unsigned blocks = blocks_per_sm * (unsigned)ctx->sm_count;
     unsigned long long *d_cycles = nullptr;
@@ -382,7 +394,7 @@ int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t block
         for (unsigned b = 0; b < blocks; ++b) sum += (double)h_cycles[b];
         const double mean = sum / blocks;
         double per_thread = (double)ivk::probe_ops_per_thread(kind, iters);
-        if (kind == IV_PROBE_SHA256) per_thread *= 64.0;       // bytes per compression
+        if (kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_FMA) per_thread *= 64.0;       // bytes per compression
         h_out[0] = (double)blocks_per_sm * warps_per_block * active_lanes * per_thread / mean;
         h_out[1] = mean;
     } else {

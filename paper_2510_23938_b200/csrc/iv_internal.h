@@ -16,7 +16,7 @@ constexpr uint32_t kMerkleRun = 512;
 // hash_chunks.cu -----------------------------------------------------------
 // One SHA-256 per chunk: digest i <- SHA-256(data[i*C .. min((i+1)*C, nbytes))).
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
-                               uint64_t n_chunks, uint8_t *d_digests, int sm_count,
+                               uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
                                cudaStream_t stream, uint64_t *launches);
 
 // hash_ragged.cu -----------------------------------------------------------
@@ -42,7 +42,7 @@ cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_man
                                   uint64_t n, const uint8_t *d_root, RootBytes manifest_root,
                                   iv_verify_result *d_result, uint64_t *d_mismatch_idx,
                                   uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
-                                  cudaStream_t stream, uint64_t *launches);
+                                  const uint32_t *d_status, cudaStream_t stream, uint64_t *launches);
 
 // probe_alu.cu -------------------------------------------------------------
 cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t iters, uint32_t active_lanes,

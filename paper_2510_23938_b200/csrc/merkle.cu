@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(kThreads)
 verify_compare_kernel(const uint8_t *__restrict__ digests, const uint8_t *__restrict__ manifest, uint64_t n,
                       const uint8_t *__restrict__ d_root, RootBytes manifest_root,
                       iv_verify_result *__restrict__ result, uint64_t *__restrict__ idx_out, uint64_t idx_cap,
-                      uint32_t *__restrict__ words, uint32_t *ticket) {
+                      uint32_t *__restrict__ words, uint32_t *ticket, const uint32_t *__restrict__ dev_status) {
     __shared__ uint32_t s_last;
     __shared__ uint32_t s_warp_sum[kThreads / 32];
     __shared__ unsigned long long s_base;
@@ -206,7 +206,7 @@ verify_compare_kernel(const uint8_t *__restrict__ digests, const uint8_t *__rest
             result->root[i] = r;
             diff |= (uint32_t)(r ^ manifest_root.b[i]);
         }
-        result->status = IVK_DEV_OK;
+        result->status = __ldcg(dev_status);   // nonzero if a kernel of this context gave up on a wait
         result->root_ok = diff == 0u ? 1u : 0u;
         result->n_mismatch = s_base;
         *ticket = 0u;
@@ -244,14 +244,14 @@ cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_man
                                   uint64_t n, const uint8_t *d_root, RootBytes manifest_root,
                                   iv_verify_result *d_result, uint64_t *d_mismatch_idx,
                                   uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
-                                  cudaStream_t stream, uint64_t *launches) {
+                                  const uint32_t *d_status, cudaStream_t stream, uint64_t *launches) {
     const uint64_t n_words = (n + 31) / 32;
     uint64_t blocks = (n_words + (kThreads / 32) - 1) / (kThreads / 32);
     if (blocks == 0) blocks = 1;
     if (blocks > 1184) blocks = 1184;
     verify_compare_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(
         d_digests, d_manifest_digests, n, d_root, manifest_root, d_result, d_mismatch_idx, idx_cap,
-        d_words, d_ticket);
+        d_words, d_ticket, d_status);
     if (launches) ++*launches;
     return cudaGetLastError();
 }

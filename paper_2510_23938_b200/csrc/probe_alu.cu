@@ -69,7 +69,9 @@ __global__ void probe_kernel(uint32_t iters, uint32_t active_lanes, uint32_t see
 }
 
 // Register-only SHA-256: `iters` compressions per thread on a block derived from the state.
-__global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, unsigned long long *cycles, uint32_t *sink) {
+template <bool FMA>
+__global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, uint32_t one, unsigned long long *cycles,
+                                 uint32_t *sink) {
     const uint32_t lane = threadIdx.x & 31u;
     uint32_t st[8], w[16];
     sha256_init(st);
@@ -80,7 +82,7 @@ __global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, unsigned
         for (uint32_t it = 0; it < iters; ++it) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) w[i] = __byte_perm(st[i & 7] + (uint32_t)i, it, 0x0123);
-            sha256_compress(st, w);
+            sha256_compress<FMA>(st, w, one);
         }
     }
     __syncthreads();
@@ -101,14 +103,15 @@ cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t i
         case IV_PROBE_PRMT: probe_kernel<IV_PROBE_PRMT><<<blocks, threads, 0, stream>>>(iters, active_lanes, sb, 0x0123u, d_cycles, d_sink); break;
         case IV_PROBE_IMAD: probe_kernel<IV_PROBE_IMAD><<<blocks, threads, 0, stream>>>(iters, active_lanes, sb, sc, d_cycles, d_sink); break;
         case IV_PROBE_MIXED: probe_kernel<IV_PROBE_MIXED><<<blocks, threads, 0, stream>>>(iters, active_lanes, sb, sc, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256: probe_sha_kernel<<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256: probe_sha_kernel<false><<<blocks, threads, 0, stream>>>(iters, active_lanes, 1u, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_FMA: probe_sha_kernel<true><<<blocks, threads, 0, stream>>>(iters, active_lanes, 1u, d_cycles, d_sink); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
 }
 
 uint64_t probe_ops_per_thread(int kind, uint32_t iters) {
-    if (kind == IV_PROBE_SHA256) return iters;                       // compressions
+    if (kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_FMA) return iters;                       // compressions
     return (uint64_t)iters * kUnroll * kChains;                      // instructions
 }
 

@@ -37,6 +37,10 @@ def _root_bytes(t: torch.Tensor) -> bytes:
     (100_003, 1000), (100_003, 1001), (100_003, 7), (65, 64), (64, 64), (63, 64), (1, 1), (1, 4096),
     (5 * 4096 + 56, 4096), (5 * 4096 + 55, 4096), (5 * 4096 + 119, 4096), (5 * 4096 + 120, 4096),
     (37 * 48 + 16, 48),              # chunk size multiple of 16 but not 64
+    (50 * (4096 + 16) + 8, 4096 + 16),   # staged path with a 16-byte remainder in every chunk
+    (33 * 8192 + 4100, 8192), (3 * 65536 + 300, 65536 + 48),
+    (20_000 * 4096 + 100, 4096),     # more than 592 warps: the many-chain launch shape, ragged last chunk
+    (19_000 * 4096, 4096),
 ])
 def test_hash_chunks_equals_oracle(ctx, nbytes, chunk):
     data = inputs.uniform_bytes(nbytes, seed=1, device="cuda")
@@ -278,6 +282,10 @@ def test_streamed_windows_may_repeat_and_phase_times_are_reported(ctx):
     ctx.verify_manifest(torch.from_numpy(whole).cuda(), manifest, res, None)
     with pytest.raises(binding.IvError):
         ctx.phase_times(0)                       # timing was off for that call
+
+
+def test_device_status_is_clean_after_all_of_the_above(ctx):
+    assert ctx.device_status() == 0
 
 
 def test_launch_counter_counts_kernels(ctx):
