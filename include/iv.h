@@ -41,7 +41,8 @@ typedef enum iv_status {
     IV_ERR_INVALID_ARG = -1, /* null pointer, zero chunk size, capacity too small, inconsistent manifest */
     IV_ERR_NOMEM = -2,       /* a device or host allocation for scratch failed */
     IV_ERR_CUDA = -3,        /* a CUDA runtime call failed; see iv_last_cuda_error */
-    IV_ERR_NO_DEVICE = -4    /* no CUDA device, or not a compute-capability-10.x device */
+    IV_ERR_NO_DEVICE = -4,   /* no CUDA device, or not a compute-capability-10.x device */
+    IV_ERR_TOO_LARGE = -5    /* the size exceeds a fixed limit of the entry point (iv_merkle_root_noalloc) */
 } iv_status;
 
 /* Opaque context.  Owns scratch memory (Merkle level buffers, tickets, the
@@ -195,6 +196,33 @@ int iv_phase_times(iv_ctx *ctx, uint32_t calls_back, float *h_ms);
 int iv_hash_ragged(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets,
                    const uint64_t *d_lengths, uint64_t n, uint8_t *d_digests,
                    void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Merkle root without allocation (the paper has no counterpart; this exists
+ * for callers of this library, see below).
+ *
+ * Same result as iv_merkle_root, for callers that cannot allocate device
+ * memory: code running inside a framework whose memory pool already owns the
+ * whole GPU, a serving loop that must never block on the allocator, a process
+ * that may only use buffers handed to it.  It needs no iv_ctx (creating one
+ * allocates) and calls no cudaMalloc, cudaFree or other allocating routine.
+ * Its scratch -- 512 intermediate digests and a ticket word -- lives in a
+ * fixed 16.25 KiB array inside the library image, which every GPU that loads
+ * the library holds until the process exits.
+ *
+ *   d_leaves, d_root   as for iv_merkle_root; the caller supplies both
+ *   n_leaves           at most IV_NOALLOC_MAX_LEAVES (512 * 512); more returns
+ *                      IV_ERR_TOO_LARGE and launches nothing
+ * Work is enqueued on cuda_stream for the CURRENT device.  The first call on
+ * a device looks up the device address of the array (once per device); make
+ * that first call before starting any stream capture.  All calls share the
+ * one array, which keeps the previous call's contents (the entry point clears
+ * the one word that must start at zero): calls that overlap on the GPU --
+ * two streams, two threads -- race and give wrong roots; serialise them.
+ */
+#define IV_NOALLOC_MAX_LEAVES (512ull * 512ull)
+int iv_merkle_root_noalloc(const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
+                           void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
  * Roofline probe (a measurement aid; the paper has no counterpart).  Runs a

@@ -21,11 +21,14 @@ IV_ERR_INVALID_ARG = -1
 IV_ERR_NOMEM = -2
 IV_ERR_CUDA = -3
 IV_ERR_NO_DEVICE = -4
+IV_ERR_TOO_LARGE = -5
+NOALLOC_MAX_LEAVES = 512 * 512
 
 EXPORTS = (
     "iv_create", "iv_destroy", "iv_strerror", "iv_last_cuda_error", "iv_kernel_launches",
     "iv_hash_chunks", "iv_merkle_root", "iv_verify_manifest", "iv_ctx_digests",
     "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
+    "iv_merkle_root_noalloc",
 )
 
 
@@ -91,6 +94,8 @@ def load_library() -> ctypes.CDLL:
     lib.iv_phase_times.restype = i32
     lib.iv_hash_ragged.argtypes = [vp, vp, vp, vp, u64, vp, vp]
     lib.iv_hash_ragged.restype = i32
+    lib.iv_merkle_root_noalloc.argtypes = [vp, u64, vp, vp]
+    lib.iv_merkle_root_noalloc.restype = i32
     lib.iv_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.iv_device_status.restype = i32
     lib.iv_probe_alu.argtypes = [vp, i32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
@@ -284,6 +289,21 @@ class _DeviceBytes:
     def __init__(self, ptr: int, nbytes: int):
         self.__cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|u1", "data": (int(ptr), False),
                                          "version": 2}
+
+
+def merkle_root_noalloc(leaves: torch.Tensor, out: torch.Tensor, n_leaves: int | None = None, stream=None) -> torch.Tensor:
+    """iv_merkle_root_noalloc: Merkle root into the caller's 32-byte device tensor `out`.
+
+    For callers that cannot allocate on the device (a pool owns the GPU, or the allocator must not
+    be touched): no context, no allocation in the library, and none here -- both tensors are the
+    caller's.  At most NOALLOC_MAX_LEAVES leaves; calls must not overlap on the GPU."""
+    lib = load_library()
+    n = leaves.numel() // 32 if n_leaves is None else int(n_leaves)
+    assert out.is_cuda and out.is_contiguous() and out.numel() >= 32
+    rc = lib.iv_merkle_root_noalloc(_dev_ptr(leaves), n, out.data_ptr(), _stream_ptr(stream))
+    if rc != IV_OK:
+        raise IvError(rc, "iv_merkle_root_noalloc")
+    return out
 
 
 def read_result(result: torch.Tensor) -> dict:

@@ -153,6 +153,7 @@ const char *iv_strerror(int code) {
         case IV_ERR_NOMEM: return "out of memory";
         case IV_ERR_CUDA: return "CUDA runtime error";
         case IV_ERR_NO_DEVICE: return "no usable CUDA device (compute capability 10.x required)";
+        case IV_ERR_TOO_LARGE: return "size exceeds the fixed limit of this entry point";
         default: return "unknown status";
     }
 }

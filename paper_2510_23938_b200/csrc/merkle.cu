@@ -257,3 +257,63 @@ cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_man
 }
 
 }  // namespace ivk
+
+// ---------------------------------------------------------------------------
+// Merkle root for callers that must not allocate.
+//
+// iv_merkle_root keeps the run roots and the ticket in memory that iv_create
+// and the first large call obtain with cudaMalloc.  Code that runs where device
+// allocation is forbidden or impossible -- inside a memory pool that already
+// owns the whole device, in a latency-critical serving loop that may not touch
+// the allocator's lock, after a fork where only pre-made buffers may be used --
+// cannot call it.  This variant keeps the same scratch in a fixed array that is
+// part of the library image, so every GPU that loads the library carries these
+// 16.25 KiB until the process exits, and the number of leaves is capped.
+// ---------------------------------------------------------------------------
+
+// 512 run roots of 32 bytes, then the ticket word (offset 16384).
+static __device__ __align__(256) unsigned char iv_noalloc_scratch[ivk::kMerkleRun * 32 + 256];
+
+namespace {
+
+constexpr int kNoAllocMaxDevices = 64;
+// Device addresses of iv_noalloc_scratch, one per device, filled on first use.  The array's
+// name is only a host-side handle: the address a kernel can use comes from cudaGetSymbolAddress.
+unsigned char *g_noalloc_ptr[kNoAllocMaxDevices] = {};
+
+}  // namespace
+
+extern "C" int iv_merkle_root_noalloc(const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
+                                      void *cuda_stream) {
+    if (!d_root || (n_leaves && !d_leaves)) return IV_ERR_INVALID_ARG;
+    if (n_leaves > IV_NOALLOC_MAX_LEAVES) return IV_ERR_TOO_LARGE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNoAllocMaxDevices) {
+        (void)cudaGetLastError();
+        return IV_ERR_NO_DEVICE;
+    }
+    unsigned char *scratch = __atomic_load_n(&g_noalloc_ptr[dev], __ATOMIC_ACQUIRE);
+    if (!scratch) {
+        // set-up, once per device, with that device current
+        if (cudaGetSymbolAddress(reinterpret_cast<void **>(&scratch), iv_noalloc_scratch) != cudaSuccess || !scratch) {
+            (void)cudaGetLastError();
+            return IV_ERR_CUDA;
+        }
+        __atomic_store_n(&g_noalloc_ptr[dev], scratch, __ATOMIC_RELEASE);
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (n_leaves == 0) {
+        ivk::empty_root_kernel<<<1, 1, 0, stream>>>(d_root);
+        return cudaGetLastError() == cudaSuccess ? IV_OK : IV_ERR_CUDA;
+    }
+    uint32_t *ticket = reinterpret_cast<uint32_t *>(scratch + ivk::kMerkleRun * 32);
+    // The array keeps whatever the previous call left; only the ticket has to start at zero.
+    if (cudaMemsetAsync(ticket, 0, sizeof(uint32_t), stream) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return IV_ERR_CUDA;
+    }
+    const uint64_t runs = (n_leaves + ivk::kMerkleRun - 1) / ivk::kMerkleRun;   // <= 512: one fused pass
+    ivk::merkle_pass_kernel<<<(unsigned)runs, ivk::kThreads, 0, stream>>>(d_leaves, n_leaves, scratch, d_root,
+                                                                           ticket, 1);
+    return cudaGetLastError() == cudaSuccess ? IV_OK : IV_ERR_CUDA;
+}
