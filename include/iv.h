@@ -247,7 +247,19 @@ typedef enum iv_probe_kind {
     IV_PROBE_IMAD = 4,   /* integer multiply-add */
     IV_PROBE_MIXED = 5,  /* LOP3 and IMAD interleaved 1:1 */
     IV_PROBE_SHA256 = 6,     /* full SHA-256 compressions, registers only */
-    IV_PROBE_SHA256_FMA = 7  /* the same with every addition issued as a multiply-add (FMA pipe) */
+    IV_PROBE_SHA256_FMA = 7, /* the same with every addition issued as a multiply-add (FMA pipe) */
+    IV_PROBE_LAT_IADD3 = 8,  /* kinds 8..11: ONE dependent chain per thread; with one warp per SM,   */
+    IV_PROBE_LAT_LOP3 = 9,   /* 32 / h_out[0] is the dependent-issue latency of the instruction in   */
+    IV_PROBE_LAT_SHF = 10,   /* clocks                                                               */
+    IV_PROBE_LAT_IMAD = 11,
+    IV_PROBE_LAT_CROSS = 12, /* one chain alternating LOP3 (ALU pipe) and IMAD (FMA pipe) */
+    IV_PROBE_ROUNDS_M0 = 13, /* kinds 13..16: the 64 rounds alone (W + K from shared memory), one   */
+    IV_PROBE_ROUNDS_M1 = 14, /* block per trip, for the four placements of the additions; reported  */
+    IV_PROBE_ROUNDS_M2 = 15, /* as message bytes per clock per SM                                    */
+    IV_PROBE_ROUNDS_M3 = 16,
+    IV_PROBE_SCHEDULE = 17,  /* the message schedule + round constants alone, one block per trip */
+    IV_PROBE_ROUNDS_M4 = 18,
+    IV_PROBE_ROUNDS_M5 = 19
 } iv_probe_kind;
 int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t blocks_per_sm,
                  uint32_t active_lanes, uint32_t iters, double *h_out);

@@ -2,6 +2,7 @@
 // (Algorithm 1: H_i = GPU_HASH(M_i), FIPS 180-4 section 6.2).
 #include "iv_internal.h"
 #include "sha256_dev.cuh"
+#include "tma_dev.cuh"
 
 namespace ivk {
 
@@ -107,48 +108,6 @@ hash_chunks_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t c
 // 64-byte block are bank-conflict free.  A request of SEG bytes amortises the
 // DRAM/TLB latency of a stream over SEG/64 compressions.
 // ---------------------------------------------------------------------------
-namespace tma {
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void fence_barrier_init() {
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Waits for a phase of the barrier, giving up after about two seconds of SM clocks.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > 4000000000ll) return false;
-    }
-    return true;
-}
-// Bulk copy global -> this CTA's shared memory; src, dst and bytes are multiples of 16.
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-}  // namespace tma
 
 template <int SEG, int STAGES, int WARPS, bool FMA>
 __global__ void __launch_bounds__(32 * WARPS)
@@ -280,13 +239,16 @@ cudaError_t launch_staged(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk
 
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
-                               cudaStream_t stream, uint64_t *launches) {
+                               const uint32_t *d_one, cudaStream_t stream, uint64_t *launches) {
     if (n_chunks == 0) return cudaSuccess;
     if (launches) ++*launches;
     const uint64_t warps = (n_chunks + 31) / 32;
     const bool aligned = ((reinterpret_cast<uintptr_t>(d_data) & 15u) == 0) && (chunk_bytes % 16u == 0);
     if (aligned && chunk_bytes >= 4096) {
         // Few chains: one warp per CTA, so every chain warp gets an SM scheduler of its own and a deep ring.
+        // Two warps per 32 chains while every warp can still have an SM scheduler of its own.
+        if (warps <= 2ull * sm_count)
+            return launch_hash_chunks_split(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one, stream);
         if (warps <= 4ull * sm_count)
             return launch_staged<512, 3, 1, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);
         // Many chains: two CTAs of four warps per SM keep two warps on every scheduler.

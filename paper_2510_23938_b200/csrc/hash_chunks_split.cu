@@ -1,0 +1,185 @@
+// Leaf hashing when chains are scarce (fewer chunks than the GPU has lanes to spare).
+//
+// A chunk is one serial compression chain, so with few chunks the time per 64-byte block of
+// ONE chain bounds the whole job.  About 40 % of SHA-256's work -- the endian swap, the
+// 48-step message schedule and the addition of the round constants -- does not depend on the
+// chaining state.  Each CTA therefore runs two warps on two SM schedulers for its 32 chains:
+//
+//   producer warp: pulls the lanes' streams through a shared-memory ring with bulk copies
+//                  (as the staged kernel does), forms W[t] + K[t] for t = 0..63 of every block
+//                  and writes them to a second ring, lane-interleaved;
+//   consumer warp: runs only the 64 rounds, reading W[t] + K[t] with 128-bit shared loads.
+//
+// The two rings are handed over through mbarriers (full / empty per slot); all waits are bounded.
+// The chain's critical path per block drops from the whole compression to the rounds alone.
+#include "iv_internal.h"
+#include "sha256_dev.cuh"
+#include "tma_dev.cuh"
+#include "sha256_split_dev.cuh"
+
+namespace ivk {
+namespace {
+
+template <int SEG, int STAGES, int NSLOT, int MODE>
+__global__ void __launch_bounds__(64)
+hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
+                         uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
+                         const uint32_t *__restrict__ one_ptr) {
+    constexpr uint32_t kLaneStride = SEG + 16;            // data ring: bytes per lane per stage
+    constexpr uint32_t kStageBytes = 32 * kLaneStride;
+    constexpr int kBlocksPerSeg = SEG / 64;
+    constexpr uint32_t kWkLane = 64 * 4 + 16;             // W+K ring: bytes per lane per slot
+    constexpr uint32_t kWkSlot = 32 * kWkLane;
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ __align__(8) uint64_t bars[STAGES + 2 * NSLOT];
+
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    const uint32_t data_base = tma::smem_u32(smem) + lane * kLaneStride;
+    const uint32_t wk_base = tma::smem_u32(smem) + STAGES * kStageBytes + lane * kWkLane;
+    const uint32_t bar_data = tma::smem_u32(&bars[0]);
+    const uint32_t bar_full = bar_data + 8 * STAGES;
+    const uint32_t bar_empty = bar_full + 8 * NSLOT;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES + 2 * NSLOT; ++s) tma::mbar_init(bar_data + 8 * s, 1);
+        tma::fence_barrier_init();
+    }
+    __syncthreads();
+    // The multiplier 1 for additions issued as multiply-adds: read from memory, so that neither
+    // compiler stage can fold the multiplication away.
+    const uint32_t one = __ldg(one_ptr);
+
+    const uint64_t i = (uint64_t)blockIdx.x * 32 + lane;
+    const bool valid = i < n_chunks;
+    const uint64_t begin = valid ? i * chunk_bytes : 0;
+    const uint64_t len = valid ? ((nbytes - begin < chunk_bytes) ? (nbytes - begin) : chunk_bytes) : 0;
+    // SHA-256 blocks of this lane's message, padding included; lane 0 holds the longest chunk of the warp.
+    const uint64_t my_total = valid ? ((len + 8) >> 6) + 1 : 0;
+    const uint64_t warp_total = __shfl_sync(0xffffffffu, my_total, 0);
+
+    if (warp == 1) {
+        // ------------------------------------------------------------------ producer
+        const uint8_t *p = data + begin;
+        const uint64_t full_bytes = len & ~63ull;
+        const uint64_t my_full = full_bytes >> 6;
+        const uint64_t warp_full = __shfl_sync(0xffffffffu, my_full, 0);
+        const uint64_t nseg = (warp_full * 64 + SEG - 1) / SEG;
+        // One arrival per stage: lane 0 announces the bytes of all 32 copies, every lane issues its own.
+        auto issue = [&](uint64_t seg, int stage) {
+            const uint64_t off = seg * SEG;
+            const uint32_t bar = bar_data + 8 * stage;
+            const uint32_t bytes = off < full_bytes ? (uint32_t)((full_bytes - off < SEG) ? (full_bytes - off) : SEG) : 0u;
+            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+            if (lane == 0) tma::mbar_arrive_expect_tx(bar, total);
+            if (bytes) tma::bulk_g2s(data_base + stage * kStageBytes, p + off, bytes, bar);
+        };
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s)
+            if ((uint64_t)s < nseg) issue(s, s);
+
+        uint32_t w[16], raw[16], tw[32];
+        int stage = 0, in_stage = 0;
+        uint32_t dparity = 0;
+        bool failed = false, tail_built = false;
+        auto fetch = [&](int blk_in_stage) {
+            const uint32_t src = data_base + stage * kStageBytes + 64 * blk_in_stage;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                tma::ld_shared_v4(src + 16 * q, raw[4 * q], raw[4 * q + 1], raw[4 * q + 2], raw[4 * q + 3]);
+        };
+        if (warp_full) {
+            failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_data, 0));
+            if (!failed) fetch(0);
+        }
+        uint64_t next_seg = STAGES;
+        int slot = 0;
+        uint32_t eparity = 1;                         // first pass over the slots finds them empty
+        for (uint64_t blk = 0; blk < warp_total && !failed; ++blk) {
+            if (blk < my_full) {
+#pragma unroll
+                for (int k = 0; k < 16; ++k) w[k] = bswap32(raw[k]);
+            } else if (blk < my_total) {
+                if (!tail_built) {
+                    (void)sha256_build_tail(p + full_bytes, (uint32_t)(len & 63u), len, tw);
+                    tail_built = true;
+                }
+                const int t = (int)(blk - my_full);
+#pragma unroll
+                for (int k = 0; k < 16; ++k) w[k] = tw[16 * t + k];
+            }
+            if (blk + 1 < warp_full) {
+                if (++in_stage == kBlocksPerSeg) {
+                    in_stage = 0;
+                    __syncwarp();
+                    if (next_seg < nseg) issue(next_seg, stage);
+                    ++next_seg;
+                    if (++stage == STAGES) { stage = 0; dparity ^= 1u; }
+                    failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_data + 8 * stage, dparity));
+                    if (failed) break;
+                }
+                fetch(in_stage);
+            }
+            failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_empty + 8 * slot, eparity));
+            if (failed) break;
+            produce_wk(w, wk_base + slot * kWkSlot, one);
+            __syncwarp();                              // all 32 lanes' stores are ordered before lane 0's arrival
+            if (lane == 0) tma::mbar_arrive(bar_full + 8 * slot);
+            if (++slot == NSLOT) { slot = 0; eparity ^= 1u; }
+        }
+        if (failed && lane == 0) atomicExch(status, (uint32_t)IVK_DEV_TIMEOUT);
+        return;
+    }
+
+    // ---------------------------------------------------------------------- consumer
+    uint32_t st[8], v[8];
+    sha256_init(st);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) v[k] = st[k];
+    int slot = 0;
+    uint32_t fparity = 0;
+    bool failed = false;
+    for (uint64_t blk = 0; blk < warp_total; ++blk) {
+        failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_full + 8 * slot, fparity));
+        if (failed) break;
+        const uint32_t src = wk_base + slot * kWkSlot;
+        rounds64<MODE>(v, src, one);
+        __syncwarp();                                  // all 32 lanes have their values in registers
+        if (lane == 0) tma::mbar_arrive(bar_empty + 8 * slot);
+        // feed-forward; a lane whose message has ended keeps its state (multiplier 0 instead of 1)
+        const uint32_t keep = (blk < my_total) ? one : 0u;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            st[k] = padd<true>(v[k], st[k], keep);     // v * keep + st
+            v[k] = st[k];
+        }
+        if (++slot == NSLOT) { slot = 0; fparity ^= 1u; }
+    }
+    if (failed) {
+        if (lane == 0) atomicExch(status, (uint32_t)IVK_DEV_TIMEOUT);
+        return;
+    }
+    if (valid) store_digest(digests + 32 * i, st);
+}
+
+}  // namespace
+
+cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                                     uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status,
+                                     const uint32_t *d_one, cudaStream_t stream) {
+    // 512-byte segments, three data stages, four W+K slots; the additions that close the two state
+    // recurrences stay three-input ALU adds, the others go to the FMA pipe (placement 3, the fastest measured).
+    constexpr int SEG = 512, STAGES = 3, NSLOT = 4, MODE = 3;
+    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * 32 * (64 * 4 + 16);
+    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const uint64_t blocks = (n_chunks + 31) / 32;
+    if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
+    kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one);
+    return cudaGetLastError();
+}
+
+}  // namespace ivk

@@ -17,6 +17,7 @@ struct iv_ctx {
     unsigned long long *d_queue = nullptr;
     uint8_t *d_root = nullptr;                // 32 bytes
     uint32_t *d_status = nullptr;             // device-side status word (0 = ok), sticky until read
+    uint32_t *d_one = nullptr;                // a device word holding 1 (multiplier for adds on the FMA pipe)
     void *d_small = nullptr;
 
     // lazily sized scratch
@@ -196,6 +197,16 @@ int iv_create(iv_ctx **out, int cuda_device) {
     ctx->d_queue = reinterpret_cast<unsigned long long *>(base + 64);     // 8 bytes
     ctx->d_tickets = reinterpret_cast<uint32_t *>(base + 128);            // kMerkleMaxPasses + 1 words
     ctx->d_status = reinterpret_cast<uint32_t *>(base + 192);
+    ctx->d_one = reinterpret_cast<uint32_t *>(base + 224);
+    {
+        const uint32_t one = 1u;
+        e = cudaMemcpy(ctx->d_one, &one, sizeof one, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            int rc = fail_cuda(nullptr, e);
+            iv_destroy(ctx);
+            return rc;
+        }
+    }
     *out = ctx;
     return IV_OK;
 }
@@ -252,7 +263,7 @@ int iv_hash_chunks(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t ch
     if (n == 0) return IV_OK;
     DeviceGuard guard(ctx->device);
     IV_TRY(ctx, ivk::launch_hash_chunks(static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
-                                        ctx->sm_count, ctx->d_status, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+                                        ctx->sm_count, ctx->d_status, ctx->d_one, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
     return IV_OK;
 }
 
@@ -280,7 +291,7 @@ int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const i
     if (rc != IV_OK) return rc;
     if ((rc = mark_phase(ctx, 0, stream)) != IV_OK) return rc;
     IV_TRY(ctx, ivk::launch_hash_chunks(static_cast<const uint8_t *>(d_data), nbytes, h_manifest->chunk_bytes, n,
-                                        ctx->d_digests, ctx->sm_count, ctx->d_status, stream, &ctx->launches));
+                                        ctx->d_digests, ctx->sm_count, ctx->d_status, ctx->d_one, stream, &ctx->launches));
     return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream);
 }
 
@@ -333,7 +344,7 @@ int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_win
         IV_TRY(ctx, cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
         IV_TRY(ctx, cudaStreamWaitEvent(stream, ctx->ev_copied[b], 0));
         IV_TRY(ctx, ivk::launch_hash_chunks(ctx->d_window[b], bytes, chunk, chunk_count(bytes, chunk),
-                                            ctx->d_digests + 32 * w * chunks_per_window, ctx->sm_count, ctx->d_status, stream,
+                                            ctx->d_digests + 32 * w * chunks_per_window, ctx->sm_count, ctx->d_status, ctx->d_one, stream,
                                             &ctx->launches));
         IV_TRY(ctx, cudaEventRecord(ctx->ev_hashed[b], stream));
     }
@@ -374,15 +385,17 @@ int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t block
     if (!ctx || !h_out || warps_per_block == 0 || warps_per_block > 32 || blocks_per_sm == 0 ||
         blocks_per_sm > 32 || active_lanes == 0 || active_lanes > 32 || iters == 0)
         return IV_ERR_INVALID_ARG;
-    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_SHA256_FMA) return IV_ERR_INVALID_ARG;
+    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_ROUNDS_M5) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     const unsigned blocks = blocks_per_sm * (unsigned)ctx->sm_count;
     unsigned long long *d_cycles = nullptr;
     IV_TRY(ctx, cudaMalloc(&d_cycles, sizeof(unsigned long long) * blocks + 64));
     uint32_t *d_sink = reinterpret_cast<uint32_t *>(d_cycles + blocks);
+    const uint32_t sink_init[2] = {0u, 1u};     // word 1 is the multiplier "1" some probe kernels read
     unsigned long long *h_cycles = static_cast<unsigned long long *>(std::malloc(sizeof(unsigned long long) * blocks));
     int rc = IV_OK;
     cudaError_t e = h_cycles ? cudaSuccess : cudaErrorMemoryAllocation;
+    if (e == cudaSuccess) e = cudaMemcpy(d_sink, sink_init, sizeof sink_init, cudaMemcpyHostToDevice);
     for (int rep = 0; rep < 2 && e == cudaSuccess; ++rep) {   // first launch warms the instruction cache
         e = ivk::launch_probe(kind, blocks, 32u * warps_per_block, iters, active_lanes, d_cycles, d_sink, nullptr);
         ++ctx->launches;
@@ -395,7 +408,7 @@ int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t block
         for (unsigned b = 0; b < blocks; ++b) sum += (double)h_cycles[b];
         const double mean = sum / blocks;
         double per_thread = (double)ivk::probe_ops_per_thread(kind, iters);
-        if (kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_FMA) per_thread *= 64.0;       // bytes per compression
+        if (kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_FMA || kind >= IV_PROBE_ROUNDS_M0) per_thread *= 64.0;       // bytes per compression
         h_out[0] = (double)blocks_per_sm * warps_per_block * active_lanes * per_thread / mean;
         h_out[1] = mean;
     } else {

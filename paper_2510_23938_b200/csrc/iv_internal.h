@@ -17,7 +17,14 @@ constexpr uint32_t kMerkleRun = 512;
 // One SHA-256 per chunk: digest i <- SHA-256(data[i*C .. min((i+1)*C, nbytes))).
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
-                               cudaStream_t stream, uint64_t *launches);
+                               const uint32_t *d_one, cudaStream_t stream, uint64_t *launches);
+
+// hash_chunks_split.cu ------------------------------------------------------
+// Same result for base and chunk size multiples of 16 bytes; two warps per 32 chains
+// (schedule producer + round consumer), for launches with few chains.
+cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                                     uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status,
+                                     const uint32_t *d_one, cudaStream_t stream);
 
 // hash_ragged.cu -----------------------------------------------------------
 // One SHA-256 per (offset, length); d_queue is one zeroed uint64 work counter.
