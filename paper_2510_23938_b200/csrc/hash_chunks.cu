@@ -1,5 +1,7 @@
 // Leaf hashing: one SHA-256 compression chain per thread, one chunk per chain
 // (Algorithm 1: H_i = GPU_HASH(M_i), FIPS 180-4 section 6.2).
+#include <cstdlib>
+
 #include "iv_internal.h"
 #include "sha256_dev.cuh"
 #include "tma_dev.cuh"
@@ -237,9 +239,17 @@ cudaError_t launch_staged(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk
     return cudaGetLastError();
 }
 
+bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count) {
+    const uint64_t warps = (n_chunks + 31) / 32;
+    const bool aligned = ((reinterpret_cast<uintptr_t>(d_data) & 15u) == 0) && (chunk_bytes % 16u == 0);
+    static const bool off = getenv("IV_NO_SLICE") != nullptr;
+    return !off && aligned && chunk_bytes >= 32768 && warps > 4ull * (uint64_t)sm_count;
+}
+
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
-                               const uint32_t *d_one, cudaStream_t stream, uint64_t *launches) {
+                               const uint32_t *d_one, void *d_slice_scratch, cudaStream_t stream,
+                               uint64_t *launches) {
     if (n_chunks == 0) return cudaSuccess;
     if (launches) ++*launches;
     const uint64_t warps = (n_chunks + 31) / 32;
@@ -251,7 +261,13 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
             return launch_hash_chunks_split(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one, stream);
         if (warps <= 4ull * sm_count)
             return launch_staged<512, 3, 1, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);
-        // Many chains: two CTAs of four warps per SM keep two warps on every scheduler.
+        // Many chains of sliceable size: chains migrate between schedulers (two launches: queue set-up + workers).
+        if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
+            if (launches) ++*launches;
+            return launch_hash_chunks_sliced(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
+                                             d_slice_scratch, sm_count, stream);
+        }
+        // Many small chunks: two CTAs of four warps per SM keep two warps on every scheduler.
         return launch_staged<256, 3, 4, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);
     }
     const unsigned warps_per_cta = warps <= (uint64_t)sm_count ? 1u : (warps <= 2ull * sm_count ? 2u : 4u);

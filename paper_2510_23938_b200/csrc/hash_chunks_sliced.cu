@@ -1,0 +1,285 @@
+// Leaf hashing when chains are plentiful but do not divide evenly over the GPU.
+//
+// One warp carries 32 chains (a "group").  With G groups on 592 SM schedulers a static
+// assignment leaves some schedulers with two warps and others with one for the whole launch
+// (28,672 chunks = 896 groups: 304 schedulers get two groups, 288 get one, and the launch lasts as
+// long as the doubly loaded ones).  Here the chains migrate instead: every chunk is cut into
+// slices, a task is (group, slice), and persistent warps take tasks from a FIFO in global
+// memory.  A group re-enters the FIFO when its slice is done, its eight-word chaining values
+// parked in global memory, so its next slice can run on any scheduler.  Because a group is in
+// the FIFO at most once, its slices run in order; a warp never waits while it holds a task, so
+// the scheme needs no co-residency and cannot deadlock.  All waits are bounded.
+//
+// Data movement is the staged kernel's: per-lane bulk copies (TMA) into a lane-interleaved
+// shared-memory ring, mbarrier completion, the next block fetched into registers before the
+// current block's rounds.
+#include <cstdlib>
+
+#include "iv_internal.h"
+#include "sha256_dev.cuh"
+#include "tma_dev.cuh"
+
+namespace ivk {
+namespace {
+
+struct SliceQueue {
+    unsigned long long head;   // next ticket to hand to a worker
+    unsigned long long tail;   // next ticket a finished slice pushes its group under
+};
+
+// slot[t] = group + 1 once ticket t has been pushed, 0 before.  The first `groups` tickets are
+// pre-filled with the groups in order; every group starts at slice 0.
+__global__ void slice_queue_init(uint32_t *__restrict__ slot, uint64_t total_tasks, uint64_t groups,
+                                 SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice) {
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total_tasks; i += stride)
+        slot[i] = i < groups ? (uint32_t)i + 1u : 0u;
+    for (uint64_t g = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += stride) next_slice[g] = 0u;
+    if (blockIdx.x == 0 && threadIdx.x == 0) { q->head = 0ull; q->tail = groups; }
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+template <int SEG, int STAGES, int MAX_WARPS>
+__global__ void __launch_bounds__(32 * MAX_WARPS)
+hash_chunks_sliced_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
+                          uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
+                          uint64_t slice_bytes, uint64_t total_tasks, uint32_t *__restrict__ slot,
+                          SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice,
+                          uint32_t *__restrict__ mid /* [groups][8][32] */) {
+    constexpr uint32_t kLaneStride = SEG + 16;
+    constexpr uint32_t kStageBytes = 32 * kLaneStride;
+    constexpr int kBlocksPerSeg = SEG / 64;
+    extern __shared__ __align__(128) uint8_t ring[];
+    __shared__ __align__(8) uint64_t bars[MAX_WARPS][STAGES];
+
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
+    const uint32_t ring_base = tma::smem_u32(ring) + warp * (STAGES * kStageBytes) + lane * kLaneStride;
+    const uint32_t bar_base = tma::smem_u32(&bars[warp][0]);
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) tma::mbar_init(bar_base + 8 * s, 1);
+        tma::fence_barrier_init();
+    }
+    __syncwarp();
+
+    // ring position, carried from task to task (every task drains what it requested)
+    int stage = 0;
+    uint32_t parity = 0;
+    bool failed = false;
+
+    for (;;) {
+        // ---- take a ticket, wait for the group that is pushed under it
+        unsigned long long t = 0;
+        if (lane == 0) t = atomicAdd(&q->head, 1ull);
+        t = __shfl_sync(0xffffffffu, t, 0);
+        if (t >= total_tasks) break;
+        uint32_t entry = 0;
+        if (lane == 0) {
+            entry = ld_acquire_u32(slot + t);
+            if (entry == 0) {
+                const long long t0 = clock64();
+                unsigned ns = 64;
+                while ((entry = ld_acquire_u32(slot + t)) == 0) {
+                    if (clock64() - t0 > 8000000000ll) break;       // about four seconds: give up
+                    __nanosleep(ns);
+                    if (ns < 2048) ns *= 2;
+                }
+            }
+        }
+        entry = __shfl_sync(0xffffffffu, entry, 0);
+        if (entry == 0) { failed = true; break; }
+        const uint64_t g = entry - 1u;
+        // lane 0 made the acquire; it reads the slice number and the warp barrier orders the other
+        // lanes' reads of the parked chaining values after it
+        uint32_t s = 0;
+        if (lane == 0) s = __ldcg(next_slice + g);
+        s = __shfl_sync(0xffffffffu, s, 0);
+        __syncwarp();
+
+        // ---- this lane's share of the slice
+        const uint64_t i = g * 32 + lane;
+        const bool valid = i < n_chunks;
+        const uint64_t begin = valid ? i * chunk_bytes : 0;
+        const uint64_t len = valid ? ((nbytes - begin < chunk_bytes) ? (nbytes - begin) : chunk_bytes) : 0;
+        const uint64_t full_bytes = len & ~63ull;
+        const uint64_t lo = (uint64_t)s * slice_bytes;
+        const uint64_t hi_full = lo + slice_bytes;
+        const uint64_t my_lo = lo < full_bytes ? lo : full_bytes;
+        const uint64_t my_hi = hi_full < full_bytes ? hi_full : full_bytes;
+        const uint64_t my_bytes = my_hi - my_lo;                       // multiple of 64
+        const uint8_t *p = data + begin + my_lo;
+        // lane 0 holds the longest chunk of its group (only the blob's last chunk can be shorter)
+        const uint64_t warp_bytes = __shfl_sync(0xffffffffu, my_bytes, 0);
+        const uint64_t warp_full = __shfl_sync(0xffffffffu, full_bytes, 0);
+        const bool last_slice = hi_full >= warp_full;
+        const uint64_t nseg = (warp_bytes + SEG - 1) / SEG;
+
+        uint32_t st[8], w[16], raw[16];
+        if (s == 0) {
+            sha256_init(st);
+        } else {
+            const uint32_t *m = mid + g * 256 + lane;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) st[k] = __ldcg(m + 32 * k);
+        }
+
+        auto issue = [&](uint64_t seg, int stg) {
+            const uint64_t off = seg * SEG;
+            const uint32_t bar = bar_base + 8 * stg;
+            const uint32_t bytes = off < my_bytes ? (uint32_t)((my_bytes - off < SEG) ? (my_bytes - off) : SEG) : 0u;
+            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+            if (lane == 0) tma::mbar_arrive_expect_tx(bar, total);
+            if (bytes) tma::bulk_g2s(ring_base + stg * kStageBytes, p + off, bytes, bar);
+        };
+        auto fetch = [&](int stg, int blk_in_stage) {
+            const uint32_t src = ring_base + stg * kStageBytes + 64 * blk_in_stage;
+#pragma unroll
+            for (int qd = 0; qd < 4; ++qd)
+                tma::ld_shared_v4(src + 16 * qd, raw[4 * qd], raw[4 * qd + 1], raw[4 * qd + 2], raw[4 * qd + 3]);
+        };
+
+        // prologue: request the first STAGES segments into the stages that follow the ring position
+        {
+            int stg = stage;
+#pragma unroll
+            for (int k = 0; k < STAGES; ++k) {
+                if ((uint64_t)k < nseg) issue(k, stg);
+                if (++stg == STAGES) stg = 0;
+            }
+        }
+        const uint64_t my_blocks = my_bytes >> 6;
+        const uint64_t warp_blocks = warp_bytes >> 6;
+        int in_stage = 0;
+        if (warp_blocks) {
+            failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_base + 8 * stage, parity));
+            if (failed) break;
+            fetch(stage, 0);
+        }
+        uint64_t next_seg = STAGES;
+        for (uint64_t blk = 0; blk < warp_blocks; ++blk) {
+#pragma unroll
+            for (int k = 0; k < 16; ++k) w[k] = bswap32(raw[k]);
+            const bool stage_done = (++in_stage == kBlocksPerSeg) || (blk + 1 == warp_blocks);
+            if (stage_done) {
+                in_stage = 0;
+                __syncwarp();                            // every lane has taken its data out of the stage
+                if (next_seg < nseg) issue(next_seg, stage);
+                ++next_seg;
+                if (++stage == STAGES) { stage = 0; parity ^= 1u; }
+                if (blk + 1 < warp_blocks) {
+                    failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_base + 8 * stage, parity));
+                    if (failed) break;
+                }
+            }
+            if (blk + 1 < warp_blocks) fetch(stage, in_stage);
+            if (blk < my_blocks) sha256_compress(st, w);
+        }
+        if (failed) break;
+
+        if (!last_slice) {
+            uint32_t *m = mid + g * 256 + lane;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) __stcg(m + 32 * k, st[k]);
+            __syncwarp();
+            if (lane == 0) {
+                __stcg(next_slice + g, s + 1u);
+                __threadfence();
+                const unsigned long long pt = atomicAdd(&q->tail, 1ull);
+                st_release_u32(slot + pt, (uint32_t)g + 1u);
+            }
+            continue;
+        }
+        if (!valid) continue;
+        const uint32_t rem = (uint32_t)(len & 63u);
+        if (rem == 0) {
+            sha256_pad_only_block(w, len);
+            sha256_compress(st, w);
+        } else {
+            uint32_t tw[32];
+            const int nblk = sha256_build_tail(data + begin + full_bytes, rem, len, tw);
+#pragma unroll 1
+            for (int tb = 0; tb < nblk; ++tb) {
+#pragma unroll
+                for (int k = 0; k < 16; ++k) w[k] = tw[16 * tb + k];
+                sha256_compress(st, w);
+            }
+        }
+        store_digest(digests + 32 * i, st);
+    }
+    if (failed && lane == 0) atomicExch(status, (uint32_t)IVK_DEV_TIMEOUT);
+}
+
+}  // namespace
+
+uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t *slice_bytes_out, uint64_t *total_tasks_out,
+                              uint64_t nbytes) {
+    const uint64_t groups = (n_chunks + 31) / 32;
+    // slices of at least 16 KiB, at most 64 per chunk, a multiple of 4 KiB
+    uint64_t slices = chunk_bytes / 16384;
+    static const uint64_t max_slices = [] { const char *e = getenv("IV_SLICES"); return e ? (uint64_t)atoi(e) : 64ull; }();
+    if (slices > max_slices) slices = max_slices;
+    if (slices < 1) slices = 1;
+    uint64_t slice_bytes = (chunk_bytes + slices - 1) / slices;
+    slice_bytes = (slice_bytes + 4095) & ~4095ull;
+    // slices are counted over the whole 64-byte blocks of a chunk, as the kernel does
+    uint64_t per_group = ((chunk_bytes & ~63ull) + slice_bytes - 1) / slice_bytes;
+    if (per_group < 1) per_group = 1;
+    // the last group's first chunk may be the blob's short last chunk
+    const uint64_t first_of_last = (groups - 1) * 32;
+    const uint64_t begin = first_of_last * chunk_bytes;
+    const uint64_t len = nbytes - begin < chunk_bytes ? nbytes - begin : chunk_bytes;
+    const uint64_t full = len & ~63ull;
+    uint64_t last_group = (full + slice_bytes - 1) / slice_bytes;
+    if (last_group < 1) last_group = 1;
+    const uint64_t total = (groups - 1) * per_group + last_group;
+    if (slice_bytes_out) *slice_bytes_out = slice_bytes;
+    if (total_tasks_out) *total_tasks_out = total;
+    // queue header (64) + slots + next_slice + chaining values
+    return 64 + 4 * total + 4 * groups + 1024 * groups + 256;
+}
+
+cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
+                                      int sm_count, cudaStream_t stream) {
+    constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8;
+    constexpr size_t smem_per_warp = (size_t)STAGES * 32 * (SEG + 16);
+    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(MAX_WARPS * smem_per_warp));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    uint64_t slice_bytes = 0, total_tasks = 0;
+    (void)sliced_scratch_bytes(n_chunks, chunk_bytes, &slice_bytes, &total_tasks, nbytes);
+    const uint64_t groups = (n_chunks + 31) / 32;
+    uint8_t *base = static_cast<uint8_t *>(d_scratch);
+    SliceQueue *q = reinterpret_cast<SliceQueue *>(base);
+    uint32_t *mid = reinterpret_cast<uint32_t *>(base + 64);                       // 1 KiB per group, 16-byte aligned
+    uint32_t *slot = reinterpret_cast<uint32_t *>(base + 64 + 1024 * groups);
+    uint32_t *next_slice = slot + total_tasks;
+    slice_queue_init<<<64, 256, 0, stream>>>(slot, total_tasks, groups, q, next_slice);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    // One persistent CTA per SM.  A worker that finds the FIFO empty only waits, and waiting warps
+    // were measured to slow their SM down, so there are never more workers than groups: as many
+    // warps per SM as the groups fill evenly, at most two per scheduler.
+    static const uint64_t forced = [] { const char *e = getenv("IV_SLICE_WARPS"); return e ? (uint64_t)atoi(e) : 0ull; }();
+    uint64_t warps = forced ? forced : groups / (uint64_t)sm_count;
+    if (warps > MAX_WARPS) warps = MAX_WARPS;
+    if (warps < 1) warps = 1;
+    kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp, stream>>>(
+        d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice, mid);
+    return cudaGetLastError();
+}
+
+}  // namespace ivk

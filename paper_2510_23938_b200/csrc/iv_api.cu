@@ -28,6 +28,8 @@ struct iv_ctx {
     uint64_t digests_valid = 0;
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
+    uint8_t *d_slices = nullptr;              // FIFO, slice counters and parked chaining values of the sliced leaf kernel
+    uint64_t slices_cap = 0;                  // bytes
 
     // streaming windows
     uint8_t *d_window[2] = {nullptr, nullptr};
@@ -97,6 +99,21 @@ int ensure_merkle_scratch(iv_ctx *ctx, uint64_t n_leaves) {
     rc = grow(ctx, &ctx->d_merkle_b, &cap_b, need, 32);
     if (rc != IV_OK) return rc;
     ctx->merkle_cap = cap_a < cap_b ? cap_a : cap_b;
+    return IV_OK;
+}
+
+// Leaf hashing with the scratch the launch shape needs.
+int hash_leaves(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n,
+                uint8_t *d_digests, cudaStream_t stream) {
+    void *scratch = nullptr;
+    if (ivk::hash_chunks_wants_slices(d_data, chunk_bytes, n, ctx->sm_count)) {
+        const uint64_t need = ivk::sliced_scratch_bytes(n, chunk_bytes, nullptr, nullptr, nbytes);
+        int rc = grow(ctx, &ctx->d_slices, &ctx->slices_cap, need, 1);
+        if (rc != IV_OK) return rc;
+        scratch = ctx->d_slices;
+    }
+    IV_TRY(ctx, ivk::launch_hash_chunks(d_data, nbytes, chunk_bytes, n, d_digests, ctx->sm_count, ctx->d_status,
+                                        ctx->d_one, scratch, stream, &ctx->launches));
     return IV_OK;
 }
 
@@ -220,6 +237,7 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_merkle_b);
     cudaFree(ctx->d_digests);
     cudaFree(ctx->d_words);
+    cudaFree(ctx->d_slices);
     cudaFree(ctx->d_window[0]);
     cudaFree(ctx->d_window[1]);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -262,9 +280,8 @@ int iv_hash_chunks(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t ch
     if (h_n_chunks) *h_n_chunks = n;
     if (n == 0) return IV_OK;
     DeviceGuard guard(ctx->device);
-    IV_TRY(ctx, ivk::launch_hash_chunks(static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
-                                        ctx->sm_count, ctx->d_status, ctx->d_one, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
-    return IV_OK;
+    return hash_leaves(ctx, static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
+                       static_cast<cudaStream_t>(cuda_stream));
 }
 
 int iv_merkle_root(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
@@ -290,8 +307,9 @@ int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const i
     rc = grow(ctx, &ctx->d_digests, &ctx->digests_cap, n + 1, 32);
     if (rc != IV_OK) return rc;
     if ((rc = mark_phase(ctx, 0, stream)) != IV_OK) return rc;
-    IV_TRY(ctx, ivk::launch_hash_chunks(static_cast<const uint8_t *>(d_data), nbytes, h_manifest->chunk_bytes, n,
-                                        ctx->d_digests, ctx->sm_count, ctx->d_status, ctx->d_one, stream, &ctx->launches));
+    rc = hash_leaves(ctx, static_cast<const uint8_t *>(d_data), nbytes, h_manifest->chunk_bytes, n, ctx->d_digests,
+                     stream);
+    if (rc != IV_OK) return rc;
     return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream);
 }
 
@@ -343,9 +361,9 @@ int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_win
         IV_TRY(ctx, cudaMemcpyAsync(ctx->d_window[b], h_windows[w], bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
         IV_TRY(ctx, cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
         IV_TRY(ctx, cudaStreamWaitEvent(stream, ctx->ev_copied[b], 0));
-        IV_TRY(ctx, ivk::launch_hash_chunks(ctx->d_window[b], bytes, chunk, chunk_count(bytes, chunk),
-                                            ctx->d_digests + 32 * w * chunks_per_window, ctx->sm_count, ctx->d_status, ctx->d_one, stream,
-                                            &ctx->launches));
+        rc = hash_leaves(ctx, ctx->d_window[b], bytes, chunk, chunk_count(bytes, chunk),
+                         ctx->d_digests + 32 * w * chunks_per_window, stream);
+        if (rc != IV_OK) return rc;
         IV_TRY(ctx, cudaEventRecord(ctx->ev_hashed[b], stream));
     }
     return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream);

@@ -17,7 +17,10 @@ constexpr uint32_t kMerkleRun = 512;
 // One SHA-256 per chunk: digest i <- SHA-256(data[i*C .. min((i+1)*C, nbytes))).
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
-                               const uint32_t *d_one, cudaStream_t stream, uint64_t *launches);
+                               const uint32_t *d_one, void *d_slice_scratch, cudaStream_t stream,
+                               uint64_t *launches);
+// True when launch_hash_chunks would use the sliced kernel (and so needs its scratch).
+bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count);
 
 // hash_chunks_split.cu ------------------------------------------------------
 // Same result for base and chunk size multiples of 16 bytes; two warps per 32 chains
@@ -25,6 +28,16 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
 cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status,
                                      const uint32_t *d_one, cudaStream_t stream);
+
+// hash_chunks_sliced.cu -----------------------------------------------------
+// Same result for many chunks of at least 32 KiB (16-byte aligned): chunks are cut into slices
+// that persistent warps take from a FIFO, so chains migrate between SM schedulers and the load
+// stays level.  d_scratch must hold sliced_scratch_bytes(...) bytes.
+uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t *slice_bytes_out,
+                              uint64_t *total_tasks_out, uint64_t nbytes);
+cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
+                                      int sm_count, cudaStream_t stream);
 
 // hash_ragged.cu -----------------------------------------------------------
 // One SHA-256 per (offset, length); d_queue is one zeroed uint64 work counter.

@@ -59,6 +59,24 @@ def test_hash_chunks_any_base_alignment(ctx, shift, chunk):
     assert np.array_equal(_host(got), oracle.hash_chunks(_host(data), chunk))
 
 
+@pytest.mark.parametrize("n_chunks,chunk,last", [
+    (19_000, 32768, 777),            # more than 592 warps of sliceable chunks: chains migrate between schedulers
+    (19_000, 49152 + 16, 49152),     # chunk size a multiple of 16 but not of 64, several slices per chunk
+    (18_945, 65536, 65536),          # exact multiple, last group holds a single chunk
+    (20_001, 32768, 63),             # the last group's only chunk is shorter than one block
+])
+def test_hash_chunks_sliced_launch_shape(ctx, n_chunks, chunk, last):
+    nbytes = (n_chunks - 1) * chunk + last
+    data = inputs.uniform_bytes(nbytes, seed=77, device="cuda")
+    got = ctx.hash_chunks(data, chunk)
+    want = oracle.hash_chunks(_host(data), chunk, nthreads=oracle.host_threads())
+    assert np.array_equal(_host(got), want)
+    assert ctx.device_status() == 0
+    # a second call reuses the FIFO scratch
+    got2 = ctx.hash_chunks(data, chunk)
+    assert torch.equal(got, got2)
+
+
 def test_hash_chunks_empty_and_argument_errors(ctx):
     data = inputs.uniform_bytes(4096, seed=2, device="cuda")
     assert ctx.hash_chunks(data[:0], 64).shape == (0, 32)
