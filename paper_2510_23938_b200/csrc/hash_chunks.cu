@@ -1,7 +1,5 @@
 // Leaf hashing: one SHA-256 compression chain per thread, one chunk per chain
 // (Algorithm 1: H_i = GPU_HASH(M_i), FIPS 180-4 section 6.2).
-#include <cstdlib>
-
 #include "iv_internal.h"
 #include "sha256_dev.cuh"
 #include "tma_dev.cuh"
@@ -242,8 +240,7 @@ cudaError_t launch_staged(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk
 bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count) {
     const uint64_t warps = (n_chunks + 31) / 32;
     const bool aligned = ((reinterpret_cast<uintptr_t>(d_data) & 15u) == 0) && (chunk_bytes % 16u == 0);
-    static const bool off = getenv("IV_NO_SLICE") != nullptr;
-    return !off && aligned && chunk_bytes >= 32768 && warps > 4ull * (uint64_t)sm_count;
+    return aligned && chunk_bytes >= 32768 && warps > 4ull * (uint64_t)sm_count;
 }
 
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
@@ -265,7 +262,7 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
         if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
             if (launches) ++*launches;
             return launch_hash_chunks_sliced(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
-                                             d_slice_scratch, sm_count, stream);
+                                             d_slice_scratch, d_one, sm_count, stream);
         }
         // Many small chunks: two CTAs of four warps per SM keep two warps on every scheduler.
         return launch_staged<256, 3, 4, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);

@@ -13,8 +13,6 @@
 // Data movement is the staged kernel's: per-lane bulk copies (TMA) into a lane-interleaved
 // shared-memory ring, mbarrier completion, the next block fetched into registers before the
 // current block's rounds.
-#include <cstdlib>
-
 #include "iv_internal.h"
 #include "sha256_dev.cuh"
 #include "tma_dev.cuh"
@@ -53,7 +51,11 @@ hash_chunks_sliced_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uin
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
                           uint64_t slice_bytes, uint64_t total_tasks, uint32_t *__restrict__ slot,
                           SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice,
-                          uint32_t *__restrict__ mid /* [groups][8][32] */) {
+                          uint32_t *__restrict__ mid /* [groups][8][32] */, const uint32_t *__restrict__ one_ptr) {
+    // Addition placement 0 (left to the compiler).  Moving the schedule's additions to the FMA
+    // pipe (placement 2) gains 4.5 % in the register-only probe but lost 5 % in this kernel.
+    constexpr int ADD = 0;
+    const uint32_t one = __ldg(one_ptr);
     constexpr uint32_t kLaneStride = SEG + 16;
     constexpr uint32_t kStageBytes = 32 * kLaneStride;
     constexpr int kBlocksPerSeg = SEG / 64;
@@ -180,7 +182,7 @@ hash_chunks_sliced_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uin
                 }
             }
             if (blk + 1 < warp_blocks) fetch(stage, in_stage);
-            if (blk < my_blocks) sha256_compress(st, w);
+            if (blk < my_blocks) sha256_compress<ADD>(st, w, one);
         }
         if (failed) break;
 
@@ -224,8 +226,7 @@ uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t 
     const uint64_t groups = (n_chunks + 31) / 32;
     // slices of at least 16 KiB, at most 64 per chunk, a multiple of 4 KiB
     uint64_t slices = chunk_bytes / 16384;
-    static const uint64_t max_slices = [] { const char *e = getenv("IV_SLICES"); return e ? (uint64_t)atoi(e) : 64ull; }();
-    if (slices > max_slices) slices = max_slices;
+    if (slices > 64) slices = 64;
     if (slices < 1) slices = 1;
     uint64_t slice_bytes = (chunk_bytes + slices - 1) / slices;
     slice_bytes = (slice_bytes + 4095) & ~4095ull;
@@ -248,7 +249,7 @@ uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t 
 
 cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                       uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
-                                      int sm_count, cudaStream_t stream) {
+                                      const uint32_t *d_one, int sm_count, cudaStream_t stream) {
     constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8;
     constexpr size_t smem_per_warp = (size_t)STAGES * 32 * (SEG + 16);
     auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS>;
@@ -270,15 +271,14 @@ cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, ui
     slice_queue_init<<<64, 256, 0, stream>>>(slot, total_tasks, groups, q, next_slice);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    // One persistent CTA per SM.  A worker that finds the FIFO empty only waits, and waiting warps
-    // were measured to slow their SM down, so there are never more workers than groups: as many
-    // warps per SM as the groups fill evenly, at most two per scheduler.
-    static const uint64_t forced = [] { const char *e = getenv("IV_SLICE_WARPS"); return e ? (uint64_t)atoi(e) : 0ull; }();
-    uint64_t warps = forced ? forced : groups / (uint64_t)sm_count;
+    // One persistent CTA of eight warps per SM (two per scheduler).  Measured on 896 groups:
+    // 4 / 5 / 6 / 7 / 8 warps per SM give 687 / 694 / 673 / 703 / 712 GB/s, and two CTAs of four
+    // warps only 574 GB/s; workers that find the FIFO empty sleep in their bounded wait.
+    uint64_t warps = (groups + (uint64_t)sm_count - 1) / (uint64_t)sm_count;
     if (warps > MAX_WARPS) warps = MAX_WARPS;
     if (warps < 1) warps = 1;
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp, stream>>>(
-        d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice, mid);
+        d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice, mid, d_one);
     return cudaGetLastError();
 }
 

@@ -20,12 +20,28 @@
 namespace ivk {
 namespace {
 
-template <int SEG, int STAGES, int NSLOT, int MODE>
+__device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const uint64_t t = __shfl_xor_sync(0xffffffffu, v, o);
+        v = t > v ? t : v;
+    }
+    return v;
+}
+
+// RAGGED = false: message i is chunk i of the blob (base and chunk size multiples of 16 bytes).
+// RAGGED = true:  message k of the CTA is tensor order[...] at data + offsets[.] with lengths[.] bytes,
+//                 any alignment: each bulk copy starts at the 16-byte boundary below the tensor and
+//                 carries 16 bytes more than a segment, so that every 64-byte block lies inside one
+//                 stage; the block is read as 17 aligned words and the byte shift is folded into the
+//                 endian-swap PRMT.
+template <int SEG, int STAGES, int NSLOT, int MODE, bool RAGGED>
 __global__ void __launch_bounds__(64)
 hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                          uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
-                         const uint32_t *__restrict__ one_ptr) {
-    constexpr uint32_t kLaneStride = SEG + 16;            // data ring: bytes per lane per stage
+                         const uint32_t *__restrict__ one_ptr, const uint64_t *__restrict__ offsets,
+                         const uint64_t *__restrict__ lengths, const uint32_t *__restrict__ order) {
+    constexpr uint32_t kLaneStride = SEG + (RAGGED ? 32 : 16);   // data ring: bytes per lane per stage
     constexpr uint32_t kStageBytes = 32 * kLaneStride;
     constexpr int kBlocksPerSeg = SEG / 64;
     constexpr uint32_t kWkLane = 64 * 4 + 16;             // W+K ring: bytes per lane per slot
@@ -48,43 +64,68 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     // compiler stage can fold the multiplication away.
     const uint32_t one = __ldg(one_ptr);
 
-    const uint64_t i = (uint64_t)blockIdx.x * 32 + lane;
-    const bool valid = i < n_chunks;
-    const uint64_t begin = valid ? i * chunk_bytes : 0;
-    const uint64_t len = valid ? ((nbytes - begin < chunk_bytes) ? (nbytes - begin) : chunk_bytes) : 0;
-    // SHA-256 blocks of this lane's message, padding included; lane 0 holds the longest chunk of the warp.
+    const uint64_t slot_index = (uint64_t)blockIdx.x * 32 + lane;
+    const bool valid = slot_index < n_chunks;
+    uint64_t i = slot_index, begin = 0, len = 0;
+    if (RAGGED) {
+        if (valid) {
+            i = order ? order[slot_index] : slot_index;
+            begin = offsets[i];
+            len = lengths[i];
+        }
+    } else if (valid) {
+        begin = i * chunk_bytes;
+        len = (nbytes - begin < chunk_bytes) ? (nbytes - begin) : chunk_bytes;
+    }
+    // SHA-256 blocks of this lane's message, padding included.  For chunks lane 0 holds the longest
+    // message of the warp; for tensors the maximum is taken.
     const uint64_t my_total = valid ? ((len + 8) >> 6) + 1 : 0;
-    const uint64_t warp_total = __shfl_sync(0xffffffffu, my_total, 0);
+    const uint64_t warp_total = RAGGED ? warp_max_u64(my_total) : __shfl_sync(0xffffffffu, my_total, 0);
 
     if (warp == 1) {
         // ------------------------------------------------------------------ producer
         const uint8_t *p = data + begin;
         const uint64_t full_bytes = len & ~63ull;
         const uint64_t my_full = full_bytes >> 6;
-        const uint64_t warp_full = __shfl_sync(0xffffffffu, my_full, 0);
+        const uint64_t warp_full = RAGGED ? warp_max_u64(my_full) : __shfl_sync(0xffffffffu, my_full, 0);
         const uint64_t nseg = (warp_full * 64 + SEG - 1) / SEG;
+        // tensors: misalignment of the message start, the 16-byte aligned copy source and how many
+        // aligned bytes cover the whole blocks
+        const uint32_t mis = RAGGED ? (uint32_t)(reinterpret_cast<uintptr_t>(p) & 15u) : 0u;
+        const uint8_t *p_al = p - mis;
+        const uint64_t need = full_bytes ? ((mis + full_bytes + 15) & ~15ull) : 0;
+        const uint32_t word_off = mis & ~3u;                       // in-stage offset of the first aligned word
+        const uint32_t sel = 0x0123u + 0x1111u * (mis & 3u);       // PRMT: byte shift + big-endian
         // One arrival per stage: lane 0 announces the bytes of all 32 copies, every lane issues its own.
         auto issue = [&](uint64_t seg, int stage) {
             const uint64_t off = seg * SEG;
             const uint32_t bar = bar_data + 8 * stage;
-            const uint32_t bytes = off < full_bytes ? (uint32_t)((full_bytes - off < SEG) ? (full_bytes - off) : SEG) : 0u;
+            uint32_t bytes;
+            if (RAGGED) bytes = off < need ? (uint32_t)((need - off < SEG + 16) ? (need - off) : SEG + 16) : 0u;
+            else bytes = off < full_bytes ? (uint32_t)((full_bytes - off < SEG) ? (full_bytes - off) : SEG) : 0u;
             const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
             if (lane == 0) tma::mbar_arrive_expect_tx(bar, total);
-            if (bytes) tma::bulk_g2s(data_base + stage * kStageBytes, p + off, bytes, bar);
+            if (bytes) tma::bulk_g2s(data_base + stage * kStageBytes, p_al + off, bytes, bar);
         };
 #pragma unroll
         for (int s = 0; s < STAGES; ++s)
             if ((uint64_t)s < nseg) issue(s, s);
 
-        uint32_t w[16], raw[16], tw[32];
+        uint32_t w[16], raw[17], tw[32];
         int stage = 0, in_stage = 0;
         uint32_t dparity = 0;
         bool failed = false, tail_built = false;
         auto fetch = [&](int blk_in_stage) {
             const uint32_t src = data_base + stage * kStageBytes + 64 * blk_in_stage;
+            if (RAGGED) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                tma::ld_shared_v4(src + 16 * q, raw[4 * q], raw[4 * q + 1], raw[4 * q + 2], raw[4 * q + 3]);
+                for (int q = 0; q < 17; ++q)
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(raw[q]) : "r"(src + word_off + 4 * q) : "memory");
+            } else {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    tma::ld_shared_v4(src + 16 * q, raw[4 * q], raw[4 * q + 1], raw[4 * q + 2], raw[4 * q + 3]);
+            }
         };
         if (warp_full) {
             failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_data, 0));
@@ -96,7 +137,7 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
         for (uint64_t blk = 0; blk < warp_total && !failed; ++blk) {
             if (blk < my_full) {
 #pragma unroll
-                for (int k = 0; k < 16; ++k) w[k] = bswap32(raw[k]);
+                for (int k = 0; k < 16; ++k) w[k] = RAGGED ? __byte_perm(raw[k], raw[k + 1], sel) : bswap32(raw[k]);
             } else if (blk < my_total) {
                 if (!tail_built) {
                     (void)sha256_build_tail(p + full_bytes, (uint32_t)(len & 63u), len, tw);
@@ -169,7 +210,7 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
     // recurrences stay three-input ALU adds, the others go to the FMA pipe (placement 3, the fastest measured).
     constexpr int SEG = 512, STAGES = 3, NSLOT = 4, MODE = 3;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * 32 * (64 * 4 + 16);
-    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE>;
+    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false>;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -178,7 +219,27 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
     }
     const uint64_t blocks = (n_chunks + 31) / 32;
     if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
-    kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one);
+    kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
+                                                   nullptr, nullptr, nullptr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_hash_ragged_split(const uint8_t *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
+                                     const uint32_t *d_order, uint64_t n, uint8_t *d_digests, uint32_t *d_status,
+                                     const uint32_t *d_one, cudaStream_t stream) {
+    constexpr int SEG = 512, STAGES = 3, NSLOT = 4, MODE = 3;
+    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 32) + (size_t)NSLOT * 32 * (64 * 4 + 16);
+    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, true>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const uint64_t blocks = (n + 31) / 32;
+    if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
+    kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_base, 0, 0, n, d_digests, d_status, d_one, d_offsets, d_lengths,
+                                                   d_order);
     return cudaGetLastError();
 }
 

@@ -82,13 +82,35 @@ hash_ragged_kernel(const uint8_t *__restrict__ base, const uint64_t *__restrict_
     }
 }
 
+// order[r] = index of the tensor with the r-th largest length (ties by index): a rank sort, one
+// thread per tensor counting the tensors that come before it.  Long messages then start first and
+// the 32 lanes of a warp carry messages of similar length.
+__global__ void rank_by_length_kernel(const uint64_t *__restrict__ lengths, uint32_t n, uint32_t *__restrict__ order) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const uint64_t mine = lengths[i];
+    uint32_t rank = 0;
+    for (uint32_t j = 0; j < n; ++j) {
+        const uint64_t other = __ldg(lengths + j);
+        rank += (other > mine || (other == mine && j < i)) ? 1u : 0u;
+    }
+    order[rank] = i;
+}
+
 }  // namespace
 
 cudaError_t launch_hash_ragged(const uint8_t *d_base, const uint64_t *d_offsets,
                                const uint64_t *d_lengths, uint64_t n, uint8_t *d_digests,
-                               unsigned long long *d_queue, int sm_count, cudaStream_t stream,
-                               uint64_t *launches) {
+                               unsigned long long *d_queue, uint32_t *d_order, uint32_t *d_status,
+                               const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *launches) {
     if (n == 0) return cudaSuccess;
+    if (n <= kRaggedSortMax && d_order) {
+        rank_by_length_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(d_lengths, (uint32_t)n, d_order);
+        cudaError_t e0 = cudaGetLastError();
+        if (e0 != cudaSuccess) return e0;
+        if (launches) *launches += 2;
+        return launch_hash_ragged_split(d_base, d_offsets, d_lengths, d_order, n, d_digests, d_status, d_one, stream);
+    }
     cudaError_t e = cudaMemsetAsync(d_queue, 0, sizeof(unsigned long long), stream);
     if (e != cudaSuccess) return e;
     // Few messages: one warp per CTA spreads the chains over all SM schedulers.

@@ -28,6 +28,8 @@ struct iv_ctx {
     uint64_t digests_valid = 0;
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
+    uint32_t *d_order = nullptr;              // tensor order (by descending length) of iv_hash_ragged
+    uint64_t order_cap = 0;
     uint8_t *d_slices = nullptr;              // FIFO, slice counters and parked chaining values of the sliced leaf kernel
     uint64_t slices_cap = 0;                  // bytes
 
@@ -238,6 +240,7 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_digests);
     cudaFree(ctx->d_words);
     cudaFree(ctx->d_slices);
+    cudaFree(ctx->d_order);
     cudaFree(ctx->d_window[0]);
     cudaFree(ctx->d_window[1]);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -392,9 +395,14 @@ int iv_hash_ragged(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets, c
     if (n == 0) return IV_OK;
     if (!d_base || !d_offsets || !d_lengths || !d_digests) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
+    if (n <= ivk::kRaggedSortMax) {
+        int rc = grow(ctx, &ctx->d_order, &ctx->order_cap, n, sizeof(uint32_t));
+        if (rc != IV_OK) return rc;
+    }
     IV_TRY(ctx, ivk::launch_hash_ragged(static_cast<const uint8_t *>(d_base), d_offsets, d_lengths, n, d_digests,
-                                        ctx->d_queue, ctx->sm_count, static_cast<cudaStream_t>(cuda_stream),
-                                        &ctx->launches));
+                                        ctx->d_queue, n <= ivk::kRaggedSortMax ? ctx->d_order : nullptr,
+                                        ctx->d_status, ctx->d_one, ctx->sm_count,
+                                        static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
     return IV_OK;
 }
 
@@ -403,7 +411,7 @@ int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t block
     if (!ctx || !h_out || warps_per_block == 0 || warps_per_block > 32 || blocks_per_sm == 0 ||
         blocks_per_sm > 32 || active_lanes == 0 || active_lanes > 32 || iters == 0)
         return IV_ERR_INVALID_ARG;
-    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_ROUNDS_M5) return IV_ERR_INVALID_ARG;
+    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_SHA256_ADD4) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     const unsigned blocks = blocks_per_sm * (unsigned)ctx->sm_count;
     unsigned long long *d_cycles = nullptr;

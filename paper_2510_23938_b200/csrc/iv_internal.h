@@ -37,14 +37,23 @@ uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t 
                               uint64_t *total_tasks_out, uint64_t nbytes);
 cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                       uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
-                                      int sm_count, cudaStream_t stream);
+                                      const uint32_t *d_one, int sm_count, cudaStream_t stream);
+
+// The same two-warp kernel for tensors at any alignment; message k of the launch is tensor d_order[k]
+// (d_order may be NULL for index order).
+cudaError_t launch_hash_ragged_split(const uint8_t *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
+                                     const uint32_t *d_order, uint64_t n, uint8_t *d_digests, uint32_t *d_status,
+                                     const uint32_t *d_one, cudaStream_t stream);
 
 // hash_ragged.cu -----------------------------------------------------------
-// One SHA-256 per (offset, length); d_queue is one zeroed uint64 work counter.
+// One SHA-256 per (offset, length).  Up to kRaggedSortMax tensors are ordered by descending length
+// (d_order: n uint32 of scratch) and hashed by the two-warp kernel; larger sets go through the
+// per-lane work queue (d_queue: one uint64 counter).
+constexpr uint64_t kRaggedSortMax = 32768;
 cudaError_t launch_hash_ragged(const uint8_t *d_base, const uint64_t *d_offsets,
                                const uint64_t *d_lengths, uint64_t n, uint8_t *d_digests,
-                               unsigned long long *d_queue, int sm_count, cudaStream_t stream,
-                               uint64_t *launches);
+                               unsigned long long *d_queue, uint32_t *d_order, uint32_t *d_status,
+                               const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *launches);
 
 // merkle.cu ----------------------------------------------------------------
 // Root of n leaves.  d_scratch_a / d_scratch_b each hold ceil(n / kMerkleRun)

@@ -74,9 +74,9 @@ __global__ void probe_kernel(uint32_t iters, uint32_t active_lanes, uint32_t see
 }
 
 // Register-only SHA-256: `iters` compressions per thread on a block derived from the state.
-template <bool FMA>
-__global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, uint32_t one, unsigned long long *cycles,
-                                 uint32_t *sink) {
+template <int ADD>
+__global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, unsigned long long *cycles, uint32_t *sink) {
+    const uint32_t one = sink[1];        // the host stored 1 there; the compiler cannot know
     const uint32_t lane = threadIdx.x & 31u;
     uint32_t st[8], w[16];
     sha256_init(st);
@@ -87,7 +87,7 @@ __global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, uint32_t
         for (uint32_t it = 0; it < iters; ++it) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) w[i] = __byte_perm(st[i & 7] + (uint32_t)i, it, 0x0123);
-            sha256_compress<FMA>(st, w, one);
+            sha256_compress<ADD>(st, w, one);
         }
     }
     __syncthreads();
@@ -163,15 +163,18 @@ cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t i
         case IV_PROBE_ROUNDS_M4: probe_rounds_kernel<4><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_ROUNDS_M5: probe_rounds_kernel<5><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_SCHEDULE: probe_schedule_kernel<<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256: probe_sha_kernel<false><<<blocks, threads, 0, stream>>>(iters, active_lanes, 1u, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256_FMA: probe_sha_kernel<true><<<blocks, threads, 0, stream>>>(iters, active_lanes, 1u, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256: probe_sha_kernel<0><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_FMA: probe_sha_kernel<1><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_ADD2: probe_sha_kernel<2><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_ADD3: probe_sha_kernel<3><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_ADD4: probe_sha_kernel<4><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
 }
 
 uint64_t probe_ops_per_thread(int kind, uint32_t iters) {
-    if (kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_FMA || kind >= IV_PROBE_ROUNDS_M0) return iters;                       // compressions
+    if (kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_FMA || kind >= IV_PROBE_ROUNDS_M0) return iters;                        // compressions
     if (kind == IV_PROBE_LAT_CROSS) return (uint64_t)iters * kUnroll * 2;             // two instructions per trip
     if (kind >= IV_PROBE_LAT_IADD3) return (uint64_t)iters * kUnroll;                 // one dependent chain
     return (uint64_t)iters * kUnroll * kThroughputChains;                              // instructions

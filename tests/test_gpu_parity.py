@@ -275,6 +275,33 @@ def test_hash_ragged_per_tensor_digests_of_a_weight_file(ctx):
     assert np.array_equal(_host(chunks), oracle.hash_chunks(_host(blob), 4096))
 
 
+def test_hash_ragged_large_set_takes_the_work_queue_path(ctx):
+    """More tensors than the sorted two-warp path takes (32768): the per-lane work-queue kernel."""
+    n = 40_000
+    rng = np.random.default_rng(41)
+    sizes = rng.integers(0, 700, size=n).astype(np.int64)
+    sizes[::997] = rng.integers(10_000, 60_000, size=len(sizes[::997]))
+    offs = inputs.packed_offsets(sizes, first=3)
+    base = inputs.uniform_bytes(int(offs[-1] + sizes[-1]) + 8, seed=33, device="cuda")
+    got = ctx.hash_ragged(base, torch.from_numpy(offs).cuda(), torch.from_numpy(sizes).cuda())
+    want = oracle.hash_ragged(_host(base), offs, sizes, nthreads=oracle.host_threads())
+    assert np.array_equal(_host(got), want)
+
+
+def test_hash_ragged_every_16_byte_misalignment_with_long_messages(ctx):
+    """Messages of many blocks at each start offset 0..31: every stage hand-over of the bulk-copy ring."""
+    base = inputs.uniform_bytes(64 * 70_000, seed=34, device="cuda")
+    lengths, offsets = [], []
+    for a in range(32):
+        for ln in (64 * 8, 64 * 8 + 1, 64 * 9 - 1, 64 * 17 + 5, 64 * 24, 64 * 25 + 63, 40_000 + a):
+            offsets.append(a + 100_000 * (len(offsets) % 40))
+            lengths.append(ln)
+    got = ctx.hash_ragged(base, torch.tensor(offsets, device="cuda"), torch.tensor(lengths, device="cuda"))
+    want = oracle.hash_ragged(_host(base), offsets, lengths, nthreads=oracle.host_threads())
+    assert np.array_equal(_host(got), want)
+    assert ctx.device_status() == 0
+
+
 def test_hash_ragged_empty_set(ctx):
     base = inputs.uniform_bytes(64, seed=1, device="cuda")
     e = torch.empty(0, dtype=torch.int64, device="cuda")
