@@ -126,9 +126,15 @@ def _physical_gpu_index(local_rank: int) -> int:
 # --------------------------------------------------------------------------------------------
 # workloads
 
-def build_workload(cfg_id: int, device, seed: int):
+def build_workload(cfg_id: int, device, seed: int, nbytes_override=None, chunk_override=None):
     from paper_2510_23938_b200 import inputs
     cfg = dict(CONFIGS[cfg_id])
+    if nbytes_override or chunk_override:
+        if nbytes_override and "nbytes" in cfg:
+            cfg["nbytes"] = int(nbytes_override) & ~1
+        if chunk_override and cfg.get("chunk"):
+            cfg["chunk"] = int(chunk_override)
+        cfg["name"] = f"custom (from config{cfg_id}): {cfg.get('nbytes', 'file')} bytes, {cfg.get('chunk')}-byte chunks"
     if cfg["kind"] == "uniform":
         data = inputs.uniform_bytes(cfg["nbytes"], seed, device)
     elif cfg["kind"] == "bf16":
@@ -191,7 +197,7 @@ def run_ours(args):
     cfg_id, fallback = pick_config(args.config, device)
     ctx = binding.Context(local_rank)
     t_setup = time.time()
-    wl = build_workload(cfg_id, device, seed=1000 + rank)
+    wl = build_workload(cfg_id, device, seed=1000 + rank, nbytes_override=args.nbytes, chunk_override=args.chunk)
     data, nbytes, chunk = wl["data"], wl["nbytes"], wl["chunk"]
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
@@ -273,7 +279,7 @@ def run_ours(args):
     peak_gbs = SM_COUNT * INT_LANES_PER_SM * 1.965e9 / INT_OPS_PER_BYTE / 1e9
     achieved = nbytes / (hash_ms * 1e-3) / 1e9
     roofline = {
-        "bound": "alu", "kernel": "hash_ragged_kernel" if ragged else "hash_chunks_kernel",
+        "bound": "alu", "kernel": ctx.last_leaf_kernel,
         "achieved": round(achieved, 2), "peak": round(peak_gbs, 1), "unit": "GB/s",
         "frac": round(achieved / peak_gbs, 4), "traffic": None,
         "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1.965 GHz / 21.875 INT32 ops per byte",
@@ -471,6 +477,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=None, choices=sorted(CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--nbytes", type=int, default=None, help="override the blob size of configs 1 and 4 (profiling)")
+    ap.add_argument("--chunk", type=int, default=None, help="override the chunk size (profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -72,6 +72,11 @@ int iv_device_status(iv_ctx *ctx, uint32_t *h_status);
 /* Number of kernels this context has launched so far (a host-side counter). */
 uint64_t iv_kernel_launches(const iv_ctx *ctx);
 
+/* Name of the leaf-hashing kernel the last hashing or verification call on this context launched
+ * (the library picks one of several by chain count, chunk size and alignment); "" before any call.
+ * Static text, never freed. */
+const char *iv_last_leaf_kernel(const iv_ctx *ctx);
+
 /* ---------------------------------------------------------------------------
  * Leaf hashing -- Algorithm 1, "chunk_count <- ceil(|M| / C)" and
  * "H_i = GPU_HASH(M_i)" with GPU_HASH = SHA-256 (FIPS 180-4 section 6.2).

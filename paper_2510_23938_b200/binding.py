@@ -28,7 +28,7 @@ EXPORTS = (
     "iv_create", "iv_destroy", "iv_strerror", "iv_last_cuda_error", "iv_kernel_launches",
     "iv_hash_chunks", "iv_merkle_root", "iv_verify_manifest", "iv_ctx_digests",
     "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
-    "iv_merkle_root_noalloc",
+    "iv_merkle_root_noalloc", "iv_last_leaf_kernel",
 )
 
 
@@ -96,6 +96,8 @@ def load_library() -> ctypes.CDLL:
     lib.iv_hash_ragged.restype = i32
     lib.iv_merkle_root_noalloc.argtypes = [vp, u64, vp, vp]
     lib.iv_merkle_root_noalloc.restype = i32
+    lib.iv_last_leaf_kernel.argtypes = [vp]
+    lib.iv_last_leaf_kernel.restype = ctypes.c_char_p
     lib.iv_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.iv_device_status.restype = i32
     lib.iv_probe_alu.argtypes = [vp, i32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
@@ -254,6 +256,10 @@ class Context:
                                       _dev_ptr(out), _stream_ptr(stream))
         self._check(rc, "iv_hash_ragged")
         return out
+
+    @property
+    def last_leaf_kernel(self) -> str:
+        return self._lib.iv_last_leaf_kernel(self._h).decode()
 
     def device_status(self) -> int:
         """iv_device_status: waits for the device, returns and clears the device-side status word."""

@@ -246,7 +246,9 @@ bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint6
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
                                const uint32_t *d_one, void *d_slice_scratch, cudaStream_t stream,
-                               uint64_t *launches) {
+                               uint64_t *launches, const char **kernel_used) {
+    const char *unused = nullptr;
+    if (!kernel_used) kernel_used = &unused;
     if (n_chunks == 0) return cudaSuccess;
     if (launches) ++*launches;
     const uint64_t warps = (n_chunks + 31) / 32;
@@ -254,19 +256,24 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
     if (aligned && chunk_bytes >= 4096) {
         // Few chains: one warp per CTA, so every chain warp gets an SM scheduler of its own and a deep ring.
         // Two warps per 32 chains while every warp can still have an SM scheduler of its own.
-        if (warps <= 2ull * sm_count)
+        if (warps <= 2ull * sm_count) {
+            *kernel_used = "hash_chunks_split_kernel";
             return launch_hash_chunks_split(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one, stream);
+        }
+        *kernel_used = "hash_chunks_staged_kernel";
         if (warps <= 4ull * sm_count)
             return launch_staged<512, 3, 1, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);
         // Many chains of sliceable size: chains migrate between schedulers (two launches: queue set-up + workers).
         if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
             if (launches) ++*launches;
+            *kernel_used = "hash_chunks_sliced_kernel";
             return launch_hash_chunks_sliced(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
                                              d_slice_scratch, d_one, sm_count, stream);
         }
         // Many small chunks: two CTAs of four warps per SM keep two warps on every scheduler.
         return launch_staged<256, 3, 4, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);
     }
+    *kernel_used = "hash_chunks_kernel";
     const unsigned warps_per_cta = warps <= (uint64_t)sm_count ? 1u : (warps <= 2ull * sm_count ? 2u : 4u);
     const unsigned threads = 32u * warps_per_cta;
     const uint64_t blocks = (n_chunks + threads - 1) / threads;

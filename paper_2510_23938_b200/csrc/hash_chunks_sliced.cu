@@ -274,9 +274,7 @@ cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, ui
     // One persistent CTA of eight warps per SM (two per scheduler).  Measured on 896 groups:
     // 4 / 5 / 6 / 7 / 8 warps per SM give 687 / 694 / 673 / 703 / 712 GB/s, and two CTAs of four
     // warps only 574 GB/s; workers that find the FIFO empty sleep in their bounded wait.
-    uint64_t warps = (groups + (uint64_t)sm_count - 1) / (uint64_t)sm_count;
-    if (warps > MAX_WARPS) warps = MAX_WARPS;
-    if (warps < 1) warps = 1;
+    const uint64_t warps = MAX_WARPS;
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp, stream>>>(
         d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice, mid, d_one);
     return cudaGetLastError();

@@ -102,13 +102,17 @@ __global__ void rank_by_length_kernel(const uint64_t *__restrict__ lengths, uint
 cudaError_t launch_hash_ragged(const uint8_t *d_base, const uint64_t *d_offsets,
                                const uint64_t *d_lengths, uint64_t n, uint8_t *d_digests,
                                unsigned long long *d_queue, uint32_t *d_order, uint32_t *d_status,
-                               const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *launches) {
+                               const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *launches,
+                               const char **kernel_used) {
+    const char *unused = nullptr;
+    if (!kernel_used) kernel_used = &unused;
     if (n == 0) return cudaSuccess;
     if (n <= kRaggedSortMax && d_order) {
         rank_by_length_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(d_lengths, (uint32_t)n, d_order);
         cudaError_t e0 = cudaGetLastError();
         if (e0 != cudaSuccess) return e0;
         if (launches) *launches += 2;
+        *kernel_used = "hash_chunks_split_kernel (tensors)";
         return launch_hash_ragged_split(d_base, d_offsets, d_lengths, d_order, n, d_digests, d_status, d_one, stream);
     }
     cudaError_t e = cudaMemsetAsync(d_queue, 0, sizeof(unsigned long long), stream);
@@ -125,6 +129,7 @@ cudaError_t launch_hash_ragged(const uint8_t *d_base, const uint64_t *d_offsets,
         const uint64_t cap = 2ull * (uint64_t)sm_count;
         blocks = (unsigned)(want < cap ? want : cap);
     }
+    *kernel_used = "hash_ragged_kernel";
     hash_ragged_kernel<<<blocks, threads, 0, stream>>>(d_base, d_offsets, d_lengths, n, d_digests, d_queue);
     if (launches) ++*launches;
     return cudaGetLastError();

@@ -11,6 +11,7 @@ struct iv_ctx {
     int sm_count = 0;
     int last_cuda_error = 0;
     uint64_t launches = 0;
+    const char *leaf_kernel = "";             // name of the leaf-hashing kernel the last call launched
 
     // small fixed block: tickets, work-queue counter, root
     uint32_t *d_tickets = nullptr;            // kMerkleMaxPasses + 1 words
@@ -115,7 +116,7 @@ int hash_leaves(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t ch
         scratch = ctx->d_slices;
     }
     IV_TRY(ctx, ivk::launch_hash_chunks(d_data, nbytes, chunk_bytes, n, d_digests, ctx->sm_count, ctx->d_status,
-                                        ctx->d_one, scratch, stream, &ctx->launches));
+                                        ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel));
     return IV_OK;
 }
 
@@ -261,6 +262,8 @@ int iv_last_cuda_error(const iv_ctx *ctx) { return ctx ? ctx->last_cuda_error : 
 
 uint64_t iv_kernel_launches(const iv_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
+const char *iv_last_leaf_kernel(const iv_ctx *ctx) { return ctx ? ctx->leaf_kernel : ""; }
+
 int iv_device_status(iv_ctx *ctx, uint32_t *h_status) {
     if (!ctx || !h_status) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
@@ -402,7 +405,7 @@ int iv_hash_ragged(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets, c
     IV_TRY(ctx, ivk::launch_hash_ragged(static_cast<const uint8_t *>(d_base), d_offsets, d_lengths, n, d_digests,
                                         ctx->d_queue, n <= ivk::kRaggedSortMax ? ctx->d_order : nullptr,
                                         ctx->d_status, ctx->d_one, ctx->sm_count,
-                                        static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+                                        static_cast<cudaStream_t>(cuda_stream), &ctx->launches, &ctx->leaf_kernel));
     return IV_OK;
 }
 

@@ -18,7 +18,7 @@ constexpr uint32_t kMerkleRun = 512;
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
                                const uint32_t *d_one, void *d_slice_scratch, cudaStream_t stream,
-                               uint64_t *launches);
+                               uint64_t *launches, const char **kernel_used);
 // True when launch_hash_chunks would use the sliced kernel (and so needs its scratch).
 bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count);
 
@@ -53,7 +53,8 @@ constexpr uint64_t kRaggedSortMax = 32768;
 cudaError_t launch_hash_ragged(const uint8_t *d_base, const uint64_t *d_offsets,
                                const uint64_t *d_lengths, uint64_t n, uint8_t *d_digests,
                                unsigned long long *d_queue, uint32_t *d_order, uint32_t *d_status,
-                               const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *launches);
+                               const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *launches,
+                               const char **kernel_used);
 
 // merkle.cu ----------------------------------------------------------------
 // Root of n leaves.  d_scratch_a / d_scratch_b each hold ceil(n / kMerkleRun)
