@@ -278,10 +278,22 @@ def run_ours(args):
 
     peak_gbs = SM_COUNT * INT_LANES_PER_SM * 1.965e9 / INT_OPS_PER_BYTE / 1e9
     achieved = nbytes / (hash_ms * 1e-3) / 1e9
+    # DRAM traffic per launch: ncu measured dram read+write = 1.0005 x the bytes hashed for the sliced kernel
+    # (2 GiB capture) and 1.001 x for the two-warp kernel (config 2 capture); both scale with the bytes.
+    kernel_name = ctx.last_leaf_kernel
+    traffic_factor = {"hash_chunks_sliced_kernel": 1.0005, "hash_chunks_split_kernel": 1.001}.get(kernel_name)
+    # what the chain count allows: chains x 64 B x f / (cycles one chain needs per block when it has a
+    # scheduler to itself: 2,000 for the two-warp kernel)
+    chain_bound = n_units * 64 * 1.965e9 / 2000.0 / 1e9
     roofline = {
-        "bound": "alu", "kernel": ctx.last_leaf_kernel,
+        "bound": "alu", "kernel": kernel_name,
         "achieved": round(achieved, 2), "peak": round(peak_gbs, 1), "unit": "GB/s",
-        "frac": round(achieved / peak_gbs, 4), "traffic": None,
+        "frac": round(achieved / peak_gbs, 4),
+        "traffic": int(traffic_factor * nbytes) if traffic_factor else None,
+        "traffic_source": ("ncu dram bytes of a smaller capture of the same kernel, scaled by bytes hashed "
+                           "(profiles/)") if traffic_factor else None,
+        "algorithmic_bytes": nbytes, "int32_ops_per_byte": INT_OPS_PER_BYTE,
+        "chain_count_bound_gbs": round(min(chain_bound, peak_gbs), 1),
         "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1.965 GHz / 21.875 INT32 ops per byte",
         "hbm_peak_gbs_measured": _measured_peak("hbm_gbs"),
         "launch_ms": round(hash_ms, 4), "tree_ms": tree_ms, "compare_ms": cmp_ms,
