@@ -110,6 +110,21 @@ int iv_hash_chunks(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t ch
 int iv_merkle_root(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
                    void *cuda_stream);
 
+/* `levels` levels of the same reduction without going all the way to the root:
+ * d_nodes[n] -> d_out[n_out], n_out = n halved (rounding up) `levels` times.  Node j
+ * of the result is the root of the aligned run of 2^levels inputs starting at
+ * j * 2^levels, which is also a node of the whole tree -- the building block for
+ * the paper's multi-GPU scheme ("global Merkle trees from distributed hash
+ * computations", section "Multi-GPU Deployment Architectures"): every GPU
+ * reduces its aligned range of leaves to such nodes, the nodes are gathered, and
+ * iv_merkle_root over them gives the global root.
+ *   d_out, out_cap   receives n_out records; out_cap (in records) must be >= n_out;
+ *                    must not overlap d_nodes
+ *   h_n_out          optional host pointer, receives n_out
+ */
+int iv_merkle_levels(iv_ctx *ctx, const uint8_t *d_nodes, uint64_t n, uint32_t levels,
+                     uint8_t *d_out, uint64_t out_cap, uint64_t *h_n_out, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------
  * Verification -- Algorithm 1, "Compare root hash with expected value", plus
  * the per-chunk comparison that locates the damage.

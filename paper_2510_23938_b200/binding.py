@@ -28,7 +28,7 @@ EXPORTS = (
     "iv_create", "iv_destroy", "iv_strerror", "iv_last_cuda_error", "iv_kernel_launches",
     "iv_hash_chunks", "iv_merkle_root", "iv_verify_manifest", "iv_ctx_digests",
     "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
-    "iv_merkle_root_noalloc", "iv_last_leaf_kernel",
+    "iv_merkle_root_noalloc", "iv_last_leaf_kernel", "iv_merkle_levels",
 )
 
 
@@ -81,6 +81,8 @@ def load_library() -> ctypes.CDLL:
     lib.iv_hash_chunks.restype = i32
     lib.iv_merkle_root.argtypes = [vp, vp, u64, vp, vp]
     lib.iv_merkle_root.restype = i32
+    lib.iv_merkle_levels.argtypes = [vp, vp, u64, ctypes.c_uint32, vp, u64, ctypes.POINTER(u64), vp]
+    lib.iv_merkle_levels.restype = i32
     lib.iv_verify_manifest.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest.restype = i32
     lib.iv_ctx_digests.argtypes = [vp]
@@ -196,6 +198,22 @@ class Context:
             out = torch.empty(32, dtype=torch.uint8, device=leaves.device)
         rc = self._lib.iv_merkle_root(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
         self._check(rc, "iv_merkle_root")
+        return out
+
+    def merkle_levels(self, nodes: torch.Tensor, levels: int, stream=None) -> torch.Tensor:
+        """iv_merkle_levels: the (ceil(n / 2^levels), 32) nodes `levels` levels above `nodes`."""
+        n = nodes.numel() // 32
+        n_out = n
+        for _ in range(levels):
+            if n_out <= 1:
+                break
+            n_out = (n_out + 1) // 2
+        out = torch.empty((n_out, 32), dtype=torch.uint8, device=nodes.device)
+        got = ctypes.c_uint64(0)
+        rc = self._lib.iv_merkle_levels(self._h, _dev_ptr(nodes), n, levels, _dev_ptr(out), n_out,
+                                        ctypes.byref(got), _stream_ptr(stream))
+        self._check(rc, "iv_merkle_levels")
+        assert got.value == n_out
         return out
 
     def make_manifest(self, total_bytes: int, chunk_bytes: int, digests: torch.Tensor, root: bytes) -> Manifest:

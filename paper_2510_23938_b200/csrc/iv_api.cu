@@ -300,6 +300,43 @@ int iv_merkle_root(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint
     return IV_OK;
 }
 
+int iv_merkle_levels(iv_ctx *ctx, const uint8_t *d_nodes, uint64_t n, uint32_t levels, uint8_t *d_out,
+                     uint64_t out_cap, uint64_t *h_n_out, void *cuda_stream) {
+    if (!ctx || levels > 63) return IV_ERR_INVALID_ARG;
+    uint64_t n_out = n;
+    for (uint32_t l = 0; l < levels && n_out > 1; ++l) n_out = (n_out + 1) / 2;
+    if (h_n_out) *h_n_out = n_out;
+    if (n == 0) return IV_OK;
+    if (!d_nodes || !d_out || n_out > out_cap) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (levels == 0 || n == 1) {
+        IV_TRY(ctx, cudaMemcpyAsync(d_out, d_nodes, 32 * n, cudaMemcpyDeviceToDevice, stream));
+        return IV_OK;
+    }
+    // up to nine levels per launch; intermediate level arrays ping-pong through the context's scratch
+    int rc = ensure_merkle_scratch(ctx, n);       // an intermediate array exists only after nine levels: n / 512 records
+    if (rc != IV_OK) return rc;
+    const uint8_t *in = d_nodes;
+    uint64_t cur = n;
+    uint32_t left = levels;
+    uint8_t *ping = ctx->d_merkle_a, *pong = ctx->d_merkle_b;
+    while (left > 0 && cur > 1) {
+        const uint32_t step = left > 9 ? 9 : left;
+        uint64_t next = cur;
+        for (uint32_t l = 0; l < step && next > 1; ++l) next = (next + 1) / 2;
+        const bool last = (left == step) || next == 1;
+        uint8_t *out = last ? d_out : ping;
+        IV_TRY(ctx, ivk::launch_merkle_levels(in, cur, step, out, stream, &ctx->launches));
+        in = out;
+        uint8_t *t = ping; ping = pong; pong = t;
+        cur = next;
+        left -= step;
+        if (last) break;
+    }
+    return IV_OK;
+}
+
 int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest *h_manifest,
                        iv_verify_result *d_result, uint64_t *d_mismatch_idx, uint64_t idx_cap,
                        void *cuda_stream) {

@@ -64,6 +64,10 @@ cudaError_t launch_merkle_root(const uint8_t *d_leaves, uint64_t n, uint8_t *d_r
                                uint8_t *d_scratch_a, uint8_t *d_scratch_b, uint32_t *d_tickets,
                                cudaStream_t stream, uint64_t *launches);
 
+// `levels` in 1..9 levels of the reduction: d_in[n] -> d_out[ceil(n / 2^levels)] (no aliasing).
+cudaError_t launch_merkle_levels(const uint8_t *d_in, uint64_t n, uint32_t levels, uint8_t *d_out,
+                                 cudaStream_t stream, uint64_t *launches);
+
 // Compare n computed digests with the manifest's, compact the mismatching
 // indices in ascending order, compare the root.  d_words holds ceil(n/32)
 // uint32 mask words; d_ticket one zeroed uint32.

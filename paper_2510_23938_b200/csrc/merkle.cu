@@ -110,6 +110,40 @@ merkle_pass_kernel(const uint8_t *__restrict__ nodes_in, uint64_t n, uint8_t *__
     if (threadIdx.x == 0) *ticket = 0u;   // ready for the next call
 }
 
+// `levels` (1..9) levels of the reduction on every aligned block of 512 input nodes:
+// nodes_in[n] -> nodes_out[ceil(n / 2^levels)].  Because pairing is index-aligned, the output is
+// exactly level `levels` of the tree over nodes_in (promotion can only happen at the very end).
+__global__ void __launch_bounds__(kThreads)
+merkle_levels_kernel(const uint8_t *__restrict__ nodes_in, uint64_t n, uint32_t levels,
+                     uint8_t *__restrict__ nodes_out) {
+    __shared__ __align__(16) uint32_t buf_a[kMerkleRun * 8];
+    __shared__ __align__(16) uint32_t buf_b[kMerkleRun * 4];
+    const uint64_t blocks = (n + kMerkleRun - 1) / kMerkleRun;
+    for (uint64_t r = blockIdx.x; r < blocks; r += gridDim.x) {
+        const uint64_t first = r * kMerkleRun;
+        uint32_t count = (uint32_t)((n - first < kMerkleRun) ? (n - first) : kMerkleRun);
+        load_nodes(nodes_in + 32 * first, count, buf_a, false);
+        uint32_t *a = buf_a, *b = buf_b;
+        for (uint32_t l = 0; l < levels && count > 1; ++l) {
+            const uint32_t parents = count >> 1;
+            for (uint32_t j = threadIdx.x; j < parents; j += blockDim.x) merkle_parent(a + 16 * j, b + 8 * j);
+            if ((count & 1u) && threadIdx.x < 8) b[8 * parents + threadIdx.x] = a[8 * (count - 1) + threadIdx.x];
+            __syncthreads();
+            uint32_t *t = a; a = b; b = t;
+            count = parents + (count & 1u);
+        }
+        // a block of 512 inputs yields 512 >> levels outputs (fewer for the ragged last block)
+        uint8_t *dst = nodes_out + 32 * (first >> levels);
+        for (uint32_t j = threadIdx.x; j < count; j += blockDim.x) {
+            uint32_t st[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) st[k] = a[8 * j + k];
+            store_digest(dst + 32 * (uint64_t)j, st);
+        }
+        __syncthreads();
+    }
+}
+
 // Root of zero leaves: SHA-256 of the empty string, computed here rather than typed in.
 __global__ void empty_root_kernel(uint8_t *d_root) {
     uint32_t st[8], w[16];
@@ -238,6 +272,15 @@ cudaError_t launch_merkle_root(const uint8_t *d_leaves, uint64_t n, uint8_t *d_r
         n = runs;
     }
     return cudaErrorInvalidValue;   // more than 512^8 leaves cannot be addressed
+}
+
+cudaError_t launch_merkle_levels(const uint8_t *d_in, uint64_t n, uint32_t levels, uint8_t *d_out,
+                                 cudaStream_t stream, uint64_t *launches) {
+    if (n == 0 || levels == 0 || levels > 9) return cudaErrorInvalidValue;
+    const uint64_t blocks = (n + kMerkleRun - 1) / kMerkleRun;
+    merkle_levels_kernel<<<(unsigned)(blocks < 4096 ? blocks : 4096), kThreads, 0, stream>>>(d_in, n, levels, d_out);
+    if (launches) ++*launches;
+    return cudaGetLastError();
 }
 
 cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_manifest_digests,

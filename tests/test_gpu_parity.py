@@ -122,6 +122,44 @@ def test_merkle_root_repeated_calls_reuse_scratch(ctx):
         assert _root_bytes(ctx.merkle_root(leaves)) == oracle.merkle_root(_host(leaves))
 
 
+@pytest.mark.parametrize("n,levels", [(1, 3), (2, 1), (5, 1), (5, 2), (5, 3), (5, 9), (511, 4), (512, 9), (513, 9),
+                                      (1000, 0), (1000, 1), (1000, 5), (1000, 10), (28_672, 6), (28_672, 12),
+                                      (300_001, 9), (300_001, 11), (300_001, 19), (300_001, 30)])
+def test_merkle_levels_equals_oracle_roots_of_aligned_runs(ctx, n, levels):
+    """Node j, `levels` levels up, is the root of the aligned run of 2^levels leaves (oracle per run)."""
+    leaves = inputs.uniform_bytes(32 * n, seed=500 + n + levels, device="cuda").view(n, 32)
+    got = _host(ctx.merkle_levels(leaves, levels))
+    host = _host(leaves)
+    run = 1 << min(levels, 40)
+    want = np.stack([np.frombuffer(oracle.merkle_root(host[s:s + run]), dtype=np.uint8) for s in range(0, n, run)])
+    assert np.array_equal(got, want)
+
+
+def test_sharded_root_emulated_ranks_on_one_gpu(ctx):
+    """The multi-GPU plan with every rank's share computed in turn on this GPU: chunk digests of the rank's
+    chunk range, iv_merkle_levels, nodes concatenated in rank order, iv_merkle_root == oracle root."""
+    from paper_2510_23938_b200 import sharded
+    chunk = 4096
+    data = inputs.uniform_bytes(chunk * 2510 - 99, seed=61, device="cuda")
+    n = binding.n_chunks(data.numel(), chunk)
+    want = oracle.merkle_root(oracle.hash_chunks(_host(data), chunk, nthreads=oracle.host_threads()))
+    for world in (1, 2, 3, 8):
+        plan = sharded.plan_shards(n, world)
+        parts = []
+        for rank in range(world):
+            lo, hi = plan.leaf_ranges[rank]
+            shard = data[lo * chunk:min(hi * chunk, data.numel())]
+            digests = ctx.hash_chunks(shard, chunk)
+            assert digests.shape[0] == hi - lo
+            if hi > lo:
+                parts.append(ctx.merkle_levels(digests, plan.level))
+        assert _root_bytes(ctx.merkle_root(torch.cat(parts))) == want
+    # and the collective entry point with a world of one
+    plan = sharded.plan_shards(n, 1)
+    root = sharded.sharded_root(ctx, ctx.hash_chunks(data, chunk), plan, 0)
+    assert _root_bytes(root) == want
+
+
 # ------------------------------------------------------------------------------------------ a4
 
 def _manifest_from_oracle(ctx, host_blob: np.ndarray, chunk: int):
