@@ -31,11 +31,15 @@ class ShardPlan:
         return max((hi - lo for lo, hi in self.node_ranges), default=0)
 
 
-def plan_shards(n_leaves: int, world: int) -> ShardPlan:
-    """Contiguous, 2^k-aligned leaf ranges, as even as the alignment allows (some may be empty)."""
-    assert n_leaves >= 0 and world >= 1
+def plan_shards(n_leaves: int, world: int, min_nodes_per_rank: int = 1) -> ShardPlan:
+    """Contiguous, 2^k-aligned leaf ranges, as even as the alignment allows (some may be empty).
+
+    A rank's share is a whole number of 2^k-leaf runs, so a large k makes the shares uneven;
+    `min_nodes_per_rank` trades a few more gathered nodes (32 bytes each) for balance: with 64 the
+    shares differ by at most one part in 64."""
+    assert n_leaves >= 0 and world >= 1 and min_nodes_per_rank >= 1
     level = 0
-    while (2 << level) * world <= n_leaves:          # largest k with 2^k * world <= n_leaves
+    while (2 << level) * world * min_nodes_per_rank <= n_leaves:   # largest k with 2^k * world * m <= n_leaves
         level += 1
     run = 1 << level
     n_nodes = -(-n_leaves // run)

@@ -49,6 +49,17 @@ def test_plan_is_aligned_contiguous_and_complete(world):
             assert all(hi > lo for lo, hi in p.node_ranges), (n, world)     # every rank has work
 
 
+def test_balanced_plan_for_equal_shards():
+    """With at least 64 nodes per rank the benchmark's shards (28,672 chunks per GPU) come out exactly equal."""
+    for world in (2, 4, 8):
+        p = sharded.plan_shards(world * 28_672, world, min_nodes_per_rank=64)
+        assert all(hi - lo == 28_672 for lo, hi in p.leaf_ranges)
+        assert p.level == 8 and p.n_nodes == world * 112
+    p = sharded.plan_shards(1000, 3, min_nodes_per_rank=64)
+    sizes = [hi - lo for lo, hi in p.leaf_ranges]
+    assert sum(sizes) == 1000 and max(sizes) - min(sizes) <= 2 * (1 << p.level)
+
+
 def test_single_process_emulation_of_ranks_gives_the_full_root():
     """All ranks' node lists concatenated in rank order reduce to the root of the whole tree."""
     ops = OracleTreeOps()
