@@ -126,6 +126,33 @@ int iv_merkle_levels(iv_ctx *ctx, const uint8_t *d_nodes, uint64_t n, uint32_t l
                      uint8_t *d_out, uint64_t out_cap, uint64_t *h_n_out, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
+ * Incremental re-verification -- the paper's hierarchical / differential
+ * verification ("incremental verification for model updates": when fine-tuning
+ * or an update touches some chunks, only those leaves and their paths to the
+ * root are recomputed).
+ *
+ * A retained tree holds every level of the tree over n leaves in one device
+ * array of iv_tree_records(n) records of 32 bytes: the n leaves first, then
+ * ceil(n/2) parents, and so on; the LAST record is the root (for n == 0 the
+ * single record is SHA-256 of the empty string).  d_tree must be 16-byte aligned.
+ *
+ * iv_tree_build   fills the array from n leaf digests (d_leaves 16-byte aligned).
+ * iv_tree_update  re-hashes the chunks listed in d_dirty (n_dirty uint64 chunk
+ *                 indices in DEVICE memory, any order, repeats allowed, each
+ *                 < ceil(nbytes / chunk_bytes)) from the current bytes of d_data,
+ *                 stores their digests in the leaf level and recomputes only the
+ *                 ancestors of those leaves.  Work is n_dirty chunk hashes plus
+ *                 n_dirty * ceil(log2 n) node hashes.  An index outside the tree
+ *                 is skipped and sets the device status to 2 (iv_device_status).
+ */
+uint64_t iv_tree_records(uint64_t n_leaves);
+int iv_tree_build(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_tree,
+                  uint64_t tree_cap, void *cuda_stream);
+int iv_tree_update(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                   const uint64_t *d_dirty, uint64_t n_dirty, uint8_t *d_tree, uint64_t tree_cap,
+                   void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * Verification -- Algorithm 1, "Compare root hash with expected value", plus
  * the per-chunk comparison that locates the damage.
  *

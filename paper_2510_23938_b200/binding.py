@@ -29,6 +29,7 @@ EXPORTS = (
     "iv_hash_chunks", "iv_merkle_root", "iv_verify_manifest", "iv_ctx_digests",
     "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
     "iv_merkle_root_noalloc", "iv_last_leaf_kernel", "iv_merkle_levels",
+    "iv_tree_records", "iv_tree_build", "iv_tree_update",
 )
 
 
@@ -83,6 +84,12 @@ def load_library() -> ctypes.CDLL:
     lib.iv_merkle_root.restype = i32
     lib.iv_merkle_levels.argtypes = [vp, vp, u64, ctypes.c_uint32, vp, u64, ctypes.POINTER(u64), vp]
     lib.iv_merkle_levels.restype = i32
+    lib.iv_tree_records.argtypes = [u64]
+    lib.iv_tree_records.restype = u64
+    lib.iv_tree_build.argtypes = [vp, vp, u64, vp, u64, vp]
+    lib.iv_tree_build.restype = i32
+    lib.iv_tree_update.argtypes = [vp, vp, u64, u64, vp, u64, vp, u64, vp]
+    lib.iv_tree_update.restype = i32
     lib.iv_verify_manifest.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest.restype = i32
     lib.iv_ctx_digests.argtypes = [vp]
@@ -215,6 +222,23 @@ class Context:
         self._check(rc, "iv_merkle_levels")
         assert got.value == n_out
         return out
+
+    def tree_build(self, leaves: torch.Tensor, stream=None) -> torch.Tensor:
+        """iv_tree_build: the retained tree (iv_tree_records(n), 32) of the (n, 32) leaf digests; root = tree[-1]."""
+        n = leaves.numel() // 32
+        records = int(self._lib.iv_tree_records(n))
+        tree = torch.empty((records, 32), dtype=torch.uint8, device=leaves.device)
+        rc = self._lib.iv_tree_build(self._h, _dev_ptr(leaves), n, _dev_ptr(tree), records, _stream_ptr(stream))
+        self._check(rc, "iv_tree_build")
+        return tree
+
+    def tree_update(self, data: torch.Tensor, chunk_bytes: int, dirty: torch.Tensor, tree: torch.Tensor,
+                    stream=None) -> None:
+        """iv_tree_update: re-hash the chunks whose indices are in the int64 device tensor `dirty`."""
+        assert dirty.dtype == torch.int64
+        rc = self._lib.iv_tree_update(self._h, _dev_ptr(data), _nbytes(data), chunk_bytes, _dev_ptr(dirty),
+                                      dirty.numel(), _dev_ptr(tree), tree.numel() // 32, _stream_ptr(stream))
+        self._check(rc, "iv_tree_update")
 
     def make_manifest(self, total_bytes: int, chunk_bytes: int, digests: torch.Tensor, root: bytes) -> Manifest:
         m = Manifest()

@@ -29,6 +29,8 @@ struct iv_ctx {
     uint64_t digests_valid = 0;
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
+    uint8_t *d_dirty_scratch = nullptr;       // offsets, lengths and fresh digests of iv_tree_update
+    uint64_t dirty_cap = 0;                   // bytes
     uint32_t *d_order = nullptr;              // tensor order (by descending length) of iv_hash_ragged
     uint64_t order_cap = 0;
     uint8_t *d_slices = nullptr;              // FIFO, slice counters and parked chaining values of the sliced leaf kernel
@@ -242,6 +244,7 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_words);
     cudaFree(ctx->d_slices);
     cudaFree(ctx->d_order);
+    cudaFree(ctx->d_dirty_scratch);
     cudaFree(ctx->d_window[0]);
     cudaFree(ctx->d_window[1]);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -334,6 +337,49 @@ int iv_merkle_levels(iv_ctx *ctx, const uint8_t *d_nodes, uint64_t n, uint32_t l
         left -= step;
         if (last) break;
     }
+    return IV_OK;
+}
+
+uint64_t iv_tree_records(uint64_t n_leaves) { return ivk::tree_records(n_leaves); }
+
+int iv_tree_build(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_tree, uint64_t tree_cap,
+                  void *cuda_stream) {
+    if (!ctx || !d_tree || (n_leaves && !d_leaves)) return IV_ERR_INVALID_ARG;
+    if (tree_cap < ivk::tree_records(n_leaves)) return IV_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_tree) | reinterpret_cast<uintptr_t>(d_leaves)) & 15u) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    IV_TRY(ctx, ivk::launch_tree_build(d_leaves, n_leaves, d_tree, static_cast<cudaStream_t>(cuda_stream),
+                                       &ctx->launches));
+    return IV_OK;
+}
+
+int iv_tree_update(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, const uint64_t *d_dirty,
+                   uint64_t n_dirty, uint8_t *d_tree, uint64_t tree_cap, void *cuda_stream) {
+    if (!ctx || chunk_bytes == 0 || !d_tree) return IV_ERR_INVALID_ARG;
+    const uint64_t n = chunk_count(nbytes, chunk_bytes);
+    if (tree_cap < ivk::tree_records(n)) return IV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(d_tree) & 15u) return IV_ERR_INVALID_ARG;
+    if (n_dirty == 0) return IV_OK;
+    if (!d_dirty || !d_data || n == 0) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // scratch: offsets[n_dirty] | lengths[n_dirty] | fresh digests[n_dirty * 32]
+    int rc = grow(ctx, &ctx->d_dirty_scratch, &ctx->dirty_cap, 48 * n_dirty + 64, 1);
+    if (rc != IV_OK) return rc;
+    uint64_t *d_off = reinterpret_cast<uint64_t *>(ctx->d_dirty_scratch);
+    uint64_t *d_len = d_off + n_dirty;
+    uint8_t *d_fresh = reinterpret_cast<uint8_t *>(d_len + n_dirty);
+    if (n_dirty <= ivk::kRaggedSortMax) {
+        rc = grow(ctx, &ctx->d_order, &ctx->order_cap, n_dirty, sizeof(uint32_t));
+        if (rc != IV_OK) return rc;
+    }
+    IV_TRY(ctx, ivk::launch_dirty_ranges(d_dirty, n_dirty, nbytes, chunk_bytes, n, d_off, d_len, ctx->d_status, stream,
+                                         &ctx->launches));
+    IV_TRY(ctx, ivk::launch_hash_ragged(static_cast<const uint8_t *>(d_data), d_off, d_len, n_dirty, d_fresh,
+                                        ctx->d_queue, n_dirty <= ivk::kRaggedSortMax ? ctx->d_order : nullptr,
+                                        ctx->d_status, ctx->d_one, ctx->sm_count, stream, &ctx->launches,
+                                        &ctx->leaf_kernel));
+    IV_TRY(ctx, ivk::launch_tree_update(d_tree, n, d_fresh, d_dirty, n_dirty, stream, &ctx->launches));
     return IV_OK;
 }
 

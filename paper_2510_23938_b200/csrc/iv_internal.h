@@ -68,6 +68,19 @@ cudaError_t launch_merkle_root(const uint8_t *d_leaves, uint64_t n, uint8_t *d_r
 cudaError_t launch_merkle_levels(const uint8_t *d_in, uint64_t n, uint32_t levels, uint8_t *d_out,
                                  cudaStream_t stream, uint64_t *launches);
 
+// Retained tree (all levels in one array, leaves first, the root last).
+constexpr int kTreeMaxLevels = 40;
+uint64_t tree_records(uint64_t n_leaves);
+cudaError_t launch_tree_build(const uint8_t *d_leaves, uint64_t n, uint8_t *d_tree, cudaStream_t stream,
+                              uint64_t *launches);
+cudaError_t launch_dirty_ranges(const uint64_t *d_dirty, uint64_t n_dirty, uint64_t nbytes, uint64_t chunk_bytes,
+                                uint64_t n_leaves, uint64_t *d_offsets, uint64_t *d_lengths, uint32_t *d_status,
+                                cudaStream_t stream, uint64_t *launches);
+// d_fresh: the new digests of the dirty leaves in dirty-list order.  Writes them into the leaf
+// level and recomputes every ancestor of a dirty leaf.
+cudaError_t launch_tree_update(uint8_t *d_tree, uint64_t n_leaves, const uint8_t *d_fresh, const uint64_t *d_dirty,
+                               uint64_t n_dirty, cudaStream_t stream, uint64_t *launches);
+
 // Compare n computed digests with the manifest's, compact the mismatching
 // indices in ascending order, compare the root.  d_words holds ceil(n/32)
 // uint32 mask words; d_ticket one zeroed uint32.

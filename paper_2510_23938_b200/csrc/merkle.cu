@@ -144,6 +144,98 @@ merkle_levels_kernel(const uint8_t *__restrict__ nodes_in, uint64_t n, uint32_t 
     }
 }
 
+// ---------------------------------------------------------------------------
+// Incremental re-verification on a retained tree (all levels kept in one array,
+// leaves first).  After some leaves changed, only their ancestors are recomputed:
+// one thread per changed leaf walks up one level per step; two changed siblings
+// compute the same parent twice and store the same bytes.
+// ---------------------------------------------------------------------------
+
+struct TreeShape {
+    uint64_t level_off[kTreeMaxLevels + 1];   // first record of each level
+    uint64_t level_n[kTreeMaxLevels + 1];     // nodes of each level
+    uint32_t levels;                          // number of parent levels (the root is level `levels`)
+};
+
+__device__ __forceinline__ void load_digest_words(const uint8_t *p, uint32_t (&w)[8]) {
+    const uint4 lo = __ldcg(reinterpret_cast<const uint4 *>(p));
+    const uint4 hi = __ldcg(reinterpret_cast<const uint4 *>(p) + 1);
+    w[0] = bswap32(lo.x); w[1] = bswap32(lo.y); w[2] = bswap32(lo.z); w[3] = bswap32(lo.w);
+    w[4] = bswap32(hi.x); w[5] = bswap32(hi.y); w[6] = bswap32(hi.z); w[7] = bswap32(hi.w);
+}
+
+// Recomputes the parent (at level l+1) of node `child` of level l; tree is 16-byte aligned.
+__device__ void tree_update_parent(uint8_t *tree, const TreeShape &shape, uint32_t l, uint64_t child) {
+    const uint64_t parent = child >> 1, left = parent << 1, right = left + 1;
+    const uint8_t *lp = tree + 32 * (shape.level_off[l] + left);
+    uint8_t *dst = tree + 32 * (shape.level_off[l + 1] + parent);
+    uint32_t st[8], w[16];
+    if (right < shape.level_n[l]) {
+        uint32_t a[8], b[8];
+        load_digest_words(lp, a);
+        load_digest_words(lp + 32, b);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { w[k] = a[k]; w[8 + k] = b[k]; }
+        sha256_init(st);
+        sha256_compress(st, w);
+        sha256_pad_only_block(w, 64);
+        sha256_compress(st, w);
+    } else {
+        load_digest_words(lp, st);               // unpaired last node moves up unchanged
+    }
+    store_digest_aligned(dst, st);
+}
+
+// All levels in one CTA (n_dirty <= blockDim.x): a block barrier separates the levels.
+__global__ void __launch_bounds__(1024)
+tree_update_small_kernel(uint8_t *__restrict__ tree, TreeShape shape, const uint64_t *__restrict__ dirty,
+                         uint32_t n_dirty) {
+    bool active = threadIdx.x < n_dirty;
+    uint64_t node = active ? dirty[threadIdx.x] : 0;
+    if (node >= shape.level_n[0]) active = false;      // an index outside the tree is skipped (status set earlier)
+    for (uint32_t l = 0; l < shape.levels; ++l) {
+        if (active) tree_update_parent(tree, shape, l, node);
+        node >>= 1;
+        __threadfence_block();
+        __syncthreads();
+    }
+}
+
+// One level per launch for long dirty lists.
+__global__ void __launch_bounds__(256)
+tree_update_level_kernel(uint8_t *__restrict__ tree, TreeShape shape, uint32_t l, const uint64_t *__restrict__ dirty,
+                         uint64_t n_dirty) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < n_dirty && dirty[t] < shape.level_n[0]) tree_update_parent(tree, shape, l, dirty[t] >> l);
+}
+
+// offsets / lengths of the dirty chunks for the per-tensor hashing kernels
+__global__ void dirty_ranges_kernel(const uint64_t *__restrict__ dirty, uint64_t n_dirty, uint64_t nbytes,
+                                    uint64_t chunk_bytes, uint64_t n_leaves, uint64_t *__restrict__ offsets,
+                                    uint64_t *__restrict__ lengths, uint32_t *__restrict__ status) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n_dirty) return;
+    const uint64_t idx = dirty[t];
+    if (idx >= n_leaves) {                      // not a chunk of this blob: hash nothing, record the fault
+        offsets[t] = 0;
+        lengths[t] = 0;
+        atomicExch(status, (uint32_t)IVK_DEV_BOUNDS);
+        return;
+    }
+    const uint64_t begin = idx * chunk_bytes;
+    offsets[t] = begin;
+    lengths[t] = (nbytes - begin < chunk_bytes) ? (nbytes - begin) : chunk_bytes;
+}
+
+// new leaf digests (in dirty-list order) into the leaf level of the tree
+__global__ void scatter_leaves_kernel(const uint8_t *__restrict__ fresh, const uint64_t *__restrict__ dirty,
+                                      uint64_t n_dirty, uint64_t n_leaves, uint8_t *__restrict__ tree) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;   // one thread per 16 bytes
+    if (t >= 2 * n_dirty || dirty[t >> 1] >= n_leaves) return;
+    const uint4 v = reinterpret_cast<const uint4 *>(fresh)[t];
+    reinterpret_cast<uint4 *>(tree + 32 * dirty[t >> 1])[t & 1] = v;
+}
+
 // Root of zero leaves: SHA-256 of the empty string, computed here rather than typed in.
 __global__ void empty_root_kernel(uint8_t *d_root) {
     uint32_t st[8], w[16];
@@ -281,6 +373,82 @@ cudaError_t launch_merkle_levels(const uint8_t *d_in, uint64_t n, uint32_t level
     merkle_levels_kernel<<<(unsigned)(blocks < 4096 ? blocks : 4096), kThreads, 0, stream>>>(d_in, n, levels, d_out);
     if (launches) ++*launches;
     return cudaGetLastError();
+}
+
+namespace {
+TreeShape make_shape(uint64_t n_leaves) {
+    TreeShape sh{};
+    uint64_t n = n_leaves, off = 0;
+    uint32_t l = 0;
+    sh.level_off[0] = 0;
+    sh.level_n[0] = n;
+    while (n > 1 && l < (uint32_t)kTreeMaxLevels) {
+        off += n;
+        n = (n + 1) / 2;
+        ++l;
+        sh.level_off[l] = off;
+        sh.level_n[l] = n;
+    }
+    sh.levels = l;
+    return sh;
+}
+}  // namespace
+
+uint64_t tree_records(uint64_t n_leaves) {
+    if (n_leaves == 0) return 1;
+    const TreeShape sh = make_shape(n_leaves);
+    return sh.level_off[sh.levels] + 1;
+}
+
+cudaError_t launch_tree_build(const uint8_t *d_leaves, uint64_t n, uint8_t *d_tree, cudaStream_t stream,
+                              uint64_t *launches) {
+    if (n == 0) {
+        empty_root_kernel<<<1, 1, 0, stream>>>(d_tree);
+        if (launches) ++*launches;
+        return cudaGetLastError();
+    }
+    cudaError_t e = cudaMemcpyAsync(d_tree, d_leaves, 32 * n, cudaMemcpyDeviceToDevice, stream);
+    if (e != cudaSuccess) return e;
+    const TreeShape sh = make_shape(n);
+    for (uint32_t l = 0; l < sh.levels; ++l) {
+        e = launch_merkle_levels(d_tree + 32 * sh.level_off[l], sh.level_n[l], 1, d_tree + 32 * sh.level_off[l + 1],
+                                 stream, launches);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+cudaError_t launch_dirty_ranges(const uint64_t *d_dirty, uint64_t n_dirty, uint64_t nbytes, uint64_t chunk_bytes,
+                                uint64_t n_leaves, uint64_t *d_offsets, uint64_t *d_lengths, uint32_t *d_status,
+                                cudaStream_t stream, uint64_t *launches) {
+    dirty_ranges_kernel<<<(unsigned)((n_dirty + 255) / 256), 256, 0, stream>>>(d_dirty, n_dirty, nbytes, chunk_bytes,
+                                                                              n_leaves, d_offsets, d_lengths, d_status);
+    if (launches) ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tree_update(uint8_t *d_tree, uint64_t n_leaves, const uint8_t *d_fresh, const uint64_t *d_dirty,
+                               uint64_t n_dirty, cudaStream_t stream, uint64_t *launches) {
+    if (n_dirty == 0 || n_leaves == 0) return cudaSuccess;
+    scatter_leaves_kernel<<<(unsigned)((2 * n_dirty + 255) / 256), 256, 0, stream>>>(d_fresh, d_dirty, n_dirty, n_leaves,
+                                                                                     d_tree);
+    if (launches) ++*launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const TreeShape sh = make_shape(n_leaves);
+    if (sh.levels == 0) return cudaSuccess;
+    if (n_dirty <= 1024) {
+        tree_update_small_kernel<<<1, 1024, 0, stream>>>(d_tree, sh, d_dirty, (uint32_t)n_dirty);
+        if (launches) ++*launches;
+        return cudaGetLastError();
+    }
+    for (uint32_t l = 0; l < sh.levels; ++l) {
+        tree_update_level_kernel<<<(unsigned)((n_dirty + 255) / 256), 256, 0, stream>>>(d_tree, sh, l, d_dirty, n_dirty);
+        if (launches) ++*launches;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_manifest_digests,

@@ -160,6 +160,57 @@ def test_sharded_root_emulated_ranks_on_one_gpu(ctx):
     assert _root_bytes(root) == want
 
 
+def _oracle_tree(leaves: np.ndarray) -> np.ndarray:
+    """Every level of the tree, leaves first: level l, node j = oracle root of the aligned run of 2^l leaves."""
+    n = len(leaves)
+    if n == 0:
+        return np.frombuffer(oracle.merkle_root(b""), dtype=np.uint8).reshape(1, 32)
+    levels, count, run = [leaves], n, 1
+    while count > 1:
+        run *= 2
+        count = (count + 1) // 2
+        levels.append(np.stack([np.frombuffer(oracle.merkle_root(leaves[s:s + run]), dtype=np.uint8)
+                                for s in range(0, n, run)]))
+    return np.concatenate(levels)
+
+
+@pytest.mark.parametrize("n_chunks,chunk,last,n_dirty", [
+    (1, 4096, 4096, 1), (2, 4096, 100, 2), (5, 1024, 1024, 2), (77, 512, 33, 9), (1000, 4096, 4096, 1),
+    (1000, 4096, 17, 40), (2510, 4096, 4096, 300), (3000, 1024, 1024, 2000), (513, 2048, 2048, 513),
+])
+def test_tree_build_and_incremental_update_equal_a_full_oracle_rebuild(ctx, n_chunks, chunk, last, n_dirty):
+    nbytes = (n_chunks - 1) * chunk + last
+    data = inputs.uniform_bytes(nbytes, seed=n_chunks + n_dirty, device="cuda")
+    leaves = ctx.hash_chunks(data, chunk)
+    tree = ctx.tree_build(leaves)
+    host_leaves = oracle.hash_chunks(_host(data), chunk, nthreads=oracle.host_threads())
+    assert np.array_equal(_host(tree), _oracle_tree(host_leaves))
+    assert _host(tree[-1]).tobytes() == oracle.merkle_root(host_leaves)
+    # change some chunks (always including the last, possibly short, one), update, compare with a rebuild
+    rng = np.random.default_rng(n_chunks * 7 + n_dirty)
+    dirty = rng.choice(n_chunks, size=min(n_dirty, n_chunks), replace=False)
+    dirty[0] = n_chunks - 1
+    dirty = np.concatenate([dirty, dirty[:3]])                      # repeats are allowed
+    pos = torch.from_numpy(np.minimum(dirty * chunk + 3, nbytes - 1)).cuda()
+    data[pos] ^= 0x5A
+    ctx.tree_update(data, chunk, torch.from_numpy(dirty.astype(np.int64)).cuda(), tree)
+    new_leaves = oracle.hash_chunks(_host(data), chunk, nthreads=oracle.host_threads())
+    assert not np.array_equal(new_leaves, host_leaves)
+    assert np.array_equal(_host(tree), _oracle_tree(new_leaves))
+    assert ctx.device_status() == 0
+
+
+def test_tree_update_rejects_an_index_outside_the_tree_without_touching_it(ctx):
+    chunk, n = 1024, 50
+    data = inputs.uniform_bytes(chunk * n, seed=5, device="cuda")
+    tree = ctx.tree_build(ctx.hash_chunks(data, chunk))
+    before = tree.clone()
+    ctx.tree_update(data, chunk, torch.tensor([n + 5], dtype=torch.int64, device="cuda"), tree)
+    assert ctx.device_status() == 2
+    assert torch.equal(tree, before)
+    assert ctx.device_status() == 0          # reading the status clears it
+
+
 # ------------------------------------------------------------------------------------------ a4
 
 def _manifest_from_oracle(ctx, host_blob: np.ndarray, chunk: int):
