@@ -215,7 +215,8 @@ def run_ours(args):
             ctx.merkle_root(digests, out=root)
     else:
         n_units = binding.n_chunks(nbytes, chunk)
-        man_digests = ctx.hash_chunks(data, chunk)
+        two_level = args.two_level
+        man_digests = ctx.hash_chunks_two_level(data, chunk, two_level) if two_level else ctx.hash_chunks(data, chunk)
         man_root = bytes(ctx.merkle_root(man_digests).cpu().numpy().tobytes())
         manifest = ctx.make_manifest(nbytes, chunk, man_digests, man_root)
         result = binding.new_result(device)
@@ -233,7 +234,10 @@ def run_ours(args):
                 shard_plan = None                       # uneven cut: fall back to independent blobs
 
         def step():
-            ctx.verify_manifest(data, manifest, result, idx)
+            if two_level:
+                ctx.verify_manifest_two_level(data, manifest, two_level, result, idx)
+            else:
+                ctx.verify_manifest(data, manifest, result, idx)
             if shard_plan is not None:
                 sharded.sharded_root(ctx, ctx.last_digests(n_units), shard_plan, rank)
         if shard_plan is not None:
@@ -330,12 +334,17 @@ def run_ours(args):
     }
     if fallback:
         out["config"]["fallback"] = fallback
+    if not ragged and args.two_level:
+        out["config"]["leaf_definition"] = (f"TWO-LEVEL (not the default): chunk digest = Merkle root over SHA-256 of "
+                                            f"{args.two_level}-byte pieces; {binding.n_chunks(nbytes, args.two_level)} chains")
+        out["roofline"]["chains"] = binding.n_chunks(nbytes, args.two_level)
+        out["roofline"]["note"] = "launch_ms covers piece hashing + the levels up to chunk digests"
 
-    if rank == 0 and not ragged and not args.no_e2e:
+    if rank == 0 and not ragged and not args.no_e2e and not args.two_level:
         out["e2e"] = measure_e2e(ctx, wl, device, args)
     elif rank == 0:
         out["e2e"] = None
-    if rank == 0 and world == 1 and not args.no_cpu:
+    if rank == 0 and world == 1 and not args.no_cpu and not (not ragged and args.two_level):
         out["cpu_baseline"] = measure_cpu_baseline(ctx, wl, device, oracle, ragged,
                                                    None if ragged else man_digests,
                                                    (d_off, d_len, digests) if ragged else None)
@@ -509,6 +518,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--nbytes", type=int, default=None, help="override the blob size of configs 1 and 4 (profiling)")
     ap.add_argument("--chunk", type=int, default=None, help="override the chunk size (profiling)")
+    ap.add_argument("--two-level", type=int, default=None, metavar="SUB_BYTES",
+                    help="two-level leaves: chunk digest = Merkle root over SHA-256 of SUB_BYTES pieces (a different, "
+                         "separately named leaf definition; not the default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()

@@ -191,6 +191,29 @@ int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
 const uint8_t *iv_ctx_digests(const iv_ctx *ctx);
 
 /* ---------------------------------------------------------------------------
+ * Two-level leaves -- a SEPARATELY NAMED mode whose digests differ from
+ * iv_hash_chunks (the paper speaks of verification "at multiple levels of
+ * granularity").  The digest of chunk i is the Merkle root (this library's tree
+ * rule) over the SHA-256 digests of its sub_bytes-sized pieces:
+ *     D_i = root( SHA-256(piece_0), SHA-256(piece_1), ... )   pieces of chunk i.
+ * A chunk is then no longer one serial SHA-256 chain but chunk_bytes/sub_bytes
+ * independent ones, which is what fills a GPU when a blob has few large chunks.
+ * chunk_bytes must be sub_bytes times a power of two (else IV_ERR_INVALID_ARG);
+ * with that, the root over the D_i equals the root over all pieces' digests, so
+ * a manifest at chunk granularity and one at piece granularity share one root.
+ * sub_bytes == chunk_bytes gives iv_hash_chunks / iv_verify_manifest exactly.
+ * Other arguments as for iv_hash_chunks / iv_verify_manifest; the manifest's
+ * digests and root must have been made in the same mode.
+ */
+int iv_hash_chunks_two_level(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                             uint64_t sub_bytes, uint8_t *d_digests, uint64_t digests_cap,
+                             uint64_t *h_n_chunks, void *cuda_stream);
+int iv_verify_manifest_two_level(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
+                                 const iv_manifest *h_manifest, uint64_t sub_bytes,
+                                 iv_verify_result *d_result, uint64_t *d_mismatch_idx,
+                                 uint64_t idx_cap, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * Streamed verification -- the whole of Algorithm 1 for a blob that lives in
  * HOST memory ("Load model chunk M_i into GPU memory ... Free GPU memory"):
  * the blob is copied window by window into two device windows owned by the

@@ -30,6 +30,7 @@ EXPORTS = (
     "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
     "iv_merkle_root_noalloc", "iv_last_leaf_kernel", "iv_merkle_levels",
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
+    "iv_hash_chunks_two_level", "iv_verify_manifest_two_level",
 )
 
 
@@ -90,6 +91,10 @@ def load_library() -> ctypes.CDLL:
     lib.iv_tree_build.restype = i32
     lib.iv_tree_update.argtypes = [vp, vp, u64, u64, vp, u64, vp, u64, vp]
     lib.iv_tree_update.restype = i32
+    lib.iv_hash_chunks_two_level.argtypes = [vp, vp, u64, u64, u64, vp, u64, ctypes.POINTER(u64), vp]
+    lib.iv_hash_chunks_two_level.restype = i32
+    lib.iv_verify_manifest_two_level.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), u64, vp, vp, u64, vp]
+    lib.iv_verify_manifest_two_level.restype = i32
     lib.iv_verify_manifest.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest.restype = i32
     lib.iv_ctx_digests.argtypes = [vp]
@@ -197,6 +202,26 @@ class Context:
                                       out.numel() // 32, ctypes.byref(got), _stream_ptr(stream))
         self._check(rc, "iv_hash_chunks")
         return out[:got.value]
+
+    def hash_chunks_two_level(self, data: torch.Tensor, chunk_bytes: int, sub_bytes: int, stream=None) -> torch.Tensor:
+        """iv_hash_chunks_two_level: digest i = Merkle root over the SHA-256 digests of chunk i's sub_bytes pieces."""
+        nb = _nbytes(data)
+        n = n_chunks(nb, chunk_bytes) if chunk_bytes > 0 else 0
+        out = torch.empty((n, 32), dtype=torch.uint8, device=data.device)
+        got = ctypes.c_uint64(0)
+        rc = self._lib.iv_hash_chunks_two_level(self._h, _dev_ptr(data), nb, chunk_bytes, sub_bytes, _dev_ptr(out), n,
+                                                ctypes.byref(got), _stream_ptr(stream))
+        self._check(rc, "iv_hash_chunks_two_level")
+        return out[:got.value]
+
+    def verify_manifest_two_level(self, data: torch.Tensor, manifest: Manifest, sub_bytes: int, result: torch.Tensor,
+                                  mismatch_idx: torch.Tensor | None, stream=None) -> None:
+        """iv_verify_manifest_two_level (asynchronous); the manifest must hold two-level digests."""
+        cap = 0 if mismatch_idx is None else mismatch_idx.numel()
+        rc = self._lib.iv_verify_manifest_two_level(self._h, _dev_ptr(data), _nbytes(data), ctypes.byref(manifest),
+                                                    sub_bytes, _dev_ptr(result), _dev_ptr(mismatch_idx), cap,
+                                                    _stream_ptr(stream))
+        self._check(rc, "iv_verify_manifest_two_level")
 
     def merkle_root(self, leaves: torch.Tensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
         """iv_merkle_root: 32-byte root (uint8 tensor on the device) of (n, 32) leaf digests."""

@@ -29,6 +29,8 @@ struct iv_ctx {
     uint64_t digests_valid = 0;
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
+    uint8_t *d_sub = nullptr;                 // sub-leaf digests of the two-level mode
+    uint64_t sub_cap = 0;                     // in digests
     uint8_t *d_dirty_scratch = nullptr;       // offsets, lengths and fresh digests of iv_tree_update
     uint64_t dirty_cap = 0;                   // bytes
     uint32_t *d_order = nullptr;              // tensor order (by descending length) of iv_hash_ragged
@@ -245,6 +247,7 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_slices);
     cudaFree(ctx->d_order);
     cudaFree(ctx->d_dirty_scratch);
+    cudaFree(ctx->d_sub);
     cudaFree(ctx->d_window[0]);
     cudaFree(ctx->d_window[1]);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -340,7 +343,73 @@ int iv_merkle_levels(iv_ctx *ctx, const uint8_t *d_nodes, uint64_t n, uint32_t l
     return IV_OK;
 }
 
+namespace {
+
+// log2(chunk_bytes / sub_bytes) when the ratio is a power of two, -1 otherwise.
+int two_level_shift(uint64_t chunk_bytes, uint64_t sub_bytes) {
+    if (sub_bytes == 0 || chunk_bytes < sub_bytes || chunk_bytes % sub_bytes) return -1;
+    uint64_t ratio = chunk_bytes / sub_bytes;
+    int k = 0;
+    while ((ratio & 1u) == 0) { ratio >>= 1; ++k; }
+    return ratio == 1 ? k : -1;
+}
+
+// Two-level leaf digests into d_out (n = ceil(nbytes / chunk_bytes) records).
+int hash_leaves_two_level(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t sub_bytes,
+                          uint8_t *d_out, uint64_t n, cudaStream_t stream) {
+    const int k = two_level_shift(chunk_bytes, sub_bytes);
+    if (k < 0) return IV_ERR_INVALID_ARG;
+    if (k == 0) return hash_leaves(ctx, d_data, nbytes, chunk_bytes, n, d_out, stream);
+    const uint64_t n_sub = chunk_count(nbytes, sub_bytes);
+    int rc = grow(ctx, &ctx->d_sub, &ctx->sub_cap, n_sub + 1, 32);
+    if (rc != IV_OK) return rc;
+    rc = hash_leaves(ctx, d_data, nbytes, sub_bytes, n_sub, ctx->d_sub, stream);
+    if (rc != IV_OK) return rc;
+    // the sub-leaves of chunk i are the aligned run [i * 2^k, (i+1) * 2^k): k levels up they are one node
+    return iv_merkle_levels(ctx, ctx->d_sub, n_sub, (uint32_t)k, d_out, n, nullptr, stream);
+}
+
+}  // namespace
+
 uint64_t iv_tree_records(uint64_t n_leaves) { return ivk::tree_records(n_leaves); }
+
+int iv_hash_chunks_two_level(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t sub_bytes,
+                             uint8_t *d_digests, uint64_t digests_cap, uint64_t *h_n_chunks, void *cuda_stream) {
+    if (!ctx || chunk_bytes == 0 || two_level_shift(chunk_bytes, sub_bytes) < 0) return IV_ERR_INVALID_ARG;
+    const uint64_t n = chunk_count(nbytes, chunk_bytes);
+    if (n > digests_cap) return IV_ERR_INVALID_ARG;
+    if (n && (!d_data || !d_digests)) return IV_ERR_INVALID_ARG;
+    if (h_n_chunks) *h_n_chunks = n;
+    if (n == 0) return IV_OK;
+    DeviceGuard guard(ctx->device);
+    return hash_leaves_two_level(ctx, static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, sub_bytes, d_digests, n,
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
+int iv_verify_manifest_two_level(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest *h_manifest,
+                                 uint64_t sub_bytes, iv_verify_result *d_result, uint64_t *d_mismatch_idx,
+                                 uint64_t idx_cap, void *cuda_stream) {
+    if (!ctx || !d_result || (idx_cap && !d_mismatch_idx)) return IV_ERR_INVALID_ARG;
+    int rc = check_manifest(h_manifest, nbytes);
+    if (rc != IV_OK) return rc;
+    if (two_level_shift(h_manifest->chunk_bytes, sub_bytes) < 0) return IV_ERR_INVALID_ARG;
+    if (nbytes && !d_data) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint64_t n = h_manifest->n_chunks;
+    rc = grow(ctx, &ctx->d_digests, &ctx->digests_cap, n + 1, 32);
+    if (rc != IV_OK) return rc;
+    // grow everything the phases need before the first phase event, so that no allocation sits between events
+    rc = grow(ctx, &ctx->d_sub, &ctx->sub_cap, chunk_count(nbytes, sub_bytes) + 1, 32);
+    if (rc != IV_OK) return rc;
+    if ((rc = mark_phase(ctx, 0, stream)) != IV_OK) return rc;
+    if (n) {
+        rc = hash_leaves_two_level(ctx, static_cast<const uint8_t *>(d_data), nbytes, h_manifest->chunk_bytes, sub_bytes,
+                                   ctx->d_digests, n, stream);
+        if (rc != IV_OK) return rc;
+    }
+    return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream);
+}
 
 int iv_tree_build(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_tree, uint64_t tree_cap,
                   void *cuda_stream) {

@@ -298,6 +298,53 @@ def test_verify_empty_blob(ctx):
     assert r["root_ok"] and r["n_mismatch"] == 0 and r["root"] == root
 
 
+# ------------------------------------------------------------------------------------------ two-level leaves
+
+def _oracle_two_level(host: np.ndarray, chunk: int, sub: int) -> np.ndarray:
+    """D_i = oracle root over the oracle digests of chunk i's pieces (the mode's definition, composed on the CPU)."""
+    out = []
+    for o in range(0, host.size, chunk):
+        pieces = oracle.hash_chunks(host[o:o + chunk], sub)
+        out.append(np.frombuffer(oracle.merkle_root(pieces), dtype=np.uint8))
+    return np.stack(out) if out else np.zeros((0, 32), dtype=np.uint8)
+
+
+@pytest.mark.parametrize("nbytes,chunk,sub", [
+    (64 << 20, 4 << 20, 64 << 10),            # 16 chunks of 64 pieces: 1024 independent chains instead of 16
+    ((8 << 20) + 12345, 1 << 20, 1 << 16),    # short last chunk whose last piece is short too
+    (300_000, 4096, 1024), (300_000, 4096, 4096), (100, 4096, 512), (5 * 8192 + 1, 8192, 8192 // 4),
+])
+def test_two_level_leaves_equal_their_definition_and_share_the_root_with_piece_granularity(ctx, nbytes, chunk, sub):
+    data = inputs.uniform_bytes(nbytes, seed=71, device="cuda")
+    host = _host(data)
+    got = ctx.hash_chunks_two_level(data, chunk, sub)
+    want = _oracle_two_level(host, chunk, sub)
+    assert np.array_equal(_host(got), want)
+    # one root for both granularities
+    root = _root_bytes(ctx.merkle_root(got))
+    assert root == oracle.merkle_root(oracle.hash_chunks(host, sub, nthreads=oracle.host_threads()))
+    # verification in this mode finds a flipped bit at its chunk
+    manifest = ctx.make_manifest(nbytes, chunk, torch.from_numpy(want).cuda(), oracle.merkle_root(want))
+    res = binding.new_result("cuda")
+    idx = torch.zeros(4, dtype=torch.int64, device="cuda")
+    ctx.verify_manifest_two_level(data, manifest, sub, res, idx)
+    r = binding.read_result(res)
+    assert r["root_ok"] and r["n_mismatch"] == 0 and r["root"] == root
+    bad = data.clone()
+    bad[nbytes - 1] ^= 1
+    ctx.verify_manifest_two_level(bad, manifest, sub, res, idx)
+    r = binding.read_result(res)
+    assert (not r["root_ok"]) and r["n_mismatch"] == 1 and int(idx[0]) == (nbytes - 1) // chunk
+
+
+def test_two_level_requires_a_power_of_two_ratio(ctx):
+    data = inputs.uniform_bytes(1 << 16, seed=1, device="cuda")
+    for chunk, sub in ((4096, 3000), (4096, 0), (4096, 8192), (12288, 4096)):
+        with pytest.raises(binding.IvError) as e:
+            ctx.hash_chunks_two_level(data, chunk, sub)
+        assert e.value.code == binding.IV_ERR_INVALID_ARG
+
+
 # ------------------------------------------------------------------------------------------ a5
 
 @pytest.mark.parametrize("pinned", [True, False])
