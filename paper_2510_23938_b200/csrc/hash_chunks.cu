@@ -267,8 +267,16 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
         if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
             if (launches) ++*launches;
             *kernel_used = "hash_chunks_sliced_kernel";
-            return launch_hash_chunks_sliced(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
-                                             d_slice_scratch, d_one, sm_count, stream);
+            uint64_t covered = 0;
+            cudaError_t e = launch_hash_chunks_sliced(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
+                                                      d_slice_scratch, d_one, sm_count, stream, &covered);
+            if (e != cudaSuccess || covered == n_chunks) return e;
+            // a short last chunk, left out by the tiled copies: one chain through the direct kernel
+            if (launches) ++*launches;
+            const uint64_t off = covered * chunk_bytes;
+            hash_chunks_kernel<true><<<1, 32, 0, stream>>>(d_data + off, nbytes - off, chunk_bytes, 1,
+                                                          d_digests + 32 * covered);
+            return cudaGetLastError();
         }
         // Many small chunks: two CTAs of four warps per SM keep two warps on every scheduler.
         return launch_staged<256, 3, 4, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);

@@ -10,9 +10,18 @@
 // the FIFO at most once, its slices run in order; a warp never waits while it holds a task, so
 // the scheme needs no co-residency and cannot deadlock.  All waits are bounded.
 //
-// Data movement is the staged kernel's: per-lane bulk copies (TMA) into a lane-interleaved
-// shared-memory ring, mbarrier completion, the next block fetched into registers before the
-// current block's rounds.
+// Data movement, TILED = false: the staged kernel's per-lane bulk copies (TMA, 1-D) into a
+// lane-interleaved shared-memory ring.  TILED = true: the blob is described to the TMA unit as a
+// 2-D tensor [chunk][byte] with the chunk size as row pitch, and ONE tiled copy of a 32-row x
+// 128-byte box brings the next two blocks of all 32 chains (instead of 32 copies issued one
+// lane after the other).  The box lands row-major, one 128-byte row per lane, with the 128-byte
+// swizzle (16-byte piece c of row r sits at piece c ^ (r mod 8)), so the lanes' 128-bit loads of
+// the same piece hit eight different bank groups.  Either way completion is counted by one
+// mbarrier per stage and the next block is in registers before the current block's rounds.
+#include <cuda.h>          // CUtensorMap (types only; the encoder is fetched through the runtime)
+
+#include <cstring>
+
 #include "iv_internal.h"
 #include "sha256_dev.cuh"
 #include "tma_dev.cuh"
@@ -45,9 +54,15 @@ __device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-template <int SEG, int STAGES, int MAX_WARPS>
+__device__ __forceinline__ void tiled_g2s(uint32_t dst, const CUtensorMap *map, uint32_t x, uint32_t y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+template <int SEG, int STAGES, int MAX_WARPS, bool TILED>
 __global__ void __launch_bounds__(32 * MAX_WARPS)
-hash_chunks_sliced_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
+hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
                           uint64_t slice_bytes, uint64_t total_tasks, uint32_t *__restrict__ slot,
                           SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice,
@@ -56,14 +71,19 @@ hash_chunks_sliced_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uin
     // pipe (placement 2) gains 4.5 % in the register-only probe but lost 5 % in this kernel.
     constexpr int ADD = 0;
     const uint32_t one = __ldg(one_ptr);
-    constexpr uint32_t kLaneStride = SEG + 16;
-    constexpr uint32_t kStageBytes = 32 * kLaneStride;
+    static_assert(!TILED || SEG == 256, "a tiled stage is two boxes of 32 rows x 128 bytes");
+    constexpr uint32_t kLaneStride = TILED ? 128 : SEG + 16;
+    constexpr uint32_t kStageBytes = TILED ? 8192 : 32 * kLaneStride;
     constexpr int kBlocksPerSeg = SEG / 64;
     extern __shared__ __align__(128) uint8_t ring[];
     __shared__ __align__(8) uint64_t bars[MAX_WARPS][STAGES];
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
-    const uint32_t ring_base = tma::smem_u32(ring) + warp * (STAGES * kStageBytes) + lane * kLaneStride;
+    // tiled boxes must start on a 1024-byte boundary (the swizzle pattern repeats every 8 rows)
+    const uint32_t ring0 = TILED ? ((tma::smem_u32(ring) + 1023u) & ~1023u) : tma::smem_u32(ring);
+    const uint32_t ring_warp = ring0 + warp * (STAGES * kStageBytes);
+    const uint32_t ring_base = ring_warp + lane * kLaneStride;
+    const uint32_t swz = (lane & 7u) * 16u;
     const uint32_t bar_base = tma::smem_u32(&bars[warp][0]);
     if (lane == 0) {
 #pragma unroll
@@ -136,16 +156,38 @@ hash_chunks_sliced_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uin
         auto issue = [&](uint64_t seg, int stg) {
             const uint64_t off = seg * SEG;
             const uint32_t bar = bar_base + 8 * stg;
-            const uint32_t bytes = off < my_bytes ? (uint32_t)((my_bytes - off < SEG) ? (my_bytes - off) : SEG) : 0u;
-            const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
-            if (lane == 0) tma::mbar_arrive_expect_tx(bar, total);
-            if (bytes) tma::bulk_g2s(ring_base + stg * kStageBytes, p + off, bytes, bar);
+            if (TILED) {
+                // one or two boxes of 32 chains x 128 bytes; a box always delivers its 4096 bytes
+                // (rows or bytes outside the tensor arrive as zeros and are never hashed)
+                if (lane == 0) {
+                    const uint32_t boxes = (warp_bytes - off > 128) ? 2u : 1u;
+                    tma::mbar_arrive_expect_tx(bar, boxes * 4096u);
+                    const uint32_t x = (uint32_t)(lo + off), y = (uint32_t)(g * 32);
+                    tiled_g2s(ring_warp + stg * kStageBytes, &tmap, x, y, bar);
+                    if (boxes == 2) tiled_g2s(ring_warp + stg * kStageBytes + 4096u, &tmap, x + 128u, y, bar);
+                }
+            } else {
+                const uint32_t bytes = off < my_bytes ? (uint32_t)((my_bytes - off < SEG) ? (my_bytes - off) : SEG) : 0u;
+                const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+                if (lane == 0) tma::mbar_arrive_expect_tx(bar, total);
+                if (bytes) tma::bulk_g2s(ring_base + stg * kStageBytes, p + off, bytes, bar);
+            }
         };
         auto fetch = [&](int stg, int blk_in_stage) {
-            const uint32_t src = ring_base + stg * kStageBytes + 64 * blk_in_stage;
+            if (TILED) {
+                // block b of the stage: box b / 2, 16-byte pieces 4 (b mod 2) .. +3 of this lane's row
+                const uint32_t row = ring_base + stg * kStageBytes + (uint32_t)(blk_in_stage >> 1) * 4096u;
+                const uint32_t c0 = (uint32_t)(blk_in_stage & 1) * 64u;
 #pragma unroll
-            for (int qd = 0; qd < 4; ++qd)
-                tma::ld_shared_v4(src + 16 * qd, raw[4 * qd], raw[4 * qd + 1], raw[4 * qd + 2], raw[4 * qd + 3]);
+                for (int qd = 0; qd < 4; ++qd)
+                    tma::ld_shared_v4(row + ((c0 + 16u * qd) ^ swz), raw[4 * qd], raw[4 * qd + 1], raw[4 * qd + 2],
+                                      raw[4 * qd + 3]);
+            } else {
+                const uint32_t src = ring_base + stg * kStageBytes + 64 * blk_in_stage;
+#pragma unroll
+                for (int qd = 0; qd < 4; ++qd)
+                    tma::ld_shared_v4(src + 16 * qd, raw[4 * qd], raw[4 * qd + 1], raw[4 * qd + 2], raw[4 * qd + 3]);
+            }
         };
 
         // prologue: request the first STAGES segments into the stages that follow the ring position
@@ -247,16 +289,51 @@ uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t 
     return 64 + 4 * total + 4 * groups + 1024 * groups + 256;
 }
 
-cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
-                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
-                                      const uint32_t *d_one, int sm_count, cudaStream_t stream) {
+namespace {
+
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link libcuda.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult st = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &st) != cudaSuccess ||
+            st != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        (void)cudaGetLastError();
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// The blob's whole chunks as a 2-D byte tensor [rows][chunk_bytes], box = 32 rows x 128 bytes, 128-byte swizzle.
+bool make_chunk_tensor_map(CUtensorMap *map, const uint8_t *d_data, uint64_t chunk_bytes, uint64_t rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || rows == 0 || chunk_bytes >= (1ull << 31) || rows >= (1ull << 31)) return false;
+    const cuuint64_t gdim[2] = {chunk_bytes, rows};
+    const cuuint64_t gstride[1] = {chunk_bytes};             // row pitch in bytes (a multiple of 16)
+    const cuuint32_t box[2] = {128, 32};
+    const cuuint32_t estride[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t *>(d_data), gdim, gstride, box, estride,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool TILED>
+cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                          uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
+                          const uint32_t *d_one, int sm_count, cudaStream_t stream) {
     constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8;
-    constexpr size_t smem_per_warp = (size_t)STAGES * 32 * (SEG + 16);
-    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS>;
+    constexpr size_t smem_per_warp = TILED ? (size_t)STAGES * 8192 : (size_t)STAGES * 32 * (SEG + 16);
+    constexpr size_t smem_pad = TILED ? 1024 : 0;
+    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED>;
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(MAX_WARPS * smem_per_warp));
+                                             (int)(MAX_WARPS * smem_per_warp + smem_pad));
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -275,9 +352,30 @@ cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, ui
     // 4 / 5 / 6 / 7 / 8 warps per SM give 687 / 694 / 673 / 703 / 712 GB/s, and two CTAs of four
     // warps only 574 GB/s; workers that find the FIFO empty sleep in their bounded wait.
     const uint64_t warps = MAX_WARPS;
-    kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp, stream>>>(
-        d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice, mid, d_one);
+    kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
+        map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
+        mid, d_one);
     return cudaGetLastError();
+}
+
+}  // namespace
+
+// Returns how many chunks (from the front of the blob) the launch covers: with the tiled copies only whole
+// chunks can be described to the TMA unit, so a short last chunk is left to the caller (*covered = n - 1).
+cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
+                                      const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *covered) {
+    const uint64_t whole = nbytes / chunk_bytes;          // n_chunks or n_chunks - 1
+    alignas(64) CUtensorMap map;
+    std::memset(&map, 0, sizeof map);
+    if (whole > 0 && make_chunk_tensor_map(&map, d_data, chunk_bytes, whole)) {
+        *covered = whole;
+        return launch_sliced<true>(map, d_data, whole * chunk_bytes, chunk_bytes, whole, d_digests, d_status, d_scratch,
+                                   d_one, sm_count, stream);
+    }
+    *covered = n_chunks;
+    return launch_sliced<false>(map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_scratch, d_one,
+                                sm_count, stream);
 }
 
 }  // namespace ivk

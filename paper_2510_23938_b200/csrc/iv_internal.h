@@ -35,9 +35,10 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
 // stays level.  d_scratch must hold sliced_scratch_bytes(...) bytes.
 uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t *slice_bytes_out,
                               uint64_t *total_tasks_out, uint64_t nbytes);
+// *covered receives the number of leading chunks the launch hashes (all, or all but a short last chunk).
 cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                       uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
-                                      const uint32_t *d_one, int sm_count, cudaStream_t stream);
+                                      const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *covered);
 
 // The same two-warp kernel for tensors at any alignment; message k of the launch is tensor d_order[k]
 // (d_order may be NULL for index order).
