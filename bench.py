@@ -297,10 +297,10 @@ def run_ours(args):
 
     peak_gbs = SM_COUNT * INT_LANES_PER_SM * 1.965e9 / INT_OPS_PER_BYTE / 1e9
     achieved = nbytes / (hash_ms * 1e-3) / 1e9
-    # DRAM traffic per launch: ncu measured dram read+write = 1.0005 x the bytes hashed for the sliced kernel
+    # DRAM traffic per launch: ncu measured dram read+write = 1.0034 x the bytes hashed for the sliced kernel
     # (2 GiB capture) and 1.001 x for the two-warp kernel (config 2 capture); both scale with the bytes.
     kernel_name = ctx.last_leaf_kernel
-    traffic_factor = {"hash_chunks_sliced_kernel": 1.0005, "hash_chunks_split_kernel": 1.001}.get(kernel_name)
+    traffic_factor = {"hash_chunks_sliced_kernel": 1.0034, "hash_chunks_split_kernel": 1.001}.get(kernel_name)
     # what the chain count allows: chains x 64 B x f / (cycles one chain needs per block when it has a
     # scheduler to itself: 2,000 for the two-warp kernel)
     chain_bound = n_units * 64 * 1.965e9 / 2000.0 / 1e9
