@@ -186,12 +186,17 @@ def run_ours(args):
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
     if rank == 0 and iv_build.is_stale():
         iv_build.build()
+    if args.same_device:                     # checking the multi-rank logic on a box with one GPU (with gloo)
+        local_rank = 0
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=device)
+        if args.dist_backend == "nccl":
+            dist.init_process_group("nccl", device_id=device)
+        else:
+            dist.init_process_group(args.dist_backend)
         dist.barrier()
 
     cfg_id, fallback = pick_config(args.config, device)
@@ -521,6 +526,9 @@ def main():
     ap.add_argument("--two-level", type=int, default=None, metavar="SUB_BYTES",
                     help="two-level leaves: chunk digest = Merkle root over SHA-256 of SUB_BYTES pieces (a different, "
                          "separately named leaf definition; not the default)")
+    ap.add_argument("--dist-backend", default="nccl", help="torch.distributed backend for --gpus > 1")
+    ap.add_argument("--same-device", action="store_true",
+                    help="put every rank on cuda:0 (only to check the multi-rank logic on a one-GPU box, with gloo)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
