@@ -240,7 +240,7 @@ cudaError_t launch_staged(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk
 bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count) {
     const uint64_t warps = (n_chunks + 31) / 32;
     const bool aligned = ((reinterpret_cast<uintptr_t>(d_data) & 15u) == 0) && (chunk_bytes % 16u == 0);
-    return aligned && chunk_bytes >= 32768 && warps > 4ull * (uint64_t)sm_count;
+    return aligned && chunk_bytes >= 4096 && warps > 2ull * (uint64_t)sm_count;
 }
 
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
@@ -260,9 +260,6 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
             *kernel_used = "hash_chunks_split_kernel";
             return launch_hash_chunks_split(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one, stream);
         }
-        *kernel_used = "hash_chunks_staged_kernel";
-        if (warps <= 4ull * sm_count)
-            return launch_staged<512, 3, 1, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);
         // Many chains of sliceable size: chains migrate between schedulers (two launches: queue set-up + workers).
         if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
             if (launches) ++*launches;
@@ -278,7 +275,10 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
                                                           d_digests + 32 * covered);
             return cudaGetLastError();
         }
-        // Many small chunks: two CTAs of four warps per SM keep two warps on every scheduler.
+        // (no scratch supplied) two CTAs of four warps per SM keep two warps on every scheduler.
+        *kernel_used = "hash_chunks_staged_kernel";
+        if (warps <= 4ull * sm_count)
+            return launch_staged<512, 3, 1, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);
         return launch_staged<256, 3, 4, false>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, stream);
     }
     *kernel_used = "hash_chunks_kernel";

@@ -348,10 +348,12 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     slice_queue_init<<<64, 256, 0, stream>>>(slot, total_tasks, groups, q, next_slice);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    // One persistent CTA of eight warps per SM (two per scheduler).  Measured on 896 groups:
-    // 4 / 5 / 6 / 7 / 8 warps per SM give 687 / 694 / 673 / 703 / 712 GB/s, and two CTAs of four
-    // warps only 574 GB/s; workers that find the FIFO empty sleep in their bounded wait.
-    const uint64_t warps = MAX_WARPS;
+    // One persistent CTA per SM, four warps (one per scheduler, every worker always has a group once there
+    // are 592 groups) or eight (two per scheduler, but with G < 1184 groups the idle workers fall at random,
+    // so some schedulers run one group or none).  With a scheduler running two groups about 1.17 times as fast
+    // as one, eight warps win from G = 0.71 x 1184 up (measured: 640 groups 4 warps 664 GB/s-equivalent
+    // against 632 with eight; 896 groups eight warps 774 against 687-740 with four).
+    const uint64_t warps = 4 * groups >= 23ull * (uint64_t)sm_count ? MAX_WARPS : 4;
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
         map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
         mid, d_one);
