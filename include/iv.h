@@ -268,6 +268,31 @@ int iv_hash_ragged(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets,
                    void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
+ * Resumable per-tensor digests -- the paper's multi-pass processing ("hash state
+ * is maintained across passes to ensure cryptographic continuity"): a tensor
+ * that is larger than a resident window, or that spans two windows, is hashed
+ * part by part.
+ *
+ * d_states holds one iv_sha_state per tensor in DEVICE memory, zero-filled by
+ * the caller before a tensor's first part.  Each call hashes, for every k, the
+ * next length_k bytes of tensor k found at d_base + offset_k and advances state
+ * k.  With finish == 0 every length must be a multiple of 64 bytes (a remainder
+ * is left unhashed and the device status is set to 2); the call with finish != 0
+ * takes the last part (any length, 0 allowed), applies the padding for the
+ * TOTAL length and writes digest k to d_digests + 32 k (d_digests may be NULL
+ * when finish == 0).  At most 32,768 tensors per call (IV_ERR_TOO_LARGE beyond).
+ */
+typedef struct iv_sha_state {
+    uint32_t h[8];     /* chaining value after the bytes hashed so far */
+    uint64_t bytes;    /* bytes hashed so far (0 = fresh) */
+    uint64_t reserved; /* keeps the record at 48 bytes */
+} iv_sha_state;
+
+int iv_hash_ragged_update(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets,
+                          const uint64_t *d_lengths, uint64_t n, iv_sha_state *d_states,
+                          int finish, uint8_t *d_digests, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * Merkle root without allocation (the paper has no counterpart; this exists
  * for callers of this library, see below).
  *

@@ -30,7 +30,7 @@ EXPORTS = (
     "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
     "iv_merkle_root_noalloc", "iv_last_leaf_kernel", "iv_merkle_levels",
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
-    "iv_hash_chunks_two_level", "iv_verify_manifest_two_level",
+    "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update",
 )
 
 
@@ -95,6 +95,8 @@ def load_library() -> ctypes.CDLL:
     lib.iv_hash_chunks_two_level.restype = i32
     lib.iv_verify_manifest_two_level.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), u64, vp, vp, u64, vp]
     lib.iv_verify_manifest_two_level.restype = i32
+    lib.iv_hash_ragged_update.argtypes = [vp, vp, vp, vp, u64, vp, i32, vp, vp]
+    lib.iv_hash_ragged_update.restype = i32
     lib.iv_verify_manifest.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest.restype = i32
     lib.iv_ctx_digests.argtypes = [vp]
@@ -347,6 +349,25 @@ class Context:
                                     active_lanes, iters, out)
         self._check(rc, "iv_probe_alu")
         return float(out[0]), float(out[1])
+
+    SHA_STATE_BYTES = 48
+
+    def new_sha_states(self, n: int) -> torch.Tensor:
+        """Zero-filled iv_sha_state records for n tensors (an (n, 48) uint8 device tensor)."""
+        return torch.zeros((n, self.SHA_STATE_BYTES), dtype=torch.uint8, device=f"cuda:{self.device}")
+
+    def hash_ragged_update(self, base: torch.Tensor, offsets: torch.Tensor, lengths: torch.Tensor,
+                           states: torch.Tensor, finish: bool, out: torch.Tensor | None = None, stream=None):
+        """iv_hash_ragged_update: hash the next part of every tensor; returns the (n, 32) digests when finishing."""
+        n = offsets.numel()
+        assert lengths.numel() == n and states.numel() == n * self.SHA_STATE_BYTES
+        if finish and out is None:
+            out = torch.empty((n, 32), dtype=torch.uint8, device=base.device)
+        rc = self._lib.iv_hash_ragged_update(self._h, _dev_ptr(base) or base.data_ptr(), _dev_ptr(offsets),
+                                             _dev_ptr(lengths), n, _dev_ptr(states), int(finish),
+                                             _dev_ptr(out) if out is not None else None, _stream_ptr(stream))
+        self._check(rc, "iv_hash_ragged_update")
+        return out if finish else None
 
     def last_digests(self, n: int) -> torch.Tensor:
         """Copy of the chunk digests the last verification on this context computed."""

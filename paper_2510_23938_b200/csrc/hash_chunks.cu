@@ -224,12 +224,8 @@ cudaError_t launch_staged(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk
                           uint8_t *d_digests, uint32_t *d_status, cudaStream_t stream) {
     constexpr size_t smem = (size_t)WARPS * STAGES * 32 * (SEG + 16);
     auto kernel = hash_chunks_staged_kernel<SEG, STAGES, WARPS, FMA>;
-    static bool configured = false;      // per-process, per-instantiation; all devices are the same model
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static bool configured[kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
     const uint64_t per_cta = 32ull * WARPS;
     const uint64_t blocks = (n_chunks + per_cta - 1) / per_cta;
     if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;

@@ -330,13 +330,8 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     constexpr size_t smem_per_warp = TILED ? (size_t)STAGES * 8192 : (size_t)STAGES * 32 * (SEG + 16);
     constexpr size_t smem_pad = TILED ? 1024 : 0;
     auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(MAX_WARPS * smem_per_warp + smem_pad));
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static bool configured[kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, total_tasks = 0;
     (void)sliced_scratch_bytes(n_chunks, chunk_bytes, &slice_bytes, &total_tasks, nbytes);
     const uint64_t groups = (n_chunks + 31) / 32;

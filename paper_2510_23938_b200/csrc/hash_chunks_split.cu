@@ -40,7 +40,8 @@ __global__ void __launch_bounds__(64)
 hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                          uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
                          const uint32_t *__restrict__ one_ptr, const uint64_t *__restrict__ offsets,
-                         const uint64_t *__restrict__ lengths, const uint32_t *__restrict__ order) {
+                         const uint64_t *__restrict__ lengths, const uint32_t *__restrict__ order,
+                         iv_sha_state *__restrict__ states, int finish) {
     constexpr uint32_t kLaneStride = SEG + (RAGGED ? 32 : 16);   // data ring: bytes per lane per stage
     constexpr uint32_t kStageBytes = 32 * kLaneStride;
     constexpr int kBlocksPerSeg = SEG / 64;
@@ -67,11 +68,25 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     const uint64_t slot_index = (uint64_t)blockIdx.x * 32 + lane;
     const bool valid = slot_index < n_chunks;
     uint64_t i = slot_index, begin = 0, len = 0;
+    // Resumable hashing (tensors only): `states` carries each message's chaining value and the bytes
+    // hashed so far from call to call; only the finishing call pads and writes digests.  A part that
+    // does not finish its message must be a whole number of blocks (the remainder is not hashed and
+    // the status word says so).
+    uint64_t done_before = 0;
+    const bool resumable = RAGGED && states != nullptr;
+    const bool finishing = !resumable || finish != 0;
     if (RAGGED) {
         if (valid) {
             i = order ? order[slot_index] : slot_index;
             begin = offsets[i];
             len = lengths[i];
+            if (resumable) {
+                done_before = states[i].bytes;
+                if (!finishing && (len & 63u)) {
+                    if (warp == 0) atomicExch(status, (uint32_t)IVK_DEV_BOUNDS);
+                    len &= ~63ull;
+                }
+            }
         }
     } else if (valid) {
         begin = i * chunk_bytes;
@@ -79,7 +94,7 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     }
     // SHA-256 blocks of this lane's message, padding included.  For chunks lane 0 holds the longest
     // message of the warp; for tensors the maximum is taken.
-    const uint64_t my_total = valid ? ((len + 8) >> 6) + 1 : 0;
+    const uint64_t my_total = !valid ? 0 : (finishing ? ((len + 8) >> 6) + 1 : (len >> 6));
     const uint64_t warp_total = RAGGED ? warp_max_u64(my_total) : __shfl_sync(0xffffffffu, my_total, 0);
 
     if (warp == 1) {
@@ -140,7 +155,7 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
                 for (int k = 0; k < 16; ++k) w[k] = RAGGED ? __byte_perm(raw[k], raw[k + 1], sel) : bswap32(raw[k]);
             } else if (blk < my_total) {
                 if (!tail_built) {
-                    (void)sha256_build_tail(p + full_bytes, (uint32_t)(len & 63u), len, tw);
+                    (void)sha256_build_tail(p + full_bytes, (uint32_t)(len & 63u), done_before + len, tw);
                     tail_built = true;
                 }
                 const int t = (int)(blk - my_full);
@@ -173,6 +188,10 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     // ---------------------------------------------------------------------- consumer
     uint32_t st[8], v[8];
     sha256_init(st);
+    if (resumable && valid && done_before != 0) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) st[k] = states[i].h[k];
+    }
 #pragma unroll
     for (int k = 0; k < 8; ++k) v[k] = st[k];
     int slot = 0;
@@ -198,7 +217,12 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
         if (lane == 0) atomicExch(status, (uint32_t)IVK_DEV_TIMEOUT);
         return;
     }
-    if (valid) store_digest(digests + 32 * i, st);
+    if (valid && resumable) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) states[i].h[k] = st[k];
+        states[i].bytes = done_before + len;
+    }
+    if (valid && finishing) store_digest(digests + 32 * i, st);
 }
 
 }  // namespace
@@ -211,35 +235,27 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
     constexpr int SEG = 512, STAGES = 3, NSLOT = 4, MODE = 3;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * 32 * (64 * 4 + 16);
     auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static bool configured[kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
     const uint64_t blocks = (n_chunks + 31) / 32;
     if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
     kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
-                                                   nullptr, nullptr, nullptr);
+                                                   nullptr, nullptr, nullptr, nullptr, 1);
     return cudaGetLastError();
 }
 
 cudaError_t launch_hash_ragged_split(const uint8_t *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
                                      const uint32_t *d_order, uint64_t n, uint8_t *d_digests, uint32_t *d_status,
-                                     const uint32_t *d_one, cudaStream_t stream) {
+                                     const uint32_t *d_one, iv_sha_state *d_states, int finish, cudaStream_t stream) {
     constexpr int SEG = 512, STAGES = 3, NSLOT = 4, MODE = 3;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 32) + (size_t)NSLOT * 32 * (64 * 4 + 16);
     auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, true>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static bool configured[kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
     const uint64_t blocks = (n + 31) / 32;
     if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
     kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_base, 0, 0, n, d_digests, d_status, d_one, d_offsets, d_lengths,
-                                                   d_order);
+                                                   d_order, d_states, finish);
     return cudaGetLastError();
 }
 

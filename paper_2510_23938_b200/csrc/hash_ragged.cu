@@ -113,7 +113,8 @@ cudaError_t launch_hash_ragged(const uint8_t *d_base, const uint64_t *d_offsets,
         if (e0 != cudaSuccess) return e0;
         if (launches) *launches += 2;
         *kernel_used = "hash_chunks_split_kernel (tensors)";
-        return launch_hash_ragged_split(d_base, d_offsets, d_lengths, d_order, n, d_digests, d_status, d_one, stream);
+        return launch_hash_ragged_split(d_base, d_offsets, d_lengths, d_order, n, d_digests, d_status, d_one, nullptr, 1,
+                                        stream);
     }
     cudaError_t e = cudaMemsetAsync(d_queue, 0, sizeof(unsigned long long), stream);
     if (e != cudaSuccess) return e;

@@ -561,6 +561,22 @@ int iv_hash_ragged(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets, c
     return IV_OK;
 }
 
+int iv_hash_ragged_update(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
+                          uint64_t n, iv_sha_state *d_states, int finish, uint8_t *d_digests, void *cuda_stream) {
+    if (!ctx) return IV_ERR_INVALID_ARG;
+    if (n == 0) return IV_OK;
+    if (!d_base || !d_offsets || !d_lengths || !d_states || (finish && !d_digests)) return IV_ERR_INVALID_ARG;
+    if (n > ivk::kRaggedSortMax) return IV_ERR_TOO_LARGE;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // index order: the parts of one tensor set keep the same message-to-lane assignment from call to call
+    IV_TRY(ctx, ivk::launch_hash_ragged_split(static_cast<const uint8_t *>(d_base), d_offsets, d_lengths, nullptr, n,
+                                              d_digests, ctx->d_status, ctx->d_one, d_states, finish, stream));
+    ++ctx->launches;
+    ctx->leaf_kernel = "hash_chunks_split_kernel (tensors)";
+    return IV_OK;
+}
+
 int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t blocks_per_sm, uint32_t active_lanes,
                  uint32_t iters, double *h_out) {
     if (!ctx || !h_out || warps_per_block == 0 || warps_per_block > 32 || blocks_per_sm == 0 ||

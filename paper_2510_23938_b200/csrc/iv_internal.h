@@ -7,6 +7,22 @@
 
 namespace ivk {
 
+// Opts a kernel into `bytes` of dynamic shared memory on the CURRENT device, once per device and
+// kernel (the attribute is per device; a process may drive several GPUs).  `done` is the caller's
+// static table, one flag per device ordinal.
+constexpr int kMaxDevices = 64;
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, size_t bytes, bool (&done)[kMaxDevices]) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (done[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) done[dev] = true;
+    return e;
+}
+
 // Device-side status values written to iv_verify_result::status.
 enum : uint32_t { IVK_DEV_OK = 0, IVK_DEV_TIMEOUT = 1, IVK_DEV_BOUNDS = 2 };
 
@@ -42,9 +58,10 @@ cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, ui
 
 // The same two-warp kernel for tensors at any alignment; message k of the launch is tensor d_order[k]
 // (d_order may be NULL for index order).
+// d_states (may be NULL): resumable hashing, see iv_hash_ragged_update; finish = 0 leaves the messages open.
 cudaError_t launch_hash_ragged_split(const uint8_t *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
                                      const uint32_t *d_order, uint64_t n, uint8_t *d_digests, uint32_t *d_status,
-                                     const uint32_t *d_one, cudaStream_t stream);
+                                     const uint32_t *d_one, iv_sha_state *d_states, int finish, cudaStream_t stream);
 
 // hash_ragged.cu -----------------------------------------------------------
 // One SHA-256 per (offset, length).  Up to kRaggedSortMax tensors are ordered by descending length

@@ -438,6 +438,37 @@ def test_hash_ragged_every_16_byte_misalignment_with_long_messages(ctx):
     assert ctx.device_status() == 0
 
 
+def test_hash_ragged_update_in_parts_equals_one_shot_digests(ctx):
+    """Multi-pass hashing: every tensor is fed in three parts (whole blocks, whole blocks, the rest) from
+    different places of the buffer; the chaining values travel in the state records."""
+    rng = np.random.default_rng(51)
+    n = 300
+    sizes = np.concatenate([rng.integers(0, 5000, size=n - 6), [0, 63, 64, 65, 200_000, 1_000_003]]).astype(np.int64)
+    offs = inputs.packed_offsets(sizes, first=5)
+    base = inputs.uniform_bytes(int(offs[-1] + sizes[-1]) + 16, seed=52, device="cuda")
+    host = _host(base)
+    want = oracle.hash_ragged(host, offs, sizes, nthreads=oracle.host_threads())
+    # cut points: multiples of 64 inside each tensor
+    blocks = sizes // 64
+    cut1 = (blocks * rng.uniform(0, 1, size=n)).astype(np.int64) * 64
+    cut2 = cut1 + ((blocks - cut1 // 64) * rng.uniform(0, 1, size=n)).astype(np.int64) * 64
+    states = ctx.new_sha_states(n)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int64)).cuda()
+    assert ctx.hash_ragged_update(base, dev(offs), dev(cut1), states, finish=False) is None
+    ctx.hash_ragged_update(base, dev(offs + cut1), dev(cut2 - cut1), states, finish=False)
+    got = ctx.hash_ragged_update(base, dev(offs + cut2), dev(sizes - cut2), states, finish=True)
+    assert np.array_equal(_host(got), want)
+    assert ctx.device_status() == 0
+    # one-shot through the same entry point
+    fresh = ctx.new_sha_states(n)
+    got1 = ctx.hash_ragged_update(base, dev(offs), dev(sizes), fresh, finish=True)
+    assert np.array_equal(_host(got1), want)
+    # a non-final part that is not a whole number of blocks is refused (status 2)
+    bad = ctx.new_sha_states(2)
+    ctx.hash_ragged_update(base, dev([0, 100]), dev([64, 65]), bad, finish=False)
+    assert ctx.device_status() == 2
+
+
 def test_hash_ragged_empty_set(ctx):
     base = inputs.uniform_bytes(64, seed=1, device="cuda")
     e = torch.empty(0, dtype=torch.int64, device="cuda")
