@@ -357,7 +357,8 @@ typedef enum iv_probe_kind {
     IV_PROBE_ROUNDS_M5 = 19,
     IV_PROBE_SHA256_ADD2 = 20, /* kinds 20..22: full compressions with the additions placed as the */
     IV_PROBE_SHA256_ADD3 = 21, /* library's addition placements 2, 3 and 4                          */
-    IV_PROBE_SHA256_ADD4 = 22
+    IV_PROBE_SHA256_ADD4 = 22,
+    IV_PROBE_ROUNDS_M3_HANDSHAKE = 23 /* kind 16 plus the consumer's per-block hand-over (barrier wait, arrival, feed-forward) */
 } iv_probe_kind;
 int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t blocks_per_sm,
                  uint32_t active_lanes, uint32_t iters, double *h_out);

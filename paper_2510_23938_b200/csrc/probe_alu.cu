@@ -97,20 +97,50 @@ __global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, unsigned
 }
 
 // The consumer half alone: 64 rounds per trip, W + K read from a (constant) shared-memory slot.
-template <int MODE>
+// HANDSHAKE adds what the split kernel's consumer does around the rounds: a wait on a "full"
+// barrier (completed just before by lane 0 itself), the warp barrier, the "empty" arrival and the
+// feed-forward, so the difference to the plain kind is the cost of the hand-over.
+template <int MODE, bool HANDSHAKE = false>
 __global__ void probe_rounds_kernel(uint32_t iters, uint32_t active_lanes, unsigned long long *cycles, uint32_t *sink) {
     __shared__ __align__(16) uint32_t slot[32 * 68];
+    __shared__ __align__(8) uint64_t bars[2];
+    if (threadIdx.x == 0) {
+        tma::mbar_init(tma::smem_u32(&bars[0]), 1);
+        tma::mbar_init(tma::smem_u32(&bars[1]), 1);
+        tma::fence_barrier_init();
+    }
     for (int i = threadIdx.x; i < 32 * 68; i += blockDim.x) slot[i] = i * 2654435761u;
     __syncthreads();
     const uint32_t one = sink[1];        // the host stored 1 there; the compiler cannot know
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t src = tma::smem_u32(slot) + lane * 272;
-    uint32_t v[8];
+    uint32_t v[8], st[8];
     sha256_init(v);
     v[0] ^= threadIdx.x;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) st[k] = v[k];
+    const uint32_t bar_full = tma::smem_u32(&bars[0]), bar_empty = tma::smem_u32(&bars[1]);
+    uint32_t parity = 0;
     const long long t0 = clock64();
     if (lane < active_lanes)
-        for (uint32_t it = 0; it < iters; ++it) rounds64<MODE>(v, src, one);
+        for (uint32_t it = 0; it < iters; ++it) {
+            if (HANDSHAKE) {
+                if (lane == 0) tma::mbar_arrive(bar_full);
+                if (!__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_full, parity))) break;
+                parity ^= 1u;
+            }
+            rounds64<MODE>(v, src, one);
+            if (HANDSHAKE) {
+                __syncwarp();
+                if (lane == 0) tma::mbar_arrive(bar_empty);
+                const uint32_t keep = (it < iters) ? one : 0u;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    st[k] = padd<true>(v[k], st[k], keep);
+                    v[k] = st[k];
+                }
+            }
+        }
     __syncthreads();
     const long long t1 = clock64();
     if ((v[0] ^ v[5]) == 0x12345u) sink[0] = v[1];
@@ -160,6 +190,7 @@ cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t i
         case IV_PROBE_ROUNDS_M1: probe_rounds_kernel<1><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_ROUNDS_M2: probe_rounds_kernel<2><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_ROUNDS_M3: probe_rounds_kernel<3><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_ROUNDS_M3_HANDSHAKE: probe_rounds_kernel<3, true><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_ROUNDS_M4: probe_rounds_kernel<4><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_ROUNDS_M5: probe_rounds_kernel<5><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_SCHEDULE: probe_schedule_kernel<<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
