@@ -186,6 +186,18 @@ int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
                        const iv_manifest *h_manifest, iv_verify_result *d_result,
                        uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream);
 
+/* Batch verification -- the paper's "multiple models can be verified simultaneously": n_blobs blobs of
+ * the same size (copies, replicas, variants that share a manifest) are verified against ONE manifest in
+ * one pass; all their chunks are independent chains of a single hashing launch, which is what fills the
+ * GPU when one blob alone has few chunks.
+ *   h_d_blobs        HOST array of n_blobs DEVICE pointers (read before returning), at most 64
+ *   d_results        DEVICE array of n_blobs iv_verify_result, one per blob
+ *   d_mismatch_idx   DEVICE array of n_blobs * idx_cap uint64: blob b's ascending list starts at b * idx_cap
+ * Everything else as for iv_verify_manifest. */
+int iv_verify_manifest_batch(iv_ctx *ctx, const void *const *h_d_blobs, uint64_t n_blobs, uint64_t nbytes,
+                             const iv_manifest *h_manifest, iv_verify_result *d_results,
+                             uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream);
+
 /* Device pointer of the digest array the last iv_verify_manifest /
  * iv_verify_streamed on this context wrote (n_chunks * 32 bytes), NULL if none. */
 const uint8_t *iv_ctx_digests(const iv_ctx *ctx);

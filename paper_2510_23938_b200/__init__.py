@@ -6,4 +6,4 @@ the thin Python binding (``binding``), the in-tree build (``build``) and the syn
 input generators used by the tests and the benchmark (``inputs``).
 """
 from .binding import (Context, IvError, Manifest, VerifyResult, load_library, n_chunks,  # noqa: F401
-                      new_result, read_result)
+                      new_result, read_result, read_results)

@@ -30,7 +30,7 @@ EXPORTS = (
     "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
     "iv_merkle_root_noalloc", "iv_last_leaf_kernel", "iv_merkle_levels",
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
-    "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update",
+    "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update", "iv_verify_manifest_batch",
 )
 
 
@@ -97,6 +97,8 @@ def load_library() -> ctypes.CDLL:
     lib.iv_verify_manifest_two_level.restype = i32
     lib.iv_hash_ragged_update.argtypes = [vp, vp, vp, vp, u64, vp, i32, vp, vp]
     lib.iv_hash_ragged_update.restype = i32
+    lib.iv_verify_manifest_batch.argtypes = [vp, ctypes.POINTER(vp), u64, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
+    lib.iv_verify_manifest_batch.restype = i32
     lib.iv_verify_manifest.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest.restype = i32
     lib.iv_ctx_digests.argtypes = [vp]
@@ -287,6 +289,18 @@ class Context:
                                           _dev_ptr(result), _dev_ptr(mismatch_idx), cap, _stream_ptr(stream))
         self._check(rc, "iv_verify_manifest")
 
+    def verify_manifest_batch(self, blobs: list, manifest: Manifest, results: torch.Tensor,
+                              mismatch_idx: torch.Tensor | None, stream=None) -> None:
+        """iv_verify_manifest_batch (asynchronous): `blobs` are equally sized device tensors, `results` a
+        (len(blobs), 48) uint8 device tensor, `mismatch_idx` a (len(blobs), cap) int64 device tensor."""
+        nb = _nbytes(blobs[0])
+        assert all(_nbytes(b) == nb and b.is_cuda and b.is_contiguous() for b in blobs)
+        ptrs = (ctypes.c_void_p * len(blobs))(*[b.data_ptr() for b in blobs])
+        cap = 0 if mismatch_idx is None else mismatch_idx.shape[1]
+        rc = self._lib.iv_verify_manifest_batch(self._h, ptrs, len(blobs), nb, ctypes.byref(manifest), _dev_ptr(results),
+                                                _dev_ptr(mismatch_idx), cap, _stream_ptr(stream))
+        self._check(rc, "iv_verify_manifest_batch")
+
     def verify_streamed(self, host_windows, window_bytes: int, nbytes: int, manifest: Manifest,
                         result: torch.Tensor, mismatch_idx: torch.Tensor | None, stream=None) -> None:
         """iv_verify_streamed (asynchronous).  `host_windows` is a CPU uint8 tensor holding the whole
@@ -409,6 +423,18 @@ def read_result(result: torch.Tensor) -> dict:
     r = VerifyResult.from_buffer_copy(raw)
     return {"status": int(r.status), "root_ok": bool(r.root_ok), "n_mismatch": int(r.n_mismatch),
             "root": bytes(r.root)}
+
+
+def read_results(results: torch.Tensor) -> list:
+    """Decodes an (n, 48) tensor of iv_verify_result records."""
+    raw = results.cpu().numpy().tobytes()
+    size = ctypes.sizeof(VerifyResult)
+    out = []
+    for o in range(0, len(raw), size):
+        r = VerifyResult.from_buffer_copy(raw[o:o + size])
+        out.append({"status": int(r.status), "root_ok": bool(r.root_ok), "n_mismatch": int(r.n_mismatch),
+                    "root": bytes(r.root)})
+    return out
 
 
 def new_result(device) -> torch.Tensor:

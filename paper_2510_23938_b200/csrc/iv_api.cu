@@ -29,6 +29,8 @@ struct iv_ctx {
     uint64_t digests_valid = 0;
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
+    uint8_t *d_batch = nullptr;               // offsets, lengths and roots of iv_verify_manifest_batch
+    uint64_t batch_cap = 0;                   // bytes
     uint8_t *d_sub = nullptr;                 // sub-leaf digests of the two-level mode
     uint64_t sub_cap = 0;                     // in digests
     uint8_t *d_dirty_scratch = nullptr;       // offsets, lengths and fresh digests of iv_tree_update
@@ -248,6 +250,7 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_order);
     cudaFree(ctx->d_dirty_scratch);
     cudaFree(ctx->d_sub);
+    cudaFree(ctx->d_batch);
     cudaFree(ctx->d_window[0]);
     cudaFree(ctx->d_window[1]);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -469,6 +472,63 @@ int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const i
                      stream);
     if (rc != IV_OK) return rc;
     return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream);
+}
+
+int iv_verify_manifest_batch(iv_ctx *ctx, const void *const *h_d_blobs, uint64_t n_blobs, uint64_t nbytes,
+                             const iv_manifest *h_manifest, iv_verify_result *d_results, uint64_t *d_mismatch_idx,
+                             uint64_t idx_cap, void *cuda_stream) {
+    if (!ctx || !d_results || (idx_cap && !d_mismatch_idx)) return IV_ERR_INVALID_ARG;
+    if (n_blobs == 0) return IV_OK;
+    if (!h_d_blobs) return IV_ERR_INVALID_ARG;
+    if (n_blobs > ivk::kMaxBatch) return IV_ERR_TOO_LARGE;
+    int rc = check_manifest(h_manifest, nbytes);
+    if (rc != IV_OK) return rc;
+    ivk::BlobList blobs{};
+    blobs.count = (uint32_t)n_blobs;
+    for (uint64_t b = 0; b < n_blobs; ++b) {
+        if (nbytes && !h_d_blobs[b]) return IV_ERR_INVALID_ARG;
+        blobs.ptr[b] = static_cast<const uint8_t *>(h_d_blobs[b]);
+    }
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint64_t n = h_manifest->n_chunks, total = n * n_blobs;
+    rc = grow(ctx, &ctx->d_digests, &ctx->digests_cap, total + 1, 32);
+    if (rc != IV_OK) return rc;
+    // scratch: offsets[total] | lengths[total] | one root per blob
+    rc = grow(ctx, &ctx->d_batch, &ctx->batch_cap, 16 * total + 32 * n_blobs + 64, 1);
+    if (rc != IV_OK) return rc;
+    uint64_t *d_off = reinterpret_cast<uint64_t *>(ctx->d_batch);
+    uint64_t *d_len = d_off + total;
+    uint8_t *d_roots = reinterpret_cast<uint8_t *>(d_len + total);
+    if (total && total <= ivk::kRaggedSortMax) {
+        rc = grow(ctx, &ctx->d_order, &ctx->order_cap, total, sizeof(uint32_t));
+        if (rc != IV_OK) return rc;
+    }
+    rc = ensure_merkle_scratch(ctx, n);
+    if (rc != IV_OK) return rc;
+    rc = grow(ctx, &ctx->d_words, &ctx->words_cap, (n + 31) / 32 + 1, sizeof(uint32_t));
+    if (rc != IV_OK) return rc;
+    if (total) {
+        // all blobs' chunks are independent chains of one launch
+        IV_TRY(ctx, ivk::launch_batch_ranges(blobs, n, nbytes, h_manifest->chunk_bytes, d_off, d_len, stream,
+                                             &ctx->launches));
+        IV_TRY(ctx, ivk::launch_hash_ragged(blobs.ptr[0], d_off, d_len, total, ctx->d_digests, ctx->d_queue,
+                                            total <= ivk::kRaggedSortMax ? ctx->d_order : nullptr, ctx->d_status,
+                                            ctx->d_one, ctx->sm_count, stream, &ctx->launches, &ctx->leaf_kernel));
+    }
+    ivk::RootBytes expect;
+    std::memcpy(expect.b, h_manifest->root, 32);
+    for (uint64_t b = 0; b < n_blobs; ++b) {
+        const uint8_t *dig = ctx->d_digests + 32 * n * b;
+        IV_TRY(ctx, ivk::launch_merkle_root(dig, n, d_roots + 32 * b, ctx->d_merkle_a, ctx->d_merkle_b, ctx->d_tickets,
+                                            stream, &ctx->launches));
+        IV_TRY(ctx, ivk::launch_verify_compare(dig, h_manifest->d_digests, n, d_roots + 32 * b, expect, d_results + b,
+                                               idx_cap ? d_mismatch_idx + b * idx_cap : nullptr, idx_cap, ctx->d_words,
+                                               ctx->d_tickets + ivk::kMerkleMaxPasses, ctx->d_status, stream,
+                                               &ctx->launches));
+    }
+    ctx->digests_valid = total;
+    return IV_OK;
 }
 
 int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_windows, uint64_t window_bytes,

@@ -86,6 +86,15 @@ cudaError_t launch_merkle_root(const uint8_t *d_leaves, uint64_t n, uint8_t *d_r
 cudaError_t launch_merkle_levels(const uint8_t *d_in, uint64_t n, uint32_t levels, uint8_t *d_out,
                                  cudaStream_t stream, uint64_t *launches);
 
+// Several blobs of equal size verified in one pass (batch verification): their chunks as one tensor list.
+constexpr uint32_t kMaxBatch = 64;
+struct BlobList {
+    const uint8_t *ptr[kMaxBatch];
+    uint32_t count;
+};
+cudaError_t launch_batch_ranges(const BlobList &blobs, uint64_t n_chunks, uint64_t nbytes, uint64_t chunk_bytes,
+                                uint64_t *d_offsets, uint64_t *d_lengths, cudaStream_t stream, uint64_t *launches);
+
 // Retained tree (all levels in one array, leaves first, the root last).
 constexpr int kTreeMaxLevels = 40;
 uint64_t tree_records(uint64_t n_leaves);

@@ -227,6 +227,18 @@ __global__ void dirty_ranges_kernel(const uint64_t *__restrict__ dirty, uint64_t
     lengths[t] = (nbytes - begin < chunk_bytes) ? (nbytes - begin) : chunk_bytes;
 }
 
+// chunk ranges of several blobs of equal size as one tensor list: offsets are relative to blob 0
+// (unsigned wrap-around makes blobs below blob 0 work too)
+__global__ void batch_ranges_kernel(BlobList blobs, uint64_t n_chunks, uint64_t nbytes, uint64_t chunk_bytes,
+                                    uint64_t *__restrict__ offsets, uint64_t *__restrict__ lengths) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n_chunks * blobs.count) return;
+    const uint64_t b = t / n_chunks, i = t - b * n_chunks;
+    const uint64_t begin = i * chunk_bytes;
+    offsets[t] = (uint64_t)(blobs.ptr[b] - blobs.ptr[0]) + begin;
+    lengths[t] = (nbytes - begin < chunk_bytes) ? (nbytes - begin) : chunk_bytes;
+}
+
 // new leaf digests (in dirty-list order) into the leaf level of the tree
 __global__ void scatter_leaves_kernel(const uint8_t *__restrict__ fresh, const uint64_t *__restrict__ dirty,
                                       uint64_t n_dirty, uint64_t n_leaves, uint8_t *__restrict__ tree) {
@@ -416,6 +428,15 @@ cudaError_t launch_tree_build(const uint8_t *d_leaves, uint64_t n, uint8_t *d_tr
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
+}
+
+cudaError_t launch_batch_ranges(const BlobList &blobs, uint64_t n_chunks, uint64_t nbytes, uint64_t chunk_bytes,
+                                uint64_t *d_offsets, uint64_t *d_lengths, cudaStream_t stream, uint64_t *launches) {
+    const uint64_t total = n_chunks * blobs.count;
+    batch_ranges_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(blobs, n_chunks, nbytes, chunk_bytes,
+                                                                            d_offsets, d_lengths);
+    if (launches) ++*launches;
+    return cudaGetLastError();
 }
 
 cudaError_t launch_dirty_ranges(const uint64_t *d_dirty, uint64_t n_dirty, uint64_t nbytes, uint64_t chunk_bytes,

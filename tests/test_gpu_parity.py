@@ -247,6 +247,42 @@ def test_verify_small_configuration_with_three_tampered_copies(ctx):
         assert idx == [off // chunk] and not r["root_ok"]
 
 
+def test_batch_verification_of_the_small_configuration_and_its_three_tampered_copies(ctx):
+    """The four verifications of the small configuration as ONE pass (4096 chains in one hashing launch)."""
+    nbytes, chunk = 64 << 20, 64 << 10
+    data = inputs.uniform_bytes(nbytes, seed=1, device="cuda")
+    manifest, digests, root = _manifest_from_oracle(ctx, _host(data), chunk)
+    blobs, want = [data], [(True, 0, [], root)]
+    for seed in (2, 3, 4):
+        off, bit = inputs.flip_position(seed, nbytes)
+        bad = data.clone()
+        bad[off] ^= (1 << bit)
+        blobs.append(bad)
+        want.append(oracle.verify(_host(bad), chunk, digests, root, nthreads=oracle.host_threads()))
+        assert want[-1][2] == [off // chunk]
+    results = torch.zeros((4, 48), dtype=torch.uint8, device="cuda")
+    idx = torch.full((4, 8), -1, dtype=torch.int64, device="cuda")
+    ctx.verify_manifest_batch(blobs, manifest, results, idx)
+    torch.cuda.synchronize()
+    for b, r in enumerate(binding.read_results(results)):
+        got = (r["root_ok"], r["n_mismatch"], [int(v) for v in idx[b, :r["n_mismatch"]].cpu()], r["root"])
+        assert got == want[b], b
+    assert ctx.device_status() == 0
+    # ragged size, unaligned blobs, capacity 0
+    content = inputs.uniform_bytes(100_003, seed=9, device="cuda")
+    small = []
+    for k in (0, 1, 5):                                   # three copies at different byte alignments
+        buf = torch.empty(100_003 + 16, dtype=torch.uint8, device="cuda")
+        buf[k:k + 100_003] = content
+        small.append(buf[k:k + 100_003])
+    small[1][77_777] ^= 4
+    m2, d2, r2 = _manifest_from_oracle(ctx, _host(small[0]), 1000)
+    res2 = torch.zeros((3, 48), dtype=torch.uint8, device="cuda")
+    ctx.verify_manifest_batch(small, m2, res2, None)
+    out = binding.read_results(res2)
+    assert [o["root_ok"] for o in out] == [True, False, True] and [o["n_mismatch"] for o in out] == [0, 1, 0]
+
+
 def test_verify_many_mismatches_ascending_exact_count_and_truncation(ctx):
     chunk, n = 512, 5000
     data = inputs.uniform_bytes(chunk * n - 17, seed=8, device="cuda")
