@@ -29,8 +29,9 @@ struct iv_ctx {
     uint64_t digests_valid = 0;
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
-    uint8_t *d_batch = nullptr;               // offsets, lengths and roots of iv_verify_manifest_batch
+    uint8_t *d_batch = nullptr;               // offsets, lengths, roots, run roots, tickets of iv_verify_manifest_batch
     uint64_t batch_cap = 0;                   // bytes
+    uint64_t batch_blobs = 0, batch_total = 0;   // shape of the last batch (the tickets' position depends on it)
     uint8_t *d_sub = nullptr;                 // sub-leaf digests of the two-level mode
     uint64_t sub_cap = 0;                     // in digests
     uint8_t *d_dirty_scratch = nullptr;       // offsets, lengths and fresh digests of iv_tree_update
@@ -494,12 +495,22 @@ int iv_verify_manifest_batch(iv_ctx *ctx, const void *const *h_d_blobs, uint64_t
     const uint64_t n = h_manifest->n_chunks, total = n * n_blobs;
     rc = grow(ctx, &ctx->d_digests, &ctx->digests_cap, total + 1, 32);
     if (rc != IV_OK) return rc;
-    // scratch: offsets[total] | lengths[total] | one root per blob
-    rc = grow(ctx, &ctx->d_batch, &ctx->batch_cap, 16 * total + 32 * n_blobs + 64, 1);
+    // scratch: offsets[total] | lengths[total] | one root per blob | 512 run roots per blob | one ticket per blob
+    const uint64_t batch_bytes = 16 * total + 32 * n_blobs + 32ull * ivk::kMerkleRun * n_blobs + 4 * n_blobs + 64;
+    const bool fresh = batch_bytes > ctx->batch_cap;
+    rc = grow(ctx, &ctx->d_batch, &ctx->batch_cap, batch_bytes, 1);
     if (rc != IV_OK) return rc;
     uint64_t *d_off = reinterpret_cast<uint64_t *>(ctx->d_batch);
     uint64_t *d_len = d_off + total;
     uint8_t *d_roots = reinterpret_cast<uint8_t *>(d_len + total);
+    uint8_t *d_runs = d_roots + 32 * n_blobs;
+    uint32_t *d_btickets = reinterpret_cast<uint32_t *>(d_runs + 32ull * ivk::kMerkleRun * n_blobs);
+    // tickets must start at zero (the kernel leaves them at zero); a regrown or differently shaped scratch is cleared
+    if (fresh || ctx->batch_blobs != n_blobs || ctx->batch_total != total) {
+        IV_TRY(ctx, cudaMemsetAsync(d_btickets, 0, 4 * n_blobs, stream));
+        ctx->batch_blobs = n_blobs;
+        ctx->batch_total = total;
+    }
     if (total && total <= ivk::kRaggedSortMax) {
         rc = grow(ctx, &ctx->d_order, &ctx->order_cap, total, sizeof(uint32_t));
         if (rc != IV_OK) return rc;
@@ -518,10 +529,15 @@ int iv_verify_manifest_batch(iv_ctx *ctx, const void *const *h_d_blobs, uint64_t
     }
     ivk::RootBytes expect;
     std::memcpy(expect.b, h_manifest->root, 32);
+    const bool one_pass = n > 0 && n <= (uint64_t)ivk::kMerkleRun * ivk::kMerkleRun;
+    if (one_pass)      // all trees in one launch
+        IV_TRY(ctx, ivk::launch_merkle_roots_batch(ctx->d_digests, n, (uint32_t)n_blobs, d_roots, d_runs, d_btickets, stream,
+                                                   &ctx->launches));
     for (uint64_t b = 0; b < n_blobs; ++b) {
         const uint8_t *dig = ctx->d_digests + 32 * n * b;
-        IV_TRY(ctx, ivk::launch_merkle_root(dig, n, d_roots + 32 * b, ctx->d_merkle_a, ctx->d_merkle_b, ctx->d_tickets,
-                                            stream, &ctx->launches));
+        if (!one_pass)
+            IV_TRY(ctx, ivk::launch_merkle_root(dig, n, d_roots + 32 * b, ctx->d_merkle_a, ctx->d_merkle_b, ctx->d_tickets,
+                                                stream, &ctx->launches));
         IV_TRY(ctx, ivk::launch_verify_compare(dig, h_manifest->d_digests, n, d_roots + 32 * b, expect, d_results + b,
                                                idx_cap ? d_mismatch_idx + b * idx_cap : nullptr, idx_cap, ctx->d_words,
                                                ctx->d_tickets + ivk::kMerkleMaxPasses, ctx->d_status, stream,

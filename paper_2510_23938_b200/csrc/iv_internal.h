@@ -82,6 +82,11 @@ cudaError_t launch_merkle_root(const uint8_t *d_leaves, uint64_t n, uint8_t *d_r
                                uint8_t *d_scratch_a, uint8_t *d_scratch_b, uint32_t *d_tickets,
                                cudaStream_t stream, uint64_t *launches);
 
+// Roots of `trees` trees of n <= 262,144 leaves each in ONE launch (leaves of tree y at d_leaves + 32 n y):
+// d_scratch holds trees * 512 records, d_tickets `trees` zeroed words.
+cudaError_t launch_merkle_roots_batch(const uint8_t *d_leaves, uint64_t n, uint32_t trees, uint8_t *d_roots,
+                                      uint8_t *d_scratch, uint32_t *d_tickets, cudaStream_t stream, uint64_t *launches);
+
 // `levels` in 1..9 levels of the reduction: d_in[n] -> d_out[ceil(n / 2^levels)] (no aliasing).
 cudaError_t launch_merkle_levels(const uint8_t *d_in, uint64_t n, uint32_t levels, uint8_t *d_out,
                                  cudaStream_t stream, uint64_t *launches);

@@ -79,12 +79,19 @@ __device__ void store_node(uint8_t *dst, const uint32_t *node) {
 
 // One pass: nodes_in[n] -> nodes_out[ceil(n/512)].  When fuse_top is set (at most
 // 512 run roots) the CTA that takes the last ticket reduces them to d_root too.
+// blockIdx.y selects one of several independent trees of the same size (batch verification): tree y
+// reads nodes_in + y * in_stride, writes nodes_out + y * out_stride, d_root + 32 y and uses ticket[y].
 __global__ void __launch_bounds__(kThreads)
 merkle_pass_kernel(const uint8_t *__restrict__ nodes_in, uint64_t n, uint8_t *__restrict__ nodes_out,
-                   uint8_t *__restrict__ d_root, uint32_t *ticket, int fuse_top) {
+                   uint8_t *__restrict__ d_root, uint32_t *ticket, int fuse_top, uint64_t in_stride = 0,
+                   uint64_t out_stride = 0) {
     __shared__ __align__(16) uint32_t buf_a[kMerkleRun * 8];
     __shared__ __align__(16) uint32_t buf_b[kMerkleRun * 4];
     __shared__ uint32_t s_last;
+    nodes_in += blockIdx.y * in_stride;
+    nodes_out += blockIdx.y * out_stride;
+    d_root += 32 * blockIdx.y;
+    ticket += blockIdx.y;
 
     const uint64_t runs = (n + kMerkleRun - 1) / kMerkleRun;
     for (uint64_t r = blockIdx.x; r < runs; r += gridDim.x) {
@@ -376,6 +383,19 @@ cudaError_t launch_merkle_root(const uint8_t *d_leaves, uint64_t n, uint8_t *d_r
         n = runs;
     }
     return cudaErrorInvalidValue;   // more than 512^8 leaves cannot be addressed
+}
+
+// The roots of `trees` trees of n leaves each (n <= 512 * 512: one fused pass), leaves of tree y at
+// d_leaves + y * 32 n, root y at d_roots + 32 y; d_scratch holds trees * 512 records, d_tickets `trees` zeroed words.
+cudaError_t launch_merkle_roots_batch(const uint8_t *d_leaves, uint64_t n, uint32_t trees, uint8_t *d_roots,
+                                      uint8_t *d_scratch, uint32_t *d_tickets, cudaStream_t stream, uint64_t *launches) {
+    if (n == 0 || trees == 0 || n > (uint64_t)kMerkleRun * kMerkleRun) return cudaErrorInvalidValue;
+    const uint64_t runs = (n + kMerkleRun - 1) / kMerkleRun;
+    const dim3 grid((unsigned)runs, trees);
+    merkle_pass_kernel<<<grid, kThreads, 0, stream>>>(d_leaves, n, d_scratch, d_roots, d_tickets, 1, 32 * n,
+                                                      32ull * kMerkleRun);
+    if (launches) ++*launches;
+    return cudaGetLastError();
 }
 
 cudaError_t launch_merkle_levels(const uint8_t *d_in, uint64_t n, uint32_t levels, uint8_t *d_out,
