@@ -7,8 +7,9 @@ Merkle root, comparison with the manifest (`iv_verify_manifest`; for the ragged 
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
 
-Multi-GPU runs are launched with torch.distributed.run, one rank per GPU; every rank verifies
-its own blob (independent problems, weak scaling, no data-path collective).
+Multi-GPU runs are launched with torch.distributed.run, one rank per GPU; the ranks' blobs are the
+shards of one blob (weak scaling): every rank verifies its shard and the global root is built from an
+all-gather of a few 32-byte tree nodes per rank (the path's only exchange).
 `--impl reference` times the CPU oracle (the plain restatement of the method) on the host cores.
 """
 from __future__ import annotations
