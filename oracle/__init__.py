@@ -66,6 +66,16 @@ def _load():
         lib.ivo_hash_ragged.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                         ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int]
         lib.ivo_hash_ragged.restype = None
+        u64p_ = ctypes.POINTER(ctypes.c_uint64)
+        lib.ivo_constants512.argtypes = [u64p_, u64p_]
+        lib.ivo_constants512.restype = None
+        lib.ivo_sha384.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u8p]
+        lib.ivo_sha384.restype = None
+        lib.ivo_hash_chunks_sha384.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64,
+                                               ctypes.c_void_p, ctypes.c_int]
+        lib.ivo_hash_chunks_sha384.restype = ctypes.c_uint64
+        lib.ivo_merkle_root_sha384.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u8p]
+        lib.ivo_merkle_root_sha384.restype = None
         _lib = lib
         return lib
 
@@ -162,3 +172,42 @@ def hash_ragged(base, offsets, lengths, nthreads: int = 1) -> np.ndarray:
     out = np.zeros((off.size, 32), dtype=np.uint8)
     _load().ivo_hash_ragged(_ptr(arr), _ptr(off), _ptr(ln), off.size, _ptr(out), nthreads)
     return out
+
+
+# ---------------------------------------------------------------------------------------------
+# SHA-384 variant
+
+def constants512():
+    """(K[80], H0 of SHA-384 [8]) as numpy uint64 arrays, derived from the primes."""
+    k = np.zeros(80, dtype=np.uint64)
+    h0 = np.zeros(8, dtype=np.uint64)
+    p64 = ctypes.POINTER(ctypes.c_uint64)
+    _load().ivo_constants512(k.ctypes.data_as(p64), h0.ctypes.data_as(p64))
+    return k, h0
+
+
+def sha384(msg) -> bytes:
+    arr = _as_u8(msg)
+    out = (ctypes.c_uint8 * 48)()
+    _load().ivo_sha384(_ptr(arr), arr.size, out)
+    return bytes(out)
+
+
+def hash_chunks_sha384(data, chunk_bytes: int, nthreads: int = 1) -> np.ndarray:
+    """SHA-384 chunk digests as an (n, 48) uint8 array."""
+    arr = _as_u8(data)
+    if chunk_bytes <= 0:
+        raise ValueError("chunk_bytes must be positive")
+    n = n_chunks(arr.size, chunk_bytes)
+    out = np.zeros((n, 48), dtype=np.uint8)
+    got = _load().ivo_hash_chunks_sha384(_ptr(arr), arr.size, chunk_bytes, _ptr(out), nthreads)
+    assert got == n
+    return out
+
+
+def merkle_root_sha384(leaves) -> bytes:
+    arr = _as_u8(leaves)
+    assert arr.size % 48 == 0
+    out = (ctypes.c_uint8 * 48)()
+    _load().ivo_merkle_root_sha384(_ptr(arr), arr.size // 48, out)
+    return bytes(out)

@@ -309,3 +309,203 @@ void ivo_hash_ragged(const uint8_t *base, const uint64_t *offsets, const uint64_
     ragged_job job = { base, offsets, lengths, digests_out };
     run_tasks(ragged_task, &job, n, nthreads);
 }
+
+/* ------------------------------------------------------------------------- */
+/* SHA-384 (FIPS 180-4 sections 4.1.3, 4.2.3, 5.1.2, 5.3.4, 6.4.2, 6.5).       */
+/* ------------------------------------------------------------------------- */
+
+static uint64_t g_k512[80];
+static uint64_t g_h0_384[8];
+static pthread_once_t g_once512 = PTHREAD_ONCE_INIT;
+
+/* 256-bit unsigned integers as four 64-bit limbs, least significant first: just
+ * enough arithmetic to test r^2 and r^3 against p * 2^128 and p * 2^192. */
+typedef struct { uint64_t w[4]; } u256;
+
+static u256 u256_from_u128(u128 v)
+{
+    u256 r = { { (uint64_t)v, (uint64_t)(v >> 64), 0, 0 } };
+    return r;
+}
+
+/* a * b for a below 2^192 and b below 2^128 (the product must fit 256 bits) */
+static u256 u256_mul(u256 a, u128 b)
+{
+    const uint64_t bl[2] = { (uint64_t)b, (uint64_t)(b >> 64) };
+    u256 r = { { 0, 0, 0, 0 } };
+    for (int i = 0; i < 4; ++i) {
+        u128 carry = 0;
+        for (int j = 0; j < 2 && i + j < 4; ++j) {
+            u128 cur = (u128)a.w[i] * bl[j] + r.w[i + j] + carry;
+            r.w[i + j] = (uint64_t)cur;
+            carry = cur >> 64;
+        }
+        for (int k = i + 2; k < 4 && carry; ++k) {
+            u128 cur = (u128)r.w[k] + carry;
+            r.w[k] = (uint64_t)cur;
+            carry = cur >> 64;
+        }
+    }
+    return r;
+}
+
+static int u256_le(u256 a, u256 b)
+{
+    for (int i = 3; i >= 0; --i) {
+        if (a.w[i] != b.w[i]) return a.w[i] < b.w[i];
+    }
+    return 1;
+}
+
+/* p * 2^shift for shift = 128 or 192 */
+static u256 u256_prime_shifted(unsigned p, int shift)
+{
+    u256 r = { { 0, 0, 0, 0 } };
+    r.w[shift / 64] = p;
+    return r;
+}
+
+/* floor(root_degree(p) * 2^64), degree 2 or 3, bit by bit from the top */
+static u128 scaled_root(unsigned p, int degree)
+{
+    const u256 target = u256_prime_shifted(p, 64 * degree);
+    u128 r = 0;
+    for (int bit = 68; bit >= 0; --bit) {
+        const u128 cand = r | ((u128)1 << bit);
+        u256 pw = u256_mul(u256_from_u128(cand), cand);
+        if (degree == 3) pw = u256_mul(pw, cand);
+        /* cand < 2^69 keeps every product below 2^207 */
+        if (u256_le(pw, target)) r = cand;
+    }
+    return r;
+}
+
+static void derive_constants512(void)
+{
+    int found = 0;
+    for (unsigned p = 2; found < 80; ++p) {
+        int prime = 1;
+        for (unsigned q = 2; q * q <= p; ++q)
+            if (p % q == 0) { prime = 0; break; }
+        if (!prime) continue;
+        g_k512[found] = (uint64_t)scaled_root(p, 3);            /* first 64 fraction bits of the cube root */
+        if (found >= 8 && found < 16)                           /* SHA-384: the 9th to 16th primes */
+            g_h0_384[found - 8] = (uint64_t)scaled_root(p, 2);  /* first 64 fraction bits of the square root */
+        ++found;
+    }
+}
+
+void ivo_constants512(uint64_t k_out[80], uint64_t h0_384_out[8])
+{
+    pthread_once(&g_once512, derive_constants512);
+    memcpy(k_out, g_k512, sizeof g_k512);
+    memcpy(h0_384_out, g_h0_384, sizeof g_h0_384);
+}
+
+static uint64_t rotr64(uint64_t x, unsigned n) { return (x >> n) | (x << (64u - n)); }
+static uint64_t ch64(uint64_t x, uint64_t y, uint64_t z) { return (x & y) ^ (~x & z); }
+static uint64_t maj64(uint64_t x, uint64_t y, uint64_t z) { return (x & y) ^ (x & z) ^ (y & z); }
+static uint64_t big_sigma0_512(uint64_t x) { return rotr64(x, 28) ^ rotr64(x, 34) ^ rotr64(x, 39); }
+static uint64_t big_sigma1_512(uint64_t x) { return rotr64(x, 14) ^ rotr64(x, 18) ^ rotr64(x, 41); }
+static uint64_t small_sigma0_512(uint64_t x) { return rotr64(x, 1) ^ rotr64(x, 8) ^ (x >> 7); }
+static uint64_t small_sigma1_512(uint64_t x) { return rotr64(x, 19) ^ rotr64(x, 61) ^ (x >> 6); }
+
+/* FIPS 180-4 section 6.4.2: one 1024-bit block into the hash state. */
+static void process_block512(uint64_t hash[8], const uint8_t block[128])
+{
+    uint64_t w[80];
+    for (int t = 0; t < 16; ++t) {
+        uint64_t v = 0;
+        for (int b = 0; b < 8; ++b) v = (v << 8) | block[8 * t + b];
+        w[t] = v;
+    }
+    for (int t = 16; t < 80; ++t)
+        w[t] = small_sigma1_512(w[t - 2]) + w[t - 7] + small_sigma0_512(w[t - 15]) + w[t - 16];
+
+    uint64_t a = hash[0], b = hash[1], c = hash[2], d = hash[3];
+    uint64_t e = hash[4], f = hash[5], g = hash[6], h = hash[7];
+    for (int t = 0; t < 80; ++t) {
+        uint64_t t1 = h + big_sigma1_512(e) + ch64(e, f, g) + g_k512[t] + w[t];
+        uint64_t t2 = big_sigma0_512(a) + maj64(a, b, c);
+        h = g; g = f; f = e; e = d + t1;
+        d = c; c = b; b = a; a = t1 + t2;
+    }
+    hash[0] += a; hash[1] += b; hash[2] += c; hash[3] += d;
+    hash[4] += e; hash[5] += f; hash[6] += g; hash[7] += h;
+}
+
+/* FIPS 180-4 section 5.1.2 (padding to 1024-bit blocks, 128-bit length) + 6.5 (truncation). */
+void ivo_sha384(const uint8_t *msg, uint64_t len, uint8_t out[48])
+{
+    pthread_once(&g_once512, derive_constants512);
+    uint64_t hash[8];
+    memcpy(hash, g_h0_384, sizeof hash);
+
+    uint64_t full = len / 128;
+    for (uint64_t i = 0; i < full; ++i)
+        process_block512(hash, msg + 128 * i);
+
+    uint8_t tail[256];
+    uint64_t rem = len - 128 * full;
+    memset(tail, 0, sizeof tail);
+    if (rem) memcpy(tail, msg + 128 * full, rem);
+    tail[rem] = 0x80;
+    uint64_t tail_len = (rem + 1 + 16 <= 128) ? 128 : 256;
+    /* the length in bits as a 128-bit big-endian integer; len < 2^64 bytes, so bits < 2^67 */
+    u128 bits = (u128)len * 8u;
+    for (int i = 0; i < 16; ++i)
+        tail[tail_len - 1 - i] = (uint8_t)(bits >> (8 * i));
+    for (uint64_t off = 0; off < tail_len; off += 128)
+        process_block512(hash, tail + off);
+
+    for (int i = 0; i < 6; ++i)                     /* the leftmost 384 bits */
+        for (int b = 0; b < 8; ++b)
+            out[8 * i + b] = (uint8_t)(hash[i] >> (56 - 8 * b));
+}
+
+typedef struct {
+    const uint8_t *data;
+    uint64_t nbytes, chunk_bytes;
+    uint8_t *out;
+} chunk384_job;
+
+static void chunk384_task(void *arg, uint64_t i)
+{
+    chunk384_job *job = (chunk384_job *)arg;
+    uint64_t begin = i * job->chunk_bytes;
+    uint64_t end = begin + job->chunk_bytes;
+    if (end > job->nbytes || end < begin) end = job->nbytes;
+    ivo_sha384(job->data + begin, end - begin, job->out + 48 * i);
+}
+
+uint64_t ivo_hash_chunks_sha384(const uint8_t *data, uint64_t nbytes, uint64_t chunk_bytes,
+                                uint8_t *digests_out, int nthreads)
+{
+    if (chunk_bytes == 0 || nbytes == 0) return 0;
+    uint64_t n = nbytes / chunk_bytes + (nbytes % chunk_bytes ? 1 : 0);
+    chunk384_job job = { data, nbytes, chunk_bytes, digests_out };
+    run_tasks(chunk384_task, &job, n, nthreads);
+    return n;
+}
+
+void ivo_merkle_root_sha384(const uint8_t *leaves, uint64_t n, uint8_t root_out[48])
+{
+    if (n == 0) { ivo_sha384((const uint8_t *)"", 0, root_out); return; }
+    uint8_t *level = (uint8_t *)malloc((size_t)n * 48);
+    memcpy(level, leaves, (size_t)n * 48);
+    while (n > 1) {
+        uint64_t parents = n / 2;
+        for (uint64_t j = 0; j < parents; ++j) {
+            uint8_t node[48];
+            ivo_sha384(level + 96 * j, 96, node);      /* left || right are adjacent records */
+            memcpy(level + 48 * j, node, 48);
+        }
+        if (n % 2) {
+            memmove(level + 48 * parents, level + 48 * (n - 1), 48);
+            ++parents;
+        }
+        n = parents;
+    }
+    memcpy(root_out, level, 48);
+    free(level);
+}

@@ -66,6 +66,19 @@ uint64_t ivo_verify(const uint8_t *data, uint64_t nbytes, uint64_t chunk_bytes,
 void ivo_hash_ragged(const uint8_t *base, const uint64_t *offsets, const uint64_t *lengths,
                      uint64_t n, uint8_t *digests_out, int nthreads);
 
+/* ---------------------------------------------------------------------------
+ * SHA-384 variant (the digest of the paper's own listings).  FIPS 180-4 section
+ * 6.5 (SHA-384 = SHA-512 with the initial value of 5.3.4, truncated to 384
+ * bits), sections 4.1.3, 4.2.3, 5.1.2.  Digests are 48 bytes.  The tree rule is
+ * the same with SHA-384 as the node hash: parent = SHA-384(left || right) over
+ * exactly 96 bytes, odd last node promoted, zero leaves give SHA-384("").
+ * ------------------------------------------------------------------------- */
+void ivo_constants512(uint64_t k_out[80], uint64_t h0_384_out[8]);
+void ivo_sha384(const uint8_t *msg, uint64_t len, uint8_t out[48]);
+uint64_t ivo_hash_chunks_sha384(const uint8_t *data, uint64_t nbytes, uint64_t chunk_bytes,
+                                uint8_t *digests_out, int nthreads);
+void ivo_merkle_root_sha384(const uint8_t *leaves, uint64_t n, uint8_t root_out[48]);
+
 #ifdef __cplusplus
 }
 #endif
