@@ -305,6 +305,20 @@ int iv_hash_ragged_update(iv_ctx *ctx, const void *d_base, const uint64_t *d_off
                           int finish, uint8_t *d_digests, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
+ * SHA-384 variant -- the digest of the paper's own kernel listings (FIPS 180-4
+ * section 6.5).  Chunking and tree rule as above with 48-byte records: digest i
+ * = SHA-384(chunk i); parent = SHA-384(left || right) over exactly 96 bytes, an
+ * unpaired last node moves up unchanged, one leaf is its own root, zero leaves
+ * give SHA-384 of the empty string.  A plain implementation (one chain per lane,
+ * direct loads): it is not tuned like the SHA-256 path.
+ */
+int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                          uint8_t *d_digests, uint64_t digests_cap, uint64_t *h_n_chunks,
+                          void *cuda_stream);
+int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
+                          void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * Merkle root without allocation (the paper has no counterpart; this exists
  * for callers of this library, see below).
  *

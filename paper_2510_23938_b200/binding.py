@@ -31,6 +31,7 @@ EXPORTS = (
     "iv_merkle_root_noalloc", "iv_last_leaf_kernel", "iv_merkle_levels",
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
     "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update", "iv_verify_manifest_batch",
+    "iv_hash_chunks_sha384", "iv_merkle_root_sha384",
 )
 
 
@@ -99,6 +100,10 @@ def load_library() -> ctypes.CDLL:
     lib.iv_hash_ragged_update.restype = i32
     lib.iv_verify_manifest_batch.argtypes = [vp, ctypes.POINTER(vp), u64, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest_batch.restype = i32
+    lib.iv_hash_chunks_sha384.argtypes = [vp, vp, u64, u64, vp, u64, ctypes.POINTER(u64), vp]
+    lib.iv_hash_chunks_sha384.restype = i32
+    lib.iv_merkle_root_sha384.argtypes = [vp, vp, u64, vp, vp]
+    lib.iv_merkle_root_sha384.restype = i32
     lib.iv_verify_manifest.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest.restype = i32
     lib.iv_ctx_digests.argtypes = [vp]
@@ -234,6 +239,25 @@ class Context:
             out = torch.empty(32, dtype=torch.uint8, device=leaves.device)
         rc = self._lib.iv_merkle_root(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
         self._check(rc, "iv_merkle_root")
+        return out
+
+    def hash_chunks_sha384(self, data: torch.Tensor, chunk_bytes: int, stream=None) -> torch.Tensor:
+        """iv_hash_chunks_sha384: (n, 48) uint8 SHA-384 digests of the chunks of `data`."""
+        nb = _nbytes(data)
+        n = n_chunks(nb, chunk_bytes) if chunk_bytes > 0 else 0
+        out = torch.empty((n, 48), dtype=torch.uint8, device=data.device)
+        got = ctypes.c_uint64(0)
+        rc = self._lib.iv_hash_chunks_sha384(self._h, _dev_ptr(data), nb, chunk_bytes, _dev_ptr(out), n,
+                                             ctypes.byref(got), _stream_ptr(stream))
+        self._check(rc, "iv_hash_chunks_sha384")
+        return out[:got.value]
+
+    def merkle_root_sha384(self, leaves: torch.Tensor, stream=None) -> torch.Tensor:
+        """iv_merkle_root_sha384: 48-byte root of (n, 48) leaf digests."""
+        n = leaves.numel() // 48
+        out = torch.empty(48, dtype=torch.uint8, device=leaves.device)
+        rc = self._lib.iv_merkle_root_sha384(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
+        self._check(rc, "iv_merkle_root_sha384")
         return out
 
     def merkle_levels(self, nodes: torch.Tensor, levels: int, stream=None) -> torch.Tensor:

@@ -29,6 +29,8 @@ struct iv_ctx {
     uint64_t digests_valid = 0;
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
+    uint8_t *d_tree384[2] = {nullptr, nullptr};   // level ping-pong of the SHA-384 tree
+    uint64_t tree384_cap = 0;                 // in records of 48 bytes, each buffer
     uint8_t *d_batch = nullptr;               // offsets, lengths, roots, run roots, tickets of iv_verify_manifest_batch
     uint64_t batch_cap = 0;                   // bytes
     uint64_t batch_blobs = 0, batch_total = 0;   // shape of the last batch (the tickets' position depends on it)
@@ -252,6 +254,8 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_dirty_scratch);
     cudaFree(ctx->d_sub);
     cudaFree(ctx->d_batch);
+    cudaFree(ctx->d_tree384[0]);
+    cudaFree(ctx->d_tree384[1]);
     cudaFree(ctx->d_window[0]);
     cudaFree(ctx->d_window[1]);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
@@ -650,6 +654,38 @@ int iv_hash_ragged_update(iv_ctx *ctx, const void *d_base, const uint64_t *d_off
                                               d_digests, ctx->d_status, ctx->d_one, d_states, finish, stream));
     ++ctx->launches;
     ctx->leaf_kernel = "hash_chunks_split_kernel (tensors)";
+    return IV_OK;
+}
+
+int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint8_t *d_digests,
+                          uint64_t digests_cap, uint64_t *h_n_chunks, void *cuda_stream) {
+    if (!ctx || chunk_bytes == 0) return IV_ERR_INVALID_ARG;
+    const uint64_t n = chunk_count(nbytes, chunk_bytes);
+    if (n > digests_cap) return IV_ERR_INVALID_ARG;
+    if (n && (!d_data || !d_digests)) return IV_ERR_INVALID_ARG;
+    if (h_n_chunks) *h_n_chunks = n;
+    if (n == 0) return IV_OK;
+    DeviceGuard guard(ctx->device);
+    IV_TRY(ctx, ivk::launch_hash_chunks_sha384(static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
+                                               ctx->sm_count, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+    ctx->leaf_kernel = "hash_chunks_sha384_kernel";
+    return IV_OK;
+}
+
+int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
+    if (!ctx || !d_root || (n_leaves && !d_leaves)) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    const uint64_t need = (n_leaves + 1) / 2 + 1;
+    if (need > ctx->tree384_cap) {
+        uint64_t cap_a = ctx->tree384_cap, cap_b = ctx->tree384_cap;
+        int rc = grow(ctx, &ctx->d_tree384[0], &cap_a, need, 48);
+        if (rc != IV_OK) return rc;
+        rc = grow(ctx, &ctx->d_tree384[1], &cap_b, need, 48);
+        if (rc != IV_OK) return rc;
+        ctx->tree384_cap = cap_a < cap_b ? cap_a : cap_b;
+    }
+    IV_TRY(ctx, ivk::launch_merkle_root_sha384(d_leaves, n_leaves, d_root, ctx->d_tree384[0], ctx->d_tree384[1],
+                                               static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
     return IV_OK;
 }
 

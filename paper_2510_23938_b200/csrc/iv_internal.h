@@ -123,6 +123,13 @@ cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_man
                                   uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
                                   const uint32_t *d_status, cudaStream_t stream, uint64_t *launches);
 
+// hash_sha384.cu -----------------------------------------------------------
+// SHA-384 variant: 48-byte chunk digests and the tree with SHA-384 parents.
+cudaError_t launch_hash_chunks_sha384(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
+                                      uint8_t *d_digests, int sm_count, cudaStream_t stream, uint64_t *launches);
+cudaError_t launch_merkle_root_sha384(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root, uint8_t *d_scratch_a,
+                                      uint8_t *d_scratch_b, cudaStream_t stream, uint64_t *launches);
+
 // probe_alu.cu -------------------------------------------------------------
 cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t iters, uint32_t active_lanes,
                          unsigned long long *d_cycles, uint32_t *d_sink, cudaStream_t stream);
