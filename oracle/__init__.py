@@ -76,6 +76,11 @@ def _load():
         lib.ivo_hash_chunks_sha384.restype = ctypes.c_uint64
         lib.ivo_merkle_root_sha384.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u8p]
         lib.ivo_merkle_root_sha384.restype = None
+        lib.ivo_hash_chunks_rfc6962.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64,
+                                                ctypes.c_void_p, ctypes.c_int]
+        lib.ivo_hash_chunks_rfc6962.restype = ctypes.c_uint64
+        lib.ivo_merkle_root_rfc6962.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u8p]
+        lib.ivo_merkle_root_rfc6962.restype = None
         _lib = lib
         return lib
 
@@ -210,4 +215,27 @@ def merkle_root_sha384(leaves) -> bytes:
     assert arr.size % 48 == 0
     out = (ctypes.c_uint8 * 48)()
     _load().ivo_merkle_root_sha384(_ptr(arr), arr.size // 48, out)
+    return bytes(out)
+
+
+# ---------------------------------------------------------------------------------------------
+# RFC 6962 mode (domain-separated Merkle Tree Hash)
+
+def hash_chunks_rfc6962(data, chunk_bytes: int, nthreads: int = 1) -> np.ndarray:
+    """Leaf hashes SHA-256(0x00 || chunk) as an (n, 32) uint8 array."""
+    arr = _as_u8(data)
+    if chunk_bytes <= 0:
+        raise ValueError("chunk_bytes must be positive")
+    n = n_chunks(arr.size, chunk_bytes)
+    out = np.zeros((n, 32), dtype=np.uint8)
+    got = _load().ivo_hash_chunks_rfc6962(_ptr(arr), arr.size, chunk_bytes, _ptr(out), nthreads)
+    assert got == n
+    return out
+
+
+def merkle_root_rfc6962(leaf_hashes) -> bytes:
+    arr = _as_u8(leaf_hashes)
+    assert arr.size % 32 == 0
+    out = (ctypes.c_uint8 * 32)()
+    _load().ivo_merkle_root_rfc6962(_ptr(arr), arr.size // 32, out)
     return bytes(out)

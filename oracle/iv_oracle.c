@@ -509,3 +509,60 @@ void ivo_merkle_root_sha384(const uint8_t *leaves, uint64_t n, uint8_t root_out[
     memcpy(root_out, level, 48);
     free(level);
 }
+
+/* ------------------------------------------------------------------------- */
+/* RFC 6962 section 2.1: domain-separated Merkle Tree Hash over SHA-256.      */
+/*   leaf hash  = SHA-256(0x00 || entry),  node = SHA-256(0x01 || left || right) */
+/*   MTH({})    = SHA-256(""),             MTH({d0}) = leaf hash of d0           */
+/*   MTH(D[n])  = node(MTH(D[0:k]), MTH(D[k:n])), k the largest power of two < n */
+/* Written as that recursion over the entries (here: the chunks of a blob).   */
+/* ------------------------------------------------------------------------- */
+
+static void rfc6962_leaf(const uint8_t *entry, uint64_t len, uint8_t out[32])
+{
+    uint8_t *msg = (uint8_t *)malloc((size_t)len + 1);
+    msg[0] = 0x00;
+    if (len) memcpy(msg + 1, entry, (size_t)len);
+    ivo_sha256(msg, len + 1, out);
+    free(msg);
+}
+
+static void rfc6962_node(const uint8_t left[32], const uint8_t right[32], uint8_t out[32])
+{
+    uint8_t msg[65];
+    msg[0] = 0x01;
+    memcpy(msg + 1, left, 32);
+    memcpy(msg + 33, right, 32);
+    ivo_sha256(msg, 65, out);
+}
+
+static void chunk6962_task(void *arg, uint64_t i)
+{
+    chunk_job *job = (chunk_job *)arg;
+    uint64_t begin = i * job->chunk_bytes;
+    uint64_t end = begin + job->chunk_bytes;
+    if (end > job->nbytes || end < begin) end = job->nbytes;
+    rfc6962_leaf(job->data + begin, end - begin, job->out + 32 * i);
+}
+
+uint64_t ivo_hash_chunks_rfc6962(const uint8_t *data, uint64_t nbytes, uint64_t chunk_bytes,
+                                 uint8_t *leaf_hashes_out, int nthreads)
+{
+    if (chunk_bytes == 0 || nbytes == 0) return 0;
+    uint64_t n = nbytes / chunk_bytes + (nbytes % chunk_bytes ? 1 : 0);
+    chunk_job job = { data, nbytes, chunk_bytes, leaf_hashes_out };
+    run_tasks(chunk6962_task, &job, n, nthreads);
+    return n;
+}
+
+void ivo_merkle_root_rfc6962(const uint8_t *leaf_hashes, uint64_t n, uint8_t root_out[32])
+{
+    if (n == 0) { ivo_sha256((const uint8_t *)"", 0, root_out); return; }
+    if (n == 1) { memcpy(root_out, leaf_hashes, 32); return; }
+    uint64_t k = 1;
+    while (k * 2 < n) k *= 2;
+    uint8_t left[32], right[32];
+    ivo_merkle_root_rfc6962(leaf_hashes, k, left);
+    ivo_merkle_root_rfc6962(leaf_hashes + 32 * k, n - k, right);
+    rfc6962_node(left, right, root_out);
+}

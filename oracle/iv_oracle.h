@@ -79,6 +79,16 @@ uint64_t ivo_hash_chunks_sha384(const uint8_t *data, uint64_t nbytes, uint64_t c
                                 uint8_t *digests_out, int nthreads);
 void ivo_merkle_root_sha384(const uint8_t *leaves, uint64_t n, uint8_t root_out[48]);
 
+/* ---------------------------------------------------------------------------
+ * RFC 6962 section 2.1 mode (the paper cites RFC 6962 for its tree): the Merkle
+ * Tree Hash with domain separation over SHA-256, the entries being the chunks.
+ * leaf = SHA-256(0x00 || chunk), node = SHA-256(0x01 || left || right), split
+ * at the largest power of two below n, empty list = SHA-256("").
+ * ------------------------------------------------------------------------- */
+uint64_t ivo_hash_chunks_rfc6962(const uint8_t *data, uint64_t nbytes, uint64_t chunk_bytes,
+                                 uint8_t *leaf_hashes_out, int nthreads);
+void ivo_merkle_root_rfc6962(const uint8_t *leaf_hashes, uint64_t n, uint8_t root_out[32]);
+
 #ifdef __cplusplus
 }
 #endif
