@@ -319,6 +319,21 @@ int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leave
                           void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
+ * RFC 6962 section 2.1 mode -- the Merkle Tree Hash the paper cites for its tree,
+ * with that RFC's domain separation, over SHA-256 with the chunks as entries:
+ * leaf hash i = SHA-256(0x00 || chunk i); node = SHA-256(0x01 || left || right)
+ * (65 bytes); the list is split at the largest power of two below n, one entry
+ * is its own leaf hash, no entry gives SHA-256 of the empty string.  Digests
+ * and root differ from the default (unprefixed) path by construction.
+ * Arguments, layout and errors as iv_hash_chunks / iv_merkle_root.
+ */
+int iv_hash_chunks_rfc6962(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                           uint8_t *d_digests, uint64_t digests_cap, uint64_t *h_n_chunks,
+                           void *cuda_stream);
+int iv_merkle_root_rfc6962(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
+                           void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
  * Merkle root without allocation (the paper has no counterpart; this exists
  * for callers of this library, see below).
  *

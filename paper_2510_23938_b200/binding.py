@@ -32,6 +32,7 @@ EXPORTS = (
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
     "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update", "iv_verify_manifest_batch",
     "iv_hash_chunks_sha384", "iv_merkle_root_sha384",
+    "iv_hash_chunks_rfc6962", "iv_merkle_root_rfc6962",
 )
 
 
@@ -104,6 +105,10 @@ def load_library() -> ctypes.CDLL:
     lib.iv_hash_chunks_sha384.restype = i32
     lib.iv_merkle_root_sha384.argtypes = [vp, vp, u64, vp, vp]
     lib.iv_merkle_root_sha384.restype = i32
+    lib.iv_hash_chunks_rfc6962.argtypes = [vp, vp, u64, u64, vp, u64, ctypes.POINTER(u64), vp]
+    lib.iv_hash_chunks_rfc6962.restype = i32
+    lib.iv_merkle_root_rfc6962.argtypes = [vp, vp, u64, vp, vp]
+    lib.iv_merkle_root_rfc6962.restype = i32
     lib.iv_verify_manifest.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest.restype = i32
     lib.iv_ctx_digests.argtypes = [vp]
@@ -258,6 +263,25 @@ class Context:
         out = torch.empty(48, dtype=torch.uint8, device=leaves.device)
         rc = self._lib.iv_merkle_root_sha384(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
         self._check(rc, "iv_merkle_root_sha384")
+        return out
+
+    def hash_chunks_rfc6962(self, data: torch.Tensor, chunk_bytes: int, stream=None) -> torch.Tensor:
+        """iv_hash_chunks_rfc6962: (n, 32) uint8 leaf hashes SHA-256(0x00 || chunk)."""
+        nb = _nbytes(data)
+        n = n_chunks(nb, chunk_bytes) if chunk_bytes > 0 else 0
+        out = torch.empty((n, 32), dtype=torch.uint8, device=data.device)
+        got = ctypes.c_uint64(0)
+        rc = self._lib.iv_hash_chunks_rfc6962(self._h, _dev_ptr(data), nb, chunk_bytes, _dev_ptr(out), n,
+                                              ctypes.byref(got), _stream_ptr(stream))
+        self._check(rc, "iv_hash_chunks_rfc6962")
+        return out[:got.value]
+
+    def merkle_root_rfc6962(self, leaves: torch.Tensor, stream=None) -> torch.Tensor:
+        """iv_merkle_root_rfc6962: 32-byte root with 0x01-prefixed nodes over (n, 32) leaf hashes."""
+        n = leaves.numel() // 32
+        out = torch.empty(32, dtype=torch.uint8, device=leaves.device)
+        rc = self._lib.iv_merkle_root_rfc6962(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
+        self._check(rc, "iv_merkle_root_rfc6962")
         return out
 
     def merkle_levels(self, nodes: torch.Tensor, levels: int, stream=None) -> torch.Tensor:

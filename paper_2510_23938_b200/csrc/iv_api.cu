@@ -29,7 +29,7 @@ struct iv_ctx {
     uint64_t digests_valid = 0;
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
-    uint8_t *d_tree384[2] = {nullptr, nullptr};   // level ping-pong of the SHA-384 tree
+    uint8_t *d_tree384[2] = {nullptr, nullptr};   // level ping-pong of the SHA-384 and RFC 6962 trees
     uint64_t tree384_cap = 0;                 // in records of 48 bytes, each buffer
     uint8_t *d_batch = nullptr;               // offsets, lengths, roots, run roots, tickets of iv_verify_manifest_batch
     uint64_t batch_cap = 0;                   // bytes
@@ -672,20 +672,50 @@ int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint
     return IV_OK;
 }
 
+// Level buffers of the variant trees: two buffers of at least `records` records of 48 bytes.
+static int ensure_variant_tree_scratch(iv_ctx *ctx, uint64_t records) {
+    if (records <= ctx->tree384_cap) return IV_OK;
+    uint64_t cap_a = ctx->tree384_cap, cap_b = ctx->tree384_cap;
+    int rc = grow(ctx, &ctx->d_tree384[0], &cap_a, records, 48);
+    if (rc != IV_OK) return rc;
+    rc = grow(ctx, &ctx->d_tree384[1], &cap_b, records, 48);
+    if (rc != IV_OK) return rc;
+    ctx->tree384_cap = cap_a < cap_b ? cap_a : cap_b;
+    return IV_OK;
+}
+
 int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
     if (!ctx || !d_root || (n_leaves && !d_leaves)) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
-    const uint64_t need = (n_leaves + 1) / 2 + 1;
-    if (need > ctx->tree384_cap) {
-        uint64_t cap_a = ctx->tree384_cap, cap_b = ctx->tree384_cap;
-        int rc = grow(ctx, &ctx->d_tree384[0], &cap_a, need, 48);
-        if (rc != IV_OK) return rc;
-        rc = grow(ctx, &ctx->d_tree384[1], &cap_b, need, 48);
-        if (rc != IV_OK) return rc;
-        ctx->tree384_cap = cap_a < cap_b ? cap_a : cap_b;
-    }
+    int rc = ensure_variant_tree_scratch(ctx, (n_leaves + 1) / 2 + 1);
+    if (rc != IV_OK) return rc;
     IV_TRY(ctx, ivk::launch_merkle_root_sha384(d_leaves, n_leaves, d_root, ctx->d_tree384[0], ctx->d_tree384[1],
                                                static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+    return IV_OK;
+}
+
+int iv_hash_chunks_rfc6962(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint8_t *d_digests,
+                           uint64_t digests_cap, uint64_t *h_n_chunks, void *cuda_stream) {
+    if (!ctx || chunk_bytes == 0) return IV_ERR_INVALID_ARG;
+    const uint64_t n = chunk_count(nbytes, chunk_bytes);
+    if (n > digests_cap) return IV_ERR_INVALID_ARG;
+    if (n && (!d_data || !d_digests)) return IV_ERR_INVALID_ARG;
+    if (h_n_chunks) *h_n_chunks = n;
+    if (n == 0) return IV_OK;
+    DeviceGuard guard(ctx->device);
+    IV_TRY(ctx, ivk::launch_hash_chunks_rfc6962(static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
+                                                ctx->sm_count, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+    ctx->leaf_kernel = "hash_chunks_rfc6962_kernel";
+    return IV_OK;
+}
+
+int iv_merkle_root_rfc6962(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
+    if (!ctx || !d_root || (n_leaves && !d_leaves)) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    int rc = ensure_variant_tree_scratch(ctx, (n_leaves + 1) / 2 + 1);
+    if (rc != IV_OK) return rc;
+    IV_TRY(ctx, ivk::launch_merkle_root_rfc6962(d_leaves, n_leaves, d_root, ctx->d_tree384[0], ctx->d_tree384[1],
+                                                static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
     return IV_OK;
 }
 

@@ -130,6 +130,13 @@ cudaError_t launch_hash_chunks_sha384(const uint8_t *d_data, uint64_t nbytes, ui
 cudaError_t launch_merkle_root_sha384(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root, uint8_t *d_scratch_a,
                                       uint8_t *d_scratch_b, cudaStream_t stream, uint64_t *launches);
 
+// hash_rfc6962.cu ----------------------------------------------------------
+// RFC 6962 section 2.1 mode: prefixed leaf hashes and the tree with prefixed nodes.
+cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
+                                       uint8_t *d_digests, int sm_count, cudaStream_t stream, uint64_t *launches);
+cudaError_t launch_merkle_root_rfc6962(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root, uint8_t *d_scratch_a,
+                                       uint8_t *d_scratch_b, cudaStream_t stream, uint64_t *launches);
+
 // probe_alu.cu -------------------------------------------------------------
 cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t iters, uint32_t active_lanes,
                          unsigned long long *d_cycles, uint32_t *d_sink, cudaStream_t stream);

@@ -1,0 +1,93 @@
+"""GPU parity of the RFC 6962 section 2.1 mode (0x00-prefixed leaf hashes, 0x01-prefixed nodes): leaf
+hashes and roots from the CUDA library equal the CPU oracle's bit for bit.  All calls go through the
+C ABI via the ctypes binding."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_23938_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu-marked tests need a CUDA device")
+    c = binding.Context(0)
+    yield c
+    c.close()
+
+
+def _host(t: torch.Tensor) -> np.ndarray:
+    return t.cpu().numpy()
+
+
+@pytest.mark.parametrize("nbytes,chunk", [
+    (64 << 20, 64 << 10),                 # the small configuration
+    (1 << 20, 4096), (1 << 20, 64), (1 << 20, 1 << 20), (1 << 20, 2 << 20),
+    ((1 << 20) + 77, 4096),
+    (100_003, 1000), (100_003, 1001), (100_003, 7), (65, 64), (64, 64), (63, 64), (62, 64), (1, 1),
+    # last-chunk lengths around the padding boundaries of the message that is one byte longer
+    (5 * 4096 + 54, 4096), (5 * 4096 + 55, 4096), (5 * 4096 + 56, 4096),
+    (5 * 4096 + 62, 4096), (5 * 4096 + 63, 4096), (5 * 4096 + 64, 4096),
+    (5 * 4096 + 118, 4096), (5 * 4096 + 119, 4096), (5 * 4096 + 127, 4096),
+    (37 * 48 + 16, 48),
+    (20_000 * 4096 + 100, 4096),
+])
+def test_leaf_hashes_equal_oracle(ctx, nbytes, chunk):
+    data = inputs.uniform_bytes(nbytes, seed=6962, device="cuda")
+    got = ctx.hash_chunks_rfc6962(data, chunk)
+    want = oracle.hash_chunks_rfc6962(_host(data), chunk, nthreads=oracle.host_threads())
+    assert got.shape == want.shape
+    assert np.array_equal(_host(got), want)
+
+
+@pytest.mark.parametrize("shift", [1, 3, 8, 13])
+@pytest.mark.parametrize("chunk", [256, 1000, 4096 + 3])
+def test_leaf_hashes_any_base_alignment(ctx, shift, chunk):
+    buf = inputs.uniform_bytes(300_000 + 16, seed=6963, device="cuda")
+    data = buf[shift:shift + 300_000]
+    got = ctx.hash_chunks_rfc6962(data, chunk)
+    assert np.array_equal(_host(got), oracle.hash_chunks_rfc6962(_host(data), chunk))
+
+
+def test_every_entry_length_of_three_blocks(ctx):
+    buf = inputs.uniform_bytes(208, seed=6964, device="cuda")          # 16-byte aligned base, any length
+    host = _host(buf)
+    for n in range(1, 193):
+        for off in (0, 16):
+            got = ctx.hash_chunks_rfc6962(buf[off:off + n], 256)
+            assert np.array_equal(_host(got), oracle.hash_chunks_rfc6962(host[off:off + n], 256)), (n, off)
+
+
+def test_empty_and_argument_errors(ctx):
+    empty = torch.empty(0, dtype=torch.uint8, device="cuda")
+    assert ctx.hash_chunks_rfc6962(empty, 4096).shape == (0, 32)
+    with pytest.raises(binding.IvError):
+        ctx.hash_chunks_rfc6962(inputs.uniform_bytes(100, seed=1, device="cuda"), 0)
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 3, 4, 5, 7, 8, 9, 127, 128, 129, 1000, 1023, 1024, 1025, 40_001])
+def test_root_equals_oracle(ctx, n):
+    leaves = inputs.uniform_bytes(32 * n, seed=6965 + n, device="cuda").reshape(n, 32)
+    got = _host(ctx.merkle_root_rfc6962(leaves)).tobytes()
+    assert got == oracle.merkle_root_rfc6962(_host(leaves))
+
+
+def test_root_unaligned_leaf_pointer(ctx):
+    buf = inputs.uniform_bytes(32 * 77 + 5, seed=6966, device="cuda")
+    leaves = buf[5:]
+    assert _host(ctx.merkle_root_rfc6962(leaves)).tobytes() == oracle.merkle_root_rfc6962(_host(leaves))
+
+
+def test_leaves_then_root_differs_from_the_default_path_and_repeats(ctx):
+    data = inputs.uniform_bytes((8 << 20) + 5, seed=6967, device="cuda")
+    want_leaves = oracle.hash_chunks_rfc6962(_host(data), 4096, nthreads=oracle.host_threads())
+    want_root = oracle.merkle_root_rfc6962(want_leaves)
+    for _ in range(3):
+        leaves = ctx.hash_chunks_rfc6962(data, 4096)
+        assert _host(ctx.merkle_root_rfc6962(leaves)).tobytes() == want_root
+    assert _host(ctx.merkle_root(ctx.hash_chunks(data, 4096))).tobytes() != want_root
+    assert ctx.device_status() == 0
