@@ -66,7 +66,8 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
                           uint64_t slice_bytes, uint64_t total_tasks, uint32_t *__restrict__ slot,
                           SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice,
-                          uint32_t *__restrict__ mid /* [groups][8][32] */, const uint32_t *__restrict__ one_ptr) {
+                          uint32_t *__restrict__ mid /* [groups][8][32] */, const uint32_t *__restrict__ one_ptr,
+                          uint32_t first_workers_first) {
     // Addition placement 0 (left to the compiler).  Moving the schedule's additions to the FMA
     // pipe (placement 2) gains 4.5 % in the register-only probe but lost 5 % in this kernel.
     constexpr int ADD = 0;
@@ -97,10 +98,33 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
     uint32_t parity = 0;
     bool failed = false;
 
+    if (first_workers_first && warp >= 4) __nanosleep(20000);   // the first workers of every CTA claim their groups first
     for (;;) {
         // ---- take a ticket, wait for the group that is pushed under it
         unsigned long long t = 0;
-        if (lane == 0) t = atomicAdd(&q->head, 1ull);
+        if (lane == 0) {
+            if (warp < 4 || !first_workers_first) {
+                t = atomicAdd(&q->head, 1ull);
+            } else {
+                // A scheduler's second worker takes a task only when one lies in the FIFO unclaimed: the
+                // first workers (one per scheduler) are served first, so no scheduler idles while another
+                // runs two groups.  With nothing left over it polls; giving up is harmless, the first
+                // workers finish the launch.
+                const long long t0 = clock64();
+                t = total_tasks;
+                for (;;) {
+                    const unsigned long long h = *reinterpret_cast<volatile unsigned long long *>(&q->head);
+                    if (h >= total_tasks) break;
+                    const unsigned long long tl = *reinterpret_cast<volatile unsigned long long *>(&q->tail);
+                    if (tl > h) {
+                        if (atomicCAS(&q->head, h, h + 1ull) == h) { t = h; break; }
+                        continue;
+                    }
+                    if (clock64() - t0 > 8000000000ll) break;
+                    __nanosleep(256);
+                }
+            }
+        }
         t = __shfl_sync(0xffffffffu, t, 0);
         if (t >= total_tasks) break;
         uint32_t entry = 0;
@@ -266,9 +290,9 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
 uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t *slice_bytes_out, uint64_t *total_tasks_out,
                               uint64_t nbytes) {
     const uint64_t groups = (n_chunks + 31) / 32;
-    // slices of at least 16 KiB, at most 64 per chunk, a multiple of 4 KiB
+    // slices of at least 16 KiB, at most 256 per chunk, a multiple of 4 KiB
     uint64_t slices = chunk_bytes / 16384;
-    if (slices > 64) slices = 64;
+    if (slices > 256) slices = 256;
     if (slices < 1) slices = 1;
     uint64_t slice_bytes = (chunk_bytes + slices - 1) / slices;
     slice_bytes = (slice_bytes + 4095) & ~4095ull;
@@ -343,15 +367,23 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     slice_queue_init<<<64, 256, 0, stream>>>(slot, total_tasks, groups, q, next_slice);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    // One persistent CTA per SM, four warps (one per scheduler, every worker always has a group once there
-    // are 592 groups) or eight (two per scheduler, but with G < 1184 groups the idle workers fall at random,
-    // so some schedulers run one group or none).  With a scheduler running two groups about 1.17 times as fast
-    // as one, eight warps win from G = 0.71 x 1184 up (measured: 640 groups 4 warps 664 GB/s-equivalent
-    // against 632 with eight; 896 groups eight warps 774 against 687-740 with four).
-    const uint64_t warps = 4 * groups >= 23ull * (uint64_t)sm_count ? MAX_WARPS : 4;
+    // One persistent CTA per SM with four workers (one per scheduler) or eight (two per scheduler).  A
+    // scheduler with two groups finishes 1.13 groups in the time a scheduler with one finishes one, so
+    // eight workers pay once G is well above 592, but with G < 1184 not every scheduler gets two.  Measured:
+    //  * four workers: 775 GB/s for every G >= 592 (4 MiB chunks, 256 slices);
+    //  * eight workers, FIFO served in arrival order: idle workers fall at random and groups that met
+    //    doubly loaded schedulers more often finish late (G = 896: 763; G = 1024: 827);
+    //  * eight workers, first workers served first (a second worker takes only what is left over): the
+    //    592 - (G - 592) schedulers with one group finish early and then take over the rest; needs fine
+    //    slices (256 per chunk) to balance (G = 832 / 896 / 960: 780 / 790 / 811; with 64 slices it loses).
+    const bool fine = ((chunk_bytes & ~63ull) + slice_bytes - 1) / slice_bytes >= 192;   // about 256 slices per chunk
+    uint64_t warps = 4;
+    uint32_t first_workers_first = 0;
+    if (fine && 5 * groups >= 28ull * (uint64_t)sm_count) { warps = MAX_WARPS; first_workers_first = groups < 8ull * sm_count; }
+    else if (!fine && 10 * groups >= 62ull * (uint64_t)sm_count) warps = MAX_WARPS;
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
         map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
-        mid, d_one);
+        mid, d_one, first_workers_first);
     return cudaGetLastError();
 }
 
