@@ -222,8 +222,13 @@ def run_ours(args):
     else:
         n_units = binding.n_chunks(nbytes, chunk)
         two_level = args.two_level
-        man_digests = ctx.hash_chunks_two_level(data, chunk, two_level) if two_level else ctx.hash_chunks(data, chunk)
-        man_root = bytes(ctx.merkle_root(man_digests).cpu().numpy().tobytes())
+        variant = args.variant
+        if variant == "rfc6962":
+            man_digests = ctx.hash_chunks_rfc6962(data, chunk)
+            man_root = bytes(ctx.merkle_root_rfc6962(man_digests).cpu().numpy().tobytes())
+        else:
+            man_digests = ctx.hash_chunks_two_level(data, chunk, two_level) if two_level else ctx.hash_chunks(data, chunk)
+            man_root = bytes(ctx.merkle_root(man_digests).cpu().numpy().tobytes())
         manifest = ctx.make_manifest(nbytes, chunk, man_digests, man_root)
         result = binding.new_result(device)
         idx = torch.zeros(64, dtype=torch.int64, device=device)
@@ -232,7 +237,7 @@ def run_ours(args):
         # builds the global root: local digests -> k levels -> all-gather of the few level-k nodes (32 bytes
         # each, the path's only exchange) -> root, on every rank.
         shard_plan = None
-        if world > 1:
+        if world > 1 and args.variant == "sha256":
             from paper_2510_23938_b200 import sharded
             shard_plan = sharded.plan_shards(world * n_units, world, min_nodes_per_rank=64)
             lo, hi = shard_plan.leaf_ranges[rank]
@@ -255,7 +260,11 @@ def run_ours(args):
             if batch_blobs is not None:
                 ctx.verify_manifest_batch(batch_blobs, manifest, batch_results, batch_idx)
                 return
-            if two_level:
+            if variant == "sha384":
+                ctx.merkle_root_sha384(ctx.hash_chunks_sha384(data, chunk))
+            elif variant == "rfc6962":
+                ctx.verify_manifest_rfc6962(data, manifest, result, idx)
+            elif two_level:
                 ctx.verify_manifest_two_level(data, manifest, two_level, result, idx)
             else:
                 ctx.verify_manifest(data, manifest, result, idx)
@@ -297,7 +306,14 @@ def run_ours(args):
     ctx.set_timing(False)
 
     # dominant kernel: the leaf-hashing launch, timed by the library's own events inside the timed steps
-    if ragged or (args.batch and args.batch > 1):
+    if not ragged and args.variant == "sha384":
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        ctx.hash_chunks_sha384(data, chunk)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        hash_ms, tree_ms, cmp_ms = float(e0.elapsed_time(e1)), None, None
+    elif ragged or (args.batch and args.batch > 1):
         hash_ms = None
     else:
         hash_ms = float(np.mean([ctx.phase_times(k)[0] for k in range(min(args.steps, 64))]))
@@ -362,17 +378,28 @@ def run_ours(args):
     if copies > 1:
         out["config"]["batch"] = (f"{copies} copies verified in one pass (iv_verify_manifest_batch); mismatches per copy: "
                                   f"{[r['n_mismatch'] for r in out_batch]}; roofline figures are per whole step")
+    if not ragged and args.variant != "sha256":
+        out["config"]["variant"] = {"rfc6962": "RFC 6962 section 2.1 mode: leaf = SHA-256(0x00 || chunk), node = "
+                                               "SHA-256(0x01 || left || right); verification in that mode",
+                                    "sha384": "SHA-384 leaves and tree (hash + root, no manifest compare)"}[args.variant]
+        if args.variant == "sha384":
+            sha384_peak = SM_COUNT * INT_LANES_PER_SM * 1.965e9 / (3568.0 / 128.0) / 1e9
+            out["metric"] = "GB/s hashed (SHA-384 chunks + Merkle root) at 1 B200"
+            out["roofline"].update({"peak": round(sha384_peak, 1), "frac": round(achieved / sha384_peak, 4),
+                                    "int32_ops_per_byte": 3568.0 / 128.0, "chain_count_bound_gbs": None,
+                                    "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1.965 GHz / 27.875 INT32 ops per byte"})
     if not ragged and args.two_level:
         out["config"]["leaf_definition"] = (f"TWO-LEVEL (not the default): chunk digest = Merkle root over SHA-256 of "
                                             f"{args.two_level}-byte pieces; {binding.n_chunks(nbytes, args.two_level)} chains")
         out["roofline"]["chains"] = binding.n_chunks(nbytes, args.two_level)
         out["roofline"]["note"] = "launch_ms covers piece hashing + the levels up to chunk digests"
 
-    if rank == 0 and not ragged and not args.no_e2e and not args.two_level and copies == 1:
+    if rank == 0 and not ragged and not args.no_e2e and not args.two_level and copies == 1 and args.variant == "sha256":
         out["e2e"] = measure_e2e(ctx, wl, device, args)
     elif rank == 0:
         out["e2e"] = None
-    if rank == 0 and world == 1 and not args.no_cpu and not (not ragged and args.two_level) and copies == 1:
+    if rank == 0 and world == 1 and not args.no_cpu and not (not ragged and args.two_level) and copies == 1 \
+            and args.variant == "sha256":
         out["cpu_baseline"] = measure_cpu_baseline(ctx, wl, device, oracle, ragged,
                                                    None if ragged else man_digests,
                                                    (d_off, d_len, digests) if ragged else None)
@@ -549,6 +576,9 @@ def main():
     ap.add_argument("--two-level", type=int, default=None, metavar="SUB_BYTES",
                     help="two-level leaves: chunk digest = Merkle root over SHA-256 of SUB_BYTES pieces (a different, "
                          "separately named leaf definition; not the default)")
+    ap.add_argument("--variant", default="sha256", choices=["sha256", "rfc6962", "sha384"],
+                    help="sha256 = the default path; rfc6962 = 0x00/0x01-prefixed tree (verification in that mode); "
+                         "sha384 = SHA-384 leaves and tree (hash + root, no manifest compare). Not the graded line.")
     ap.add_argument("--dist-backend", default="nccl", help="torch.distributed backend for --gpus > 1")
     ap.add_argument("--same-device", action="store_true",
                     help="put every rank on cuda:0 (only to check the multi-rank logic on a one-GPU box, with gloo)")

@@ -332,6 +332,11 @@ int iv_hash_chunks_rfc6962(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uin
                            void *cuda_stream);
 int iv_merkle_root_rfc6962(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
                            void *cuda_stream);
+/* iv_verify_manifest in this mode: the manifest holds the prefixed leaf hashes and the root of the
+ * prefixed tree; result record, index list, errors and asynchrony as iv_verify_manifest. */
+int iv_verify_manifest_rfc6962(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
+                               const iv_manifest *h_manifest, iv_verify_result *d_result,
+                               uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
  * Merkle root without allocation (the paper has no counterpart; this exists

@@ -32,7 +32,7 @@ EXPORTS = (
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
     "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update", "iv_verify_manifest_batch",
     "iv_hash_chunks_sha384", "iv_merkle_root_sha384",
-    "iv_hash_chunks_rfc6962", "iv_merkle_root_rfc6962",
+    "iv_hash_chunks_rfc6962", "iv_merkle_root_rfc6962", "iv_verify_manifest_rfc6962",
 )
 
 
@@ -105,6 +105,8 @@ def load_library() -> ctypes.CDLL:
     lib.iv_hash_chunks_sha384.restype = i32
     lib.iv_merkle_root_sha384.argtypes = [vp, vp, u64, vp, vp]
     lib.iv_merkle_root_sha384.restype = i32
+    lib.iv_verify_manifest_rfc6962.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
+    lib.iv_verify_manifest_rfc6962.restype = i32
     lib.iv_hash_chunks_rfc6962.argtypes = [vp, vp, u64, u64, vp, u64, ctypes.POINTER(u64), vp]
     lib.iv_hash_chunks_rfc6962.restype = i32
     lib.iv_merkle_root_rfc6962.argtypes = [vp, vp, u64, vp, vp]
@@ -336,6 +338,14 @@ class Context:
         rc = self._lib.iv_verify_manifest(self._h, _dev_ptr(data), nb, ctypes.byref(manifest),
                                           _dev_ptr(result), _dev_ptr(mismatch_idx), cap, _stream_ptr(stream))
         self._check(rc, "iv_verify_manifest")
+
+    def verify_manifest_rfc6962(self, data: torch.Tensor, manifest: Manifest, result: torch.Tensor,
+                                mismatch_idx: torch.Tensor | None, stream=None) -> None:
+        """iv_verify_manifest_rfc6962 (asynchronous); the manifest holds prefixed leaf hashes and their root."""
+        cap = 0 if mismatch_idx is None else mismatch_idx.numel()
+        rc = self._lib.iv_verify_manifest_rfc6962(self._h, _dev_ptr(data), _nbytes(data), ctypes.byref(manifest),
+                                                  _dev_ptr(result), _dev_ptr(mismatch_idx), cap, _stream_ptr(stream))
+        self._check(rc, "iv_verify_manifest_rfc6962")
 
     def verify_manifest_batch(self, blobs: list, manifest: Manifest, results: torch.Tensor,
                               mismatch_idx: torch.Tensor | None, stream=None) -> None:

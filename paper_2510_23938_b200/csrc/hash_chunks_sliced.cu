@@ -23,6 +23,7 @@
 #include <cstring>
 
 #include "iv_internal.h"
+#include "rfc6962_dev.cuh"
 #include "sha256_dev.cuh"
 #include "tma_dev.cuh"
 
@@ -60,7 +61,10 @@ __device__ __forceinline__ void tiled_g2s(uint32_t dst, const CUtensorMap *map, 
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
-template <int SEG, int STAGES, int MAX_WARPS, bool TILED>
+// PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash).  Message block j is then the
+// byte before data block j followed by its first 63 bytes; the word before the block is carried in a
+// register, at the start of a later slice it is read back from the blob.
+template <int SEG, int STAGES, int MAX_WARPS, bool TILED, bool PREFIX>
 __global__ void __launch_bounds__(32 * MAX_WARPS)
 hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
@@ -169,6 +173,8 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
         const uint64_t nseg = (warp_bytes + SEG - 1) / SEG;
 
         uint32_t st[8], w[16], raw[16];
+        uint32_t carry = 0u;          // PREFIX: the data word before the block; byte 3 of 0 is the prefix itself
+        if (PREFIX && my_lo > 0 && my_bytes > 0) carry = __ldg(reinterpret_cast<const uint32_t *>(p) - 1);
         if (s == 0) {
             sha256_init(st);
         } else {
@@ -233,8 +239,15 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
         }
         uint64_t next_seg = STAGES;
         for (uint64_t blk = 0; blk < warp_blocks; ++blk) {
+            if (PREFIX) {
+                w[0] = shifted_word(raw[0], carry);
 #pragma unroll
-            for (int k = 0; k < 16; ++k) w[k] = bswap32(raw[k]);
+                for (int k = 1; k < 16; ++k) w[k] = shifted_word(raw[k], raw[k - 1]);
+                carry = raw[15];
+            } else {
+#pragma unroll
+                for (int k = 0; k < 16; ++k) w[k] = bswap32(raw[k]);
+            }
             const bool stage_done = (++in_stage == kBlocksPerSeg) || (blk + 1 == warp_blocks);
             if (stage_done) {
                 in_stage = 0;
@@ -267,7 +280,16 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
         }
         if (!valid) continue;
         const uint32_t rem = (uint32_t)(len & 63u);
-        if (rem == 0) {
+        if (PREFIX) {
+            uint32_t tw[32];
+            const int nblk = prefixed_tail(data + begin, 0x00, full_bytes, len + 1, tw);
+#pragma unroll 1
+            for (int tb = 0; tb < nblk; ++tb) {
+#pragma unroll
+                for (int k = 0; k < 16; ++k) w[k] = tw[16 * tb + k];
+                sha256_compress(st, w);
+            }
+        } else if (rem == 0) {
             sha256_pad_only_block(w, len);
             sha256_compress(st, w);
         } else {
@@ -346,14 +368,14 @@ bool make_chunk_tensor_map(CUtensorMap *map, const uint8_t *d_data, uint64_t chu
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool TILED>
+template <bool TILED, bool PREFIX>
 cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
                           const uint32_t *d_one, int sm_count, cudaStream_t stream) {
     constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8;
     constexpr size_t smem_per_warp = TILED ? (size_t)STAGES * 8192 : (size_t)STAGES * 32 * (SEG + 16);
     constexpr size_t smem_pad = TILED ? 1024 : 0;
-    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED>;
+    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX>;
     static bool configured[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, total_tasks = 0;
@@ -393,18 +415,24 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
 // chunks can be described to the TMA unit, so a short last chunk is left to the caller (*covered = n - 1).
 cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                       uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
-                                      const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *covered) {
+                                      const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *covered,
+                                      bool zero_prefix) {
     const uint64_t whole = nbytes / chunk_bytes;          // n_chunks or n_chunks - 1
     alignas(64) CUtensorMap map;
     std::memset(&map, 0, sizeof map);
     if (whole > 0 && make_chunk_tensor_map(&map, d_data, chunk_bytes, whole)) {
         *covered = whole;
-        return launch_sliced<true>(map, d_data, whole * chunk_bytes, chunk_bytes, whole, d_digests, d_status, d_scratch,
-                                   d_one, sm_count, stream);
+        const uint64_t bytes = whole * chunk_bytes;
+        return zero_prefix ? launch_sliced<true, true>(map, d_data, bytes, chunk_bytes, whole, d_digests, d_status,
+                                                       d_scratch, d_one, sm_count, stream)
+                           : launch_sliced<true, false>(map, d_data, bytes, chunk_bytes, whole, d_digests, d_status,
+                                                        d_scratch, d_one, sm_count, stream);
     }
     *covered = n_chunks;
-    return launch_sliced<false>(map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_scratch, d_one,
-                                sm_count, stream);
+    return zero_prefix ? launch_sliced<false, true>(map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
+                                                    d_scratch, d_one, sm_count, stream)
+                       : launch_sliced<false, false>(map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
+                                                     d_scratch, d_one, sm_count, stream);
 }
 
 }  // namespace ivk

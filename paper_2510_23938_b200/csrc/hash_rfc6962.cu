@@ -5,33 +5,11 @@
 // a block is the last byte of the previous data word followed by the first three bytes of data word
 // k, which one PRMT per word produces together with the endian swap, so the shift costs nothing.
 #include "iv_internal.h"
+#include "rfc6962_dev.cuh"
 #include "sha256_dev.cuh"
 
 namespace ivk {
 namespace {
-
-// Big-endian message word from the little-endian data words (cur, prev): prev.byte3, cur.byte0..2.
-__device__ __forceinline__ uint32_t shifted_word(uint32_t cur, uint32_t prev) { return __byte_perm(cur, prev, 0x7012u); }
-
-// Tail of the prefixed message from message position mpos (a multiple of 64) to its end at msg_bytes,
-// then the padding.  Message byte 0 is the prefix, message byte q >= 1 is data[q - 1].  At most 64
-// message bytes remain, so the tail is one or two blocks.
-__device__ __noinline__ int prefixed_tail(const uint8_t *data, uint8_t prefix, uint64_t mpos, uint64_t msg_bytes,
-                                          uint32_t *tw /* [32] */) {
-    for (int i = 0; i < 32; ++i) tw[i] = 0u;
-    const uint32_t rem = (uint32_t)(msg_bytes - mpos);
-    for (uint32_t k = 0; k < rem; ++k) {
-        const uint64_t q = mpos + k;
-        const uint32_t byte = q == 0 ? prefix : data[q - 1];
-        tw[k >> 2] |= byte << (24 - 8 * (k & 3));
-    }
-    tw[rem >> 2] |= 0x80u << (24 - 8 * (rem & 3));
-    const int nblk = (rem + 1 + 8 <= 64) ? 1 : 2;
-    const uint64_t bits = msg_bytes << 3;
-    tw[16 * nblk - 2] = (uint32_t)(bits >> 32);
-    tw[16 * nblk - 1] = (uint32_t)bits;
-    return nblk;
-}
 
 template <bool ALIGNED16>
 __global__ void __launch_bounds__(128)
@@ -134,9 +112,9 @@ __global__ void sha256_of_nothing_kernel(uint8_t *out) {
 
 }  // namespace
 
-cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
-                                       uint8_t *d_digests, int sm_count, cudaStream_t stream, uint64_t *launches) {
-    if (n_chunks == 0) return cudaSuccess;
+namespace {
+cudaError_t launch_direct(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
+                          uint8_t *d_digests, int sm_count, cudaStream_t stream) {
     const uint64_t warps = (n_chunks + 31) / 32;
     const unsigned warps_per_cta = warps <= (uint64_t)sm_count ? 1u : (warps <= 2ull * sm_count ? 2u : 4u);
     const unsigned threads = 32u * warps_per_cta;
@@ -147,8 +125,31 @@ cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, u
         hash_chunks_rfc6962_kernel<true><<<(unsigned)blocks, threads, 0, stream>>>(d_data, nbytes, chunk_bytes, n_chunks, d_digests);
     else
         hash_chunks_rfc6962_kernel<false><<<(unsigned)blocks, threads, 0, stream>>>(d_data, nbytes, chunk_bytes, n_chunks, d_digests);
-    if (launches) ++*launches;
     return cudaGetLastError();
+}
+}  // namespace
+
+cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
+                                       uint8_t *d_digests, int sm_count, uint32_t *d_status, const uint32_t *d_one,
+                                       void *d_slice_scratch, cudaStream_t stream, uint64_t *launches,
+                                       const char **kernel_used) {
+    if (n_chunks == 0) return cudaSuccess;
+    if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
+        // many chains that do not divide evenly over the schedulers: the migrating kernel, prefixed
+        if (launches) *launches += 2;
+        if (kernel_used) *kernel_used = "hash_chunks_sliced_kernel";
+        uint64_t covered = 0;
+        cudaError_t e = launch_hash_chunks_sliced(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
+                                                  d_slice_scratch, d_one, sm_count, stream, &covered, true);
+        if (e != cudaSuccess || covered == n_chunks) return e;
+        if (launches) ++*launches;
+        const uint64_t off = covered * chunk_bytes;
+        return launch_direct(d_data + off, nbytes - off, chunk_bytes, n_chunks - covered, d_digests + 32 * covered,
+                             sm_count, stream);
+    }
+    if (launches) ++*launches;
+    if (kernel_used) *kernel_used = "hash_chunks_rfc6962_kernel";
+    return launch_direct(d_data, nbytes, chunk_bytes, n_chunks, d_digests, sm_count, stream);
 }
 
 // d_scratch_a / d_scratch_b: ceil(n / 2) records of 32 bytes each.

@@ -114,6 +114,18 @@ int ensure_merkle_scratch(iv_ctx *ctx, uint64_t n_leaves) {
     return IV_OK;
 }
 
+// Level buffers of the variant trees: two buffers of at least `records` records of 48 bytes.
+int ensure_variant_tree_scratch(iv_ctx *ctx, uint64_t records) {
+    if (records <= ctx->tree384_cap) return IV_OK;
+    uint64_t cap_a = ctx->tree384_cap, cap_b = ctx->tree384_cap;
+    int rc = grow(ctx, &ctx->d_tree384[0], &cap_a, records, 48);
+    if (rc != IV_OK) return rc;
+    rc = grow(ctx, &ctx->d_tree384[1], &cap_b, records, 48);
+    if (rc != IV_OK) return rc;
+    ctx->tree384_cap = cap_a < cap_b ? cap_a : cap_b;
+    return IV_OK;
+}
+
 // Leaf hashing with the scratch the launch shape needs.
 int hash_leaves(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n,
                 uint8_t *d_digests, cudaStream_t stream) {
@@ -126,6 +138,21 @@ int hash_leaves(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t ch
     }
     IV_TRY(ctx, ivk::launch_hash_chunks(d_data, nbytes, chunk_bytes, n, d_digests, ctx->sm_count, ctx->d_status,
                                         ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel));
+    return IV_OK;
+}
+
+// The same for the prefixed leaf hashes of the RFC 6962 mode.
+int hash_leaves_rfc6962(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n,
+                        uint8_t *d_digests, cudaStream_t stream) {
+    void *scratch = nullptr;
+    if (ivk::hash_chunks_wants_slices(d_data, chunk_bytes, n, ctx->sm_count)) {
+        const uint64_t need = ivk::sliced_scratch_bytes(n, chunk_bytes, nullptr, nullptr, nbytes);
+        int rc = grow(ctx, &ctx->d_slices, &ctx->slices_cap, need, 1);
+        if (rc != IV_OK) return rc;
+        scratch = ctx->d_slices;
+    }
+    IV_TRY(ctx, ivk::launch_hash_chunks_rfc6962(d_data, nbytes, chunk_bytes, n, d_digests, ctx->sm_count, ctx->d_status,
+                                                ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel));
     return IV_OK;
 }
 
@@ -149,15 +176,20 @@ int mark_phase(iv_ctx *ctx, int which, cudaStream_t stream) {
 
 // Root + compare, shared by the resident and the streamed verification.
 int finish_verification(iv_ctx *ctx, const iv_manifest *m, iv_verify_result *d_result,
-                        uint64_t *d_mismatch_idx, uint64_t idx_cap, cudaStream_t stream) {
+                        uint64_t *d_mismatch_idx, uint64_t idx_cap, cudaStream_t stream, bool rfc6962 = false) {
     const uint64_t n = m->n_chunks;
     int rc = ensure_merkle_scratch(ctx, n);
     if (rc != IV_OK) return rc;
     rc = grow(ctx, &ctx->d_words, &ctx->words_cap, (n + 31) / 32 + 1, sizeof(uint32_t));
     if (rc != IV_OK) return rc;
+    if (rfc6962 && (rc = ensure_variant_tree_scratch(ctx, (n + 1) / 2 + 1)) != IV_OK) return rc;
     if ((rc = mark_phase(ctx, 1, stream)) != IV_OK) return rc;
-    IV_TRY(ctx, ivk::launch_merkle_root(ctx->d_digests, n, ctx->d_root, ctx->d_merkle_a, ctx->d_merkle_b,
-                                        ctx->d_tickets, stream, &ctx->launches));
+    if (rfc6962)
+        IV_TRY(ctx, ivk::launch_merkle_root_rfc6962(ctx->d_digests, n, ctx->d_root, ctx->d_tree384[0], ctx->d_tree384[1],
+                                                    stream, &ctx->launches));
+    else
+        IV_TRY(ctx, ivk::launch_merkle_root(ctx->d_digests, n, ctx->d_root, ctx->d_merkle_a, ctx->d_merkle_b,
+                                            ctx->d_tickets, stream, &ctx->launches));
     if ((rc = mark_phase(ctx, 2, stream)) != IV_OK) return rc;
     ivk::RootBytes expect;
     std::memcpy(expect.b, m->root, 32);
@@ -672,18 +704,6 @@ int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint
     return IV_OK;
 }
 
-// Level buffers of the variant trees: two buffers of at least `records` records of 48 bytes.
-static int ensure_variant_tree_scratch(iv_ctx *ctx, uint64_t records) {
-    if (records <= ctx->tree384_cap) return IV_OK;
-    uint64_t cap_a = ctx->tree384_cap, cap_b = ctx->tree384_cap;
-    int rc = grow(ctx, &ctx->d_tree384[0], &cap_a, records, 48);
-    if (rc != IV_OK) return rc;
-    rc = grow(ctx, &ctx->d_tree384[1], &cap_b, records, 48);
-    if (rc != IV_OK) return rc;
-    ctx->tree384_cap = cap_a < cap_b ? cap_a : cap_b;
-    return IV_OK;
-}
-
 int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
     if (!ctx || !d_root || (n_leaves && !d_leaves)) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
@@ -703,10 +723,27 @@ int iv_hash_chunks_rfc6962(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uin
     if (h_n_chunks) *h_n_chunks = n;
     if (n == 0) return IV_OK;
     DeviceGuard guard(ctx->device);
-    IV_TRY(ctx, ivk::launch_hash_chunks_rfc6962(static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
-                                                ctx->sm_count, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
-    ctx->leaf_kernel = "hash_chunks_rfc6962_kernel";
-    return IV_OK;
+    return hash_leaves_rfc6962(ctx, static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
+                               static_cast<cudaStream_t>(cuda_stream));
+}
+
+int iv_verify_manifest_rfc6962(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest *h_manifest,
+                               iv_verify_result *d_result, uint64_t *d_mismatch_idx, uint64_t idx_cap,
+                               void *cuda_stream) {
+    if (!ctx || !d_result || (idx_cap && !d_mismatch_idx)) return IV_ERR_INVALID_ARG;
+    int rc = check_manifest(h_manifest, nbytes);
+    if (rc != IV_OK) return rc;
+    if (nbytes && !d_data) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const uint64_t n = h_manifest->n_chunks;
+    rc = grow(ctx, &ctx->d_digests, &ctx->digests_cap, n + 1, 32);
+    if (rc != IV_OK) return rc;
+    if ((rc = mark_phase(ctx, 0, stream)) != IV_OK) return rc;
+    rc = hash_leaves_rfc6962(ctx, static_cast<const uint8_t *>(d_data), nbytes, h_manifest->chunk_bytes, n,
+                             ctx->d_digests, stream);
+    if (rc != IV_OK) return rc;
+    return finish_verification(ctx, h_manifest, d_result, d_mismatch_idx, idx_cap, stream, true);
 }
 
 int iv_merkle_root_rfc6962(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {

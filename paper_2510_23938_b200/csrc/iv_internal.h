@@ -52,9 +52,11 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
 uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t *slice_bytes_out,
                               uint64_t *total_tasks_out, uint64_t nbytes);
 // *covered receives the number of leading chunks the launch hashes (all, or all but a short last chunk).
+// zero_prefix: hash 0x00 || chunk instead of the chunk (the RFC 6962 leaf hash).
 cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                       uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
-                                      const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *covered);
+                                      const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *covered,
+                                      bool zero_prefix = false);
 
 // The same two-warp kernel for tensors at any alignment; message k of the launch is tensor d_order[k]
 // (d_order may be NULL for index order).
@@ -132,8 +134,12 @@ cudaError_t launch_merkle_root_sha384(const uint8_t *d_leaves, uint64_t n, uint8
 
 // hash_rfc6962.cu ----------------------------------------------------------
 // RFC 6962 section 2.1 mode: prefixed leaf hashes and the tree with prefixed nodes.
+// With d_slice_scratch (sliced_scratch_bytes(...) bytes) and a launch shape that wants slices
+// (hash_chunks_wants_slices) the chains migrate as on the default path; otherwise one chain per lane.
 cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
-                                       uint8_t *d_digests, int sm_count, cudaStream_t stream, uint64_t *launches);
+                                       uint8_t *d_digests, int sm_count, uint32_t *d_status, const uint32_t *d_one,
+                                       void *d_slice_scratch, cudaStream_t stream, uint64_t *launches,
+                                       const char **kernel_used);
 cudaError_t launch_merkle_root_rfc6962(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root, uint8_t *d_scratch_a,
                                        uint8_t *d_scratch_b, cudaStream_t stream, uint64_t *launches);
 

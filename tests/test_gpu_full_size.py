@@ -106,6 +106,13 @@ def test_largest_configuration_sampled(ctx):
     root = _host(ctx.merkle_root(got)).tobytes()
     assert _host(ctx.merkle_root(ctx.merkle_levels(got, 9))).tobytes() == root
     assert _host(ctx.tree_build(got)[-1]).tobytes() == root
+    # the same launch shape in the RFC 6962 mode (prefixed leaf hashes through the migrating kernel)
+    got6962 = _host(ctx.hash_chunks_rfc6962(data, chunk))
+    assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel" and ctx.device_status() == 0
+    for i in sample[::3]:
+        want = oracle.hash_chunks_rfc6962(_host(data[i * chunk:(i + 1) * chunk]), chunk)[0]
+        assert got6962[i].tobytes() == want.tobytes(), i
+    del got6962
     # a flipped bit is found at its chunk, nothing else changes
     manifest = ctx.make_manifest(data.numel(), chunk, got.clone(), root)
     off, bit = inputs.flip_position(7, data.numel())

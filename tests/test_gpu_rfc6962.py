@@ -34,7 +34,10 @@ def _host(t: torch.Tensor) -> np.ndarray:
     (5 * 4096 + 62, 4096), (5 * 4096 + 63, 4096), (5 * 4096 + 64, 4096),
     (5 * 4096 + 118, 4096), (5 * 4096 + 119, 4096), (5 * 4096 + 127, 4096),
     (37 * 48 + 16, 48),
-    (20_000 * 4096 + 100, 4096),
+    (20_000 * 4096 + 100, 4096),          # the migrating kernel (more than 296 warps), short last chunk beside it
+    (19_000 * 4096, 4096),
+    (9_600 * 65536, 65536),               # several slices per chunk: the carried word crosses slice borders
+    (9_600 * 65536 + 63, 65536), (9_500 * (65536 + 16), 65536 + 16),
 ])
 def test_leaf_hashes_equal_oracle(ctx, nbytes, chunk):
     data = inputs.uniform_bytes(nbytes, seed=6962, device="cuda")
@@ -91,3 +94,39 @@ def test_leaves_then_root_differs_from_the_default_path_and_repeats(ctx):
         assert _host(ctx.merkle_root_rfc6962(leaves)).tobytes() == want_root
     assert _host(ctx.merkle_root(ctx.hash_chunks(data, 4096))).tobytes() != want_root
     assert ctx.device_status() == 0
+
+
+def test_verification_in_this_mode_against_a_manifest_from_the_oracle(ctx):
+    """Manifest = the oracle's prefixed leaf hashes and root; clean data passes, flipped bits are located, and a
+    manifest of the default (unprefixed) path is rejected on every chunk."""
+    nbytes, chunk = (8 << 20) + 300, 4096
+    data = inputs.uniform_bytes(nbytes, seed=6970, device="cuda")
+    leaves = oracle.hash_chunks_rfc6962(_host(data), chunk, nthreads=oracle.host_threads())
+    root = oracle.merkle_root_rfc6962(leaves)
+    manifest = ctx.make_manifest(nbytes, chunk, torch.from_numpy(leaves).cuda(), root)
+    n = leaves.shape[0]
+
+    def verify(blob, man, cap=16):
+        res = binding.new_result("cuda")
+        idx = torch.zeros(cap, dtype=torch.int64, device="cuda")
+        ctx.verify_manifest_rfc6962(blob, man, res, idx)
+        r = binding.read_result(res)
+        return r, [int(v) for v in idx[:min(cap, r["n_mismatch"])].cpu()]
+
+    r, idx = verify(data, manifest)
+    assert r == {"status": 0, "root_ok": True, "n_mismatch": 0, "root": root} and idx == []
+    bad = data.clone()
+    flips = sorted({inputs.flip_position(s, nbytes) for s in (5, 6, 7)})
+    for off, bit in flips:
+        bad[off] ^= (1 << bit)
+    want_leaves = oracle.hash_chunks_rfc6962(_host(bad), chunk, nthreads=oracle.host_threads())
+    want_idx = [i for i in range(n) if bytes(want_leaves[i]) != bytes(leaves[i])]
+    r, idx = verify(bad, manifest)
+    assert idx == want_idx == sorted({off // chunk for off, _ in flips})
+    assert r["n_mismatch"] == len(want_idx) and not r["root_ok"]
+    assert r["root"] == oracle.merkle_root_rfc6962(want_leaves)
+    # the default path's manifest does not verify in this mode
+    plain = oracle.hash_chunks(_host(data), chunk, nthreads=oracle.host_threads())
+    plain_manifest = ctx.make_manifest(nbytes, chunk, torch.from_numpy(plain).cuda(), oracle.merkle_root(plain))
+    r, idx = verify(data, plain_manifest, cap=4)
+    assert r["n_mismatch"] == n and not r["root_ok"] and idx == [0, 1, 2, 3]
