@@ -404,7 +404,10 @@ typedef enum iv_probe_kind {
     IV_PROBE_SHA256_ADD2 = 20, /* kinds 20..22: full compressions with the additions placed as the */
     IV_PROBE_SHA256_ADD3 = 21, /* library's addition placements 2, 3 and 4                          */
     IV_PROBE_SHA256_ADD4 = 22,
-    IV_PROBE_ROUNDS_M3_HANDSHAKE = 23 /* kind 16 plus the consumer's per-block hand-over (barrier wait, arrival, feed-forward) */
+    IV_PROBE_ROUNDS_M3_HANDSHAKE = 23, /* kind 16 plus the consumer's per-block hand-over (barrier wait, arrival, feed-forward) */
+    IV_PROBE_SHA256_STREAM = 24, /* full compressions of a message that does not depend on the chaining value */
+    IV_PROBE_SHA256_ADD6 = 25,   /* full compressions, the schedule's plain shifts as multiply-high (FMA pipe) */
+    IV_PROBE_SHA256_ADD7 = 26    /* full compressions, the schedule's shifts and rotations as multiply-adds (FMA pipe) */
 } iv_probe_kind;
 int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t blocks_per_sm,
                  uint32_t active_lanes, uint32_t iters, double *h_out);

@@ -411,7 +411,8 @@ class Context:
     PROBE_KINDS = {"iadd3": 0, "lop3": 1, "shf": 2, "prmt": 3, "imad": 4, "mixed": 5, "sha256": 6, "sha256_fma": 7,
                    "lat_iadd3": 8, "lat_lop3": 9, "lat_shf": 10, "lat_imad": 11, "lat_cross": 12,
                    "rounds_m0": 13, "rounds_m1": 14, "rounds_m2": 15, "rounds_m3": 16, "schedule": 17, "rounds_m4": 18, "rounds_m5": 19,
-                   "sha256_add2": 20, "sha256_add3": 21, "sha256_add4": 22, "rounds_m3_handshake": 23}
+                   "sha256_add2": 20, "sha256_add3": 21, "sha256_add4": 22, "rounds_m3_handshake": 23,
+                   "sha256_stream": 24, "sha256_add6": 25, "sha256_add7": 26}
 
     def probe_alu(self, kind: str, warps_per_block: int = 4, blocks_per_sm: int = 1, active_lanes: int = 32,
                   iters: int = 2000) -> tuple[float, float]:

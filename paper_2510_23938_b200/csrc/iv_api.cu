@@ -761,7 +761,7 @@ int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t block
     if (!ctx || !h_out || warps_per_block == 0 || warps_per_block > 32 || blocks_per_sm == 0 ||
         blocks_per_sm > 32 || active_lanes == 0 || active_lanes > 32 || iters == 0)
         return IV_ERR_INVALID_ARG;
-    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_ROUNDS_M3_HANDSHAKE) return IV_ERR_INVALID_ARG;
+    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_SHA256_ADD7) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     const unsigned blocks = blocks_per_sm * (unsigned)ctx->sm_count;
     unsigned long long *d_cycles = nullptr;

@@ -96,6 +96,33 @@ __global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, unsigned
     if (threadIdx.x == 0) cycles[blockIdx.x] = (unsigned long long)(t1 - t0);
 }
 
+// Register-only SHA-256 over a message that does not depend on the chaining value (as data from
+// memory does not), so the schedule of one block is free to overlap the rounds of the one before.
+__global__ void probe_sha_stream_kernel(uint32_t iters, uint32_t active_lanes, unsigned long long *cycles, uint32_t *sink) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t mul = sink[1] * 0x9e3779b9u;       // the host stored 1 in sink[1]
+    uint32_t st[8];
+    sha256_init(st);
+    st[0] ^= threadIdx.x + blockIdx.x * blockDim.x;
+    __syncthreads();
+    const long long t0 = clock64();
+    if (lane < active_lanes) {
+        uint32_t w[16];
+        uint32_t x = threadIdx.x;
+#pragma unroll 1
+        for (uint32_t it = 0; it < iters; ++it) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) w[i] = bswap32(x + (uint32_t)i * mul);
+            x += mul;
+            sha256_compress<0>(st, w, 1u);
+        }
+    }
+    __syncthreads();
+    const long long t1 = clock64();
+    if ((st[0] ^ st[5]) == 0x12345u) sink[0] = st[1];
+    if (threadIdx.x == 0) cycles[blockIdx.x] = (unsigned long long)(t1 - t0);
+}
+
 // The consumer half alone: 64 rounds per trip, W + K read from a (constant) shared-memory slot.
 // HANDSHAKE adds what the split kernel's consumer does around the rounds: a wait on a "full"
 // barrier (completed just before by lane 0 itself), the warp barrier, the "empty" arrival and the
@@ -199,6 +226,9 @@ cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t i
         case IV_PROBE_SHA256_ADD2: probe_sha_kernel<2><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_SHA256_ADD3: probe_sha_kernel<3><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_SHA256_ADD4: probe_sha_kernel<4><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_ADD6: probe_sha_kernel<6><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_ADD7: probe_sha_kernel<7><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_STREAM: probe_sha_stream_kernel<<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
