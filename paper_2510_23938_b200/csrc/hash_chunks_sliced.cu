@@ -10,6 +10,13 @@
 // the FIFO at most once, its slices run in order; a warp never waits while it holds a task, so
 // the scheme needs no co-residency and cannot deadlock.  All waits are bounded.
 //
+// Service order.  A scheduler that runs two groups completes about 1.13 groups in the time a
+// scheduler with one group completes one, so between 592 and 1,184 groups the best fill has one
+// group on every scheduler and the surplus spread as second groups.  The launcher can therefore
+// ask for "first workers first": warps 0..3 of a CTA (one per scheduler) take tickets as they
+// come, warps 4..7 take a task only when one lies in the FIFO unclaimed.  The schedulers left
+// with one group finish early and then take over what remains of the others.
+//
 // Data movement, TILED = false: the staged kernel's per-lane bulk copies (TMA, 1-D) into a
 // lane-interleaved shared-memory ring.  TILED = true: the blob is described to the TMA unit as a
 // 2-D tensor [chunk][byte] with the chunk size as row pitch, and ONE tiled copy of a 32-row x
