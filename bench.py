@@ -472,7 +472,18 @@ def measure_e2e(ctx, wl, device, args):
     e1.record(stream)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
+    # what the host link alone delivers: one pinned window copied to the device, nothing else running
+    dst = torch.empty(ring[0].numel(), dtype=torch.uint8, device=device)
+    dst.copy_(ring[0], non_blocking=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    dst.copy_(ring[0], non_blocking=True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    link_gbs = ring[0].numel() / (e0.elapsed_time(e1) * 1e-3) / 1e9
+    del dst
     return {"value": round(e_nbytes / (ms * 1e-3) / 1e9, 3), "unit": "GB/s", "ms_per_step": round(ms, 3),
+            "h2d_copy_alone_gbs": round(link_gbs, 2),
             "steps": steps, "h2d_bytes_per_step": int(e_nbytes), "d2h_bytes_per_step": 48,
             "api": "iv_verify_streamed, pinned host windows of %d MiB, two device windows" % (window // MIB),
             "host_ring_windows": r, "periodic_blob": periodic, "verified_ok": bool(ok)}
