@@ -62,23 +62,45 @@ __device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
+// A scheduler's second worker takes a task only when one lies in the FIFO unclaimed: the first
+// workers (one per scheduler) are served first, so no scheduler idles while another runs two
+// groups.  With nothing left over it polls; giving up (the return value total_tasks ends the
+// worker) is harmless, the first workers finish the launch.  Kept out of line so that the hashing
+// loop's register allocation does not depend on it.
+__device__ __noinline__ unsigned long long take_leftover_ticket(SliceQueue *q, unsigned long long total_tasks,
+                                                                bool first_take) {
+    if (first_take) __nanosleep(20000);      // at launch, let the first workers of every CTA claim their groups
+    const long long t0 = clock64();
+    for (;;) {
+        const unsigned long long h = *reinterpret_cast<volatile unsigned long long *>(&q->head);
+        if (h >= total_tasks) return total_tasks;
+        const unsigned long long tl = *reinterpret_cast<volatile unsigned long long *>(&q->tail);
+        if (tl > h) {
+            if (atomicCAS(&q->head, h, h + 1ull) == h) return h;
+            continue;
+        }
+        if (clock64() - t0 > 8000000000ll) return total_tasks;
+        __nanosleep(256);
+    }
+}
+
 __device__ __forceinline__ void tiled_g2s(uint32_t dst, const CUtensorMap *map, uint32_t x, uint32_t y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
+// FWF ("first workers first"): warps 4..7 take only left-over tasks, see the service order above.
 // PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash).  Message block j is then the
 // byte before data block j followed by its first 63 bytes; the word before the block is carried in a
 // register, at the start of a later slice it is read back from the blob.
-template <int SEG, int STAGES, int MAX_WARPS, bool TILED, bool PREFIX>
+template <int SEG, int STAGES, int MAX_WARPS, bool TILED, bool PREFIX, bool FWF>
 __global__ void __launch_bounds__(32 * MAX_WARPS)
 hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
                           uint64_t slice_bytes, uint64_t total_tasks, uint32_t *__restrict__ slot,
                           SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice,
-                          uint32_t *__restrict__ mid /* [groups][8][32] */, const uint32_t *__restrict__ one_ptr,
-                          uint32_t first_workers_first) {
+                          uint32_t *__restrict__ mid /* [groups][8][32] */, const uint32_t *__restrict__ one_ptr) {
     // Addition placement 0 (left to the compiler).  Moving the schedule's additions to the FMA
     // pipe (placement 2) gains 4.5 % in the register-only probe but lost 5 % in this kernel.
     constexpr int ADD = 0;
@@ -109,33 +131,12 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
     uint32_t parity = 0;
     bool failed = false;
 
-    if (first_workers_first && warp >= 4) __nanosleep(20000);   // the first workers of every CTA claim their groups first
+    bool first_take = true;
     for (;;) {
         // ---- take a ticket, wait for the group that is pushed under it
         unsigned long long t = 0;
-        if (lane == 0) {
-            if (warp < 4 || !first_workers_first) {
-                t = atomicAdd(&q->head, 1ull);
-            } else {
-                // A scheduler's second worker takes a task only when one lies in the FIFO unclaimed: the
-                // first workers (one per scheduler) are served first, so no scheduler idles while another
-                // runs two groups.  With nothing left over it polls; giving up is harmless, the first
-                // workers finish the launch.
-                const long long t0 = clock64();
-                t = total_tasks;
-                for (;;) {
-                    const unsigned long long h = *reinterpret_cast<volatile unsigned long long *>(&q->head);
-                    if (h >= total_tasks) break;
-                    const unsigned long long tl = *reinterpret_cast<volatile unsigned long long *>(&q->tail);
-                    if (tl > h) {
-                        if (atomicCAS(&q->head, h, h + 1ull) == h) { t = h; break; }
-                        continue;
-                    }
-                    if (clock64() - t0 > 8000000000ll) break;
-                    __nanosleep(256);
-                }
-            }
-        }
+        if (lane == 0) t = (!FWF || warp < 4) ? atomicAdd(&q->head, 1ull) : take_leftover_ticket(q, total_tasks, first_take);
+        first_take = false;
         t = __shfl_sync(0xffffffffu, t, 0);
         if (t >= total_tasks) break;
         uint32_t entry = 0;
@@ -382,9 +383,11 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8;
     constexpr size_t smem_per_warp = TILED ? (size_t)STAGES * 8192 : (size_t)STAGES * 32 * (SEG + 16);
     constexpr size_t smem_pad = TILED ? 1024 : 0;
-    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX>;
-    static bool configured[kMaxDevices] = {};
-    if (cudaError_t e0 = ensure_dynamic_smem(kernel, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
+    auto kernel_plain = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX, false>;
+    auto kernel_fwf = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX, true>;
+    static bool configured[kMaxDevices] = {}, configured_fwf[kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel_plain, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel_fwf, MAX_WARPS * smem_per_warp + smem_pad, configured_fwf); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, total_tasks = 0;
     (void)sliced_scratch_bytes(n_chunks, chunk_bytes, &slice_bytes, &total_tasks, nbytes);
     const uint64_t groups = (n_chunks + 31) / 32;
@@ -407,12 +410,13 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     //    slices (256 per chunk) to balance (G = 832 / 896 / 960: 780 / 790 / 811; with 64 slices it loses).
     const bool fine = ((chunk_bytes & ~63ull) + slice_bytes - 1) / slice_bytes >= 192;   // about 256 slices per chunk
     uint64_t warps = 4;
-    uint32_t first_workers_first = 0;
+    bool first_workers_first = false;
     if (fine && 5 * groups >= 28ull * (uint64_t)sm_count) { warps = MAX_WARPS; first_workers_first = groups < 8ull * sm_count; }
     else if (!fine && 10 * groups >= 62ull * (uint64_t)sm_count) warps = MAX_WARPS;
+    auto kernel = first_workers_first ? kernel_fwf : kernel_plain;
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
         map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
-        mid, d_one, first_workers_first);
+        mid, d_one);
     return cudaGetLastError();
 }
 
