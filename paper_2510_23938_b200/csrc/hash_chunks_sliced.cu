@@ -407,19 +407,21 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     // One persistent CTA per SM with four workers (one per scheduler) or eight (two per scheduler).  A
-    // scheduler with two groups finishes 1.13 groups in the time a scheduler with one finishes one, so
-    // eight workers pay once G is well above 592, but with G < 1184 not every scheduler gets two.  Measured:
-    //  * four workers: 775 GB/s for every G >= 592 (4 MiB chunks, 256 slices);
+    // scheduler with two groups finishes 1.11 groups in the time a scheduler with one finishes one, so
+    // eight workers pay once G is well above 592, but with G < 1184 not every scheduler gets two.  Measured
+    // (GB/s at G = 864 / 896 / 960 / 1024 / 1100 groups):
+    //  * four workers: 798 for every G >= 592;
     //  * eight workers, FIFO served in arrival order: idle workers fall at random and groups that met
-    //    doubly loaded schedulers more often finish late (G = 896: 763; G = 1024: 827);
+    //    doubly loaded schedulers more often finish late (4 MiB chunks: 777 / 791 / 818 / 841 / 866);
     //  * eight workers, first workers served first (a second worker takes only what is left over): the
-    //    592 - (G - 592) schedulers with one group finish early and then take over the rest; needs fine
-    //    slices (256 per chunk) to balance (G = 832 / 896 / 960: 780 / 790 / 811; with 64 slices it loses).
+    //    schedulers with one group finish early and then take over the rest; needs fine slices (256
+    //    per chunk) to balance (4 MiB chunks: 801 / 806 / 825 / 842 / 865; 1 MiB chunks with 64 slices:
+    //    767 / 763 / 795 / 822 / 853 against 764 / 780 / 812 / 833 / 860 in arrival order).
     const bool fine = ((chunk_bytes & ~63ull) + slice_bytes - 1) / slice_bytes >= 192;   // about 256 slices per chunk
     uint64_t warps = 4;
     bool first_workers_first = false;
-    if (fine && 5 * groups >= 28ull * (uint64_t)sm_count) { warps = MAX_WARPS; first_workers_first = groups < 8ull * sm_count; }
-    else if (!fine && 10 * groups >= 62ull * (uint64_t)sm_count) warps = MAX_WARPS;
+    if (fine && 20 * groups >= 117ull * (uint64_t)sm_count) { warps = MAX_WARPS; first_workers_first = groups < 8ull * sm_count; }
+    else if (!fine && 10 * groups >= 63ull * (uint64_t)sm_count) warps = MAX_WARPS;
     auto kernel = first_workers_first ? kernel_fwf : kernel_plain;
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
         map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
