@@ -113,6 +113,12 @@ def test_largest_configuration_sampled(ctx):
         want = oracle.hash_chunks_rfc6962(_host(data[i * chunk:(i + 1) * chunk]), chunk)[0]
         assert got6962[i].tobytes() == want.tobytes(), i
     del got6962
+    # and with SHA-384 digests
+    got384 = _host(ctx.hash_chunks_sha384(data, chunk))
+    assert ctx.device_status() == 0
+    for i in sample[1::3]:
+        assert got384[i].tobytes() == oracle.sha384(_host(data[i * chunk:(i + 1) * chunk])), i
+    del got384
     # a flipped bit is found at its chunk, nothing else changes
     manifest = ctx.make_manifest(data.numel(), chunk, got.clone(), root)
     off, bit = inputs.flip_position(7, data.numel())

@@ -85,6 +85,8 @@ def test_migrating_kernel_on_random_large_shapes(ctx):
         got = ctx.hash_chunks_rfc6962(data, chunk)
         assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel"
         assert np.array_equal(_host(got), oracle.hash_chunks_rfc6962(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk)
+        got = ctx.hash_chunks_sha384(data, chunk)
+        assert np.array_equal(_host(got), oracle.hash_chunks_sha384(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk)
         del data
     assert ctx.device_status() == 0
 

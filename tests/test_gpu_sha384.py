@@ -32,7 +32,10 @@ def _host(t: torch.Tensor) -> np.ndarray:
     # remainders around the one-block / two-block padding boundary (111 | 112 bytes)
     (5 * 4096 + 111, 4096), (5 * 4096 + 112, 4096), (5 * 4096 + 239, 4096), (5 * 4096 + 240, 4096),
     (37 * 48 + 16, 48),                   # multiple of 16 but not of 128
-    (20_000 * 4096 + 100, 4096),          # several waves of warps
+    (20_000 * 4096 + 100, 4096),          # several waves of warps, short last chunk
+    (19_000 * 4096, 4096),
+    (9_600 * 65536, 65536),               # larger chunks, many chains
+    (9_600 * 65536 + 127, 65536), (9_500 * (65536 + 16), 65536 + 16), (9_500 * (65536 + 112), 65536 + 112),
 ])
 def test_hash_chunks_sha384_equals_oracle(ctx, nbytes, chunk):
     data = inputs.uniform_bytes(nbytes, seed=384, device="cuda")
