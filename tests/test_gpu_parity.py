@@ -542,3 +542,33 @@ def test_launch_counter_counts_kernels(ctx):
     d = ctx.hash_chunks(data, 1024)
     ctx.merkle_root(d)
     assert ctx.kernel_launches == before + 2
+
+
+def test_two_contexts_on_two_streams_at_once():
+    """One context per stream (the header's rule): two verifications enqueued back to back on two streams
+    overlap on the GPU and both come out right; a third call on the default stream runs beside them."""
+    a, b = binding.Context(0), binding.Context(0)
+    try:
+        sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+        da = inputs.uniform_bytes((96 << 20) + 5, seed=71, device="cuda")
+        db = inputs.uniform_bytes(80 << 20, seed=72, device="cuda")
+        torch.cuda.synchronize()
+        man_a, _, root_a = _manifest_from_oracle(a, _host(da), 1 << 20)
+        man_b, _, root_b = _manifest_from_oracle(b, _host(db), 64 << 10)
+        ra, rb = binding.new_result("cuda"), binding.new_result("cuda")
+        ia = torch.zeros(4, dtype=torch.int64, device="cuda")
+        ib = torch.zeros(4, dtype=torch.int64, device="cuda")
+        db[12345] ^= 1
+        torch.cuda.synchronize()
+        for _ in range(3):
+            a.verify_manifest(da, man_a, ra, ia, stream=sa)
+            b.verify_manifest(db, man_b, rb, ib, stream=sb)
+        torch.cuda.synchronize()
+        r = binding.read_result(ra)
+        assert r["root_ok"] and r["n_mismatch"] == 0 and r["root"] == root_a
+        r = binding.read_result(rb)
+        assert (not r["root_ok"]) and r["n_mismatch"] == 1 and int(ib[0]) == 12345 // (64 << 10)
+        assert a.device_status() == 0 and b.device_status() == 0
+    finally:
+        a.close()
+        b.close()
