@@ -35,7 +35,8 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
 //                 carries 16 bytes more than a segment, so that every 64-byte block lies inside one
 //                 stage; the block is read as 17 aligned words and the byte shift is folded into the
 //                 endian-swap PRMT.
-template <int SEG, int STAGES, int NSLOT, int MODE, bool RAGGED>
+// PAIR: blocks handed over per W+K slot (1 or 2); with 2 the barrier traffic per block halves.
+template <int SEG, int STAGES, int NSLOT, int MODE, bool RAGGED, int PAIR = 1>
 __global__ void __launch_bounds__(64)
 hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                          uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
@@ -46,7 +47,8 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     constexpr uint32_t kStageBytes = 32 * kLaneStride;
     constexpr int kBlocksPerSeg = SEG / 64;
     constexpr uint32_t kWkLane = 64 * 4 + 16;             // W+K ring: bytes per lane per slot
-    constexpr uint32_t kWkSlot = 32 * kWkLane;
+    constexpr uint32_t kWkBlock = 32 * kWkLane;           // one block's W+K for the 32 lanes
+    constexpr uint32_t kWkSlot = PAIR * kWkBlock;
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ __align__(8) uint64_t bars[STAGES + 2 * NSLOT];
 
@@ -174,12 +176,17 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
                 }
                 fetch(in_stage);
             }
-            failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_empty + 8 * slot, eparity));
-            if (failed) break;
-            produce_wk(w, wk_base + slot * kWkSlot, one);
-            __syncwarp();                              // all 32 lanes' stores are ordered before lane 0's arrival
-            if (lane == 0) tma::mbar_arrive(bar_full + 8 * slot);
-            if (++slot == NSLOT) { slot = 0; eparity ^= 1u; }
+            const uint32_t in_slot = (uint32_t)(blk % PAIR);
+            if (in_slot == 0) {
+                failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_empty + 8 * slot, eparity));
+                if (failed) break;
+            }
+            produce_wk(w, wk_base + slot * kWkSlot + in_slot * kWkBlock, one);
+            if (in_slot == PAIR - 1 || blk + 1 == warp_total) {
+                __syncwarp();                          // all 32 lanes' stores are ordered before lane 0's arrival
+                if (lane == 0) tma::mbar_arrive(bar_full + 8 * slot);
+                if (++slot == NSLOT) { slot = 0; eparity ^= 1u; }
+            }
         }
         if (failed && lane == 0) atomicExch(status, (uint32_t)IVK_DEV_TIMEOUT);
         return;
@@ -198,12 +205,19 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     uint32_t fparity = 0;
     bool failed = false;
     for (uint64_t blk = 0; blk < warp_total; ++blk) {
-        failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_full + 8 * slot, fparity));
-        if (failed) break;
-        const uint32_t src = wk_base + slot * kWkSlot;
+        const uint32_t in_slot = (uint32_t)(blk % PAIR);
+        if (in_slot == 0) {
+            // every lane tests the same barrier word, so the outcome is uniform without a vote
+            failed = !tma::mbar_wait_bounded(bar_full + 8 * slot, fparity);
+            if (failed) break;
+        }
+        const uint32_t src = wk_base + slot * kWkSlot + in_slot * kWkBlock;
         rounds64<MODE>(v, src, one);
-        __syncwarp();                                  // all 32 lanes have their values in registers
-        if (lane == 0) tma::mbar_arrive(bar_empty + 8 * slot);
+        const bool slot_done = in_slot == PAIR - 1 || blk + 1 == warp_total;
+        if (slot_done) {
+            __syncwarp();                              // all 32 lanes have their values in registers
+            if (lane == 0) tma::mbar_arrive(bar_empty + 8 * slot);
+        }
         // feed-forward; a lane whose message has ended keeps its state (multiplier 0 instead of 1)
         const uint32_t keep = (blk < my_total) ? one : 0u;
 #pragma unroll
@@ -211,7 +225,7 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
             st[k] = padd<true>(v[k], st[k], keep);     // v * keep + st
             v[k] = st[k];
         }
-        if (++slot == NSLOT) { slot = 0; fparity ^= 1u; }
+        if (slot_done && ++slot == NSLOT) { slot = 0; fparity ^= 1u; }
     }
     if (failed) {
         if (lane == 0) atomicExch(status, (uint32_t)IVK_DEV_TIMEOUT);
@@ -230,11 +244,12 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
 cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status,
                                      const uint32_t *d_one, cudaStream_t stream) {
-    // 512-byte segments, three data stages, four W+K slots; the additions that close the two state
+    // 512-byte segments, three data stages, three W+K slots of two blocks each (two blocks per hand-over
+    // halve the barrier traffic: +1 % over four single-block slots; 104 KB per CTA, two CTAs per SM); the additions that close the two state
     // recurrences stay three-input ALU adds, the others go to the FMA pipe (placement 3, the fastest measured).
-    constexpr int SEG = 512, STAGES = 3, NSLOT = 4, MODE = 3;
-    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * 32 * (64 * 4 + 16);
-    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false>;
+    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, MODE = 3, PAIR = 2;
+    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
+    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false, PAIR>;
     static bool configured[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
     const uint64_t blocks = (n_chunks + 31) / 32;
@@ -247,9 +262,9 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
 cudaError_t launch_hash_ragged_split(const uint8_t *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
                                      const uint32_t *d_order, uint64_t n, uint8_t *d_digests, uint32_t *d_status,
                                      const uint32_t *d_one, iv_sha_state *d_states, int finish, cudaStream_t stream) {
-    constexpr int SEG = 512, STAGES = 3, NSLOT = 4, MODE = 3;
-    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 32) + (size_t)NSLOT * 32 * (64 * 4 + 16);
-    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, true>;
+    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, MODE = 3, PAIR = 2;
+    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 32) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
+    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, true, PAIR>;
     static bool configured[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
     const uint64_t blocks = (n + 31) / 32;
