@@ -94,16 +94,17 @@ __device__ __forceinline__ void tiled_g2s(uint32_t dst, const CUtensorMap *map, 
 // PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash).  Message block j is then the
 // byte before data block j followed by its first 63 bytes; the word before the block is carried in a
 // register, at the start of a later slice it is read back from the blob.
-template <int SEG, int STAGES, int MAX_WARPS, bool TILED, bool PREFIX, bool FWF>
+// ADD: where the additions of the compression go (see sha256_compress).
+template <int SEG, int STAGES, int MAX_WARPS, bool TILED, bool PREFIX, bool FWF, int ADD>
 __global__ void __launch_bounds__(32 * MAX_WARPS)
 hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
                           uint64_t slice_bytes, uint64_t total_tasks, uint32_t *__restrict__ slot,
                           SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice,
                           uint32_t *__restrict__ mid /* [groups][8][32] */, const uint32_t *__restrict__ one_ptr) {
-    // Addition placement 0 (left to the compiler).  Moving the schedule's additions to the FMA
-    // pipe (placement 2) gains 4.5 % in the register-only probe but lost 5 % in this kernel.
-    constexpr int ADD = 0;
+    // With two warps per scheduler addition placement 0 (left to the compiler) is the fastest; moving the
+    // schedule's additions to the FMA pipe (placement 2) lengthens the dependency chains and needs three warps
+    // per scheduler to pay (launcher below).
     const uint32_t one = __ldg(one_ptr);
     static_assert(!TILED || SEG == 256, "a tiled stage is two boxes of 32 rows x 128 bytes");
     constexpr uint32_t kLaneStride = TILED ? 128 : SEG + 16;
@@ -387,14 +388,19 @@ template <bool TILED, bool PREFIX>
 cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
                           const uint32_t *d_one, int sm_count, cudaStream_t stream) {
-    constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8;
+    // Three instances: up to eight workers per SM with three stages each (arrival order or first workers
+    // first), and twelve workers with two stages each for launches that keep all of them busy.
+    constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8, MANY_STAGES = 2, MANY_WARPS = 12;
     constexpr size_t smem_per_warp = TILED ? (size_t)STAGES * 8192 : (size_t)STAGES * 32 * (SEG + 16);
+    constexpr size_t many_per_warp = TILED ? (size_t)MANY_STAGES * 8192 : (size_t)MANY_STAGES * 32 * (SEG + 16);
     constexpr size_t smem_pad = TILED ? 1024 : 0;
-    auto kernel_plain = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX, false>;
-    auto kernel_fwf = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX, true>;
-    static bool configured[kMaxDevices] = {}, configured_fwf[kMaxDevices] = {};
+    auto kernel_plain = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX, false, 0>;
+    auto kernel_fwf = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX, true, 0>;
+    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, TILED, PREFIX, false, 2>;
+    static bool configured[kMaxDevices] = {}, configured_fwf[kMaxDevices] = {}, configured_many[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel_plain, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
     if (cudaError_t e0 = ensure_dynamic_smem(kernel_fwf, MAX_WARPS * smem_per_warp + smem_pad, configured_fwf); e0 != cudaSuccess) return e0;
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel_many, MANY_WARPS * many_per_warp + smem_pad, configured_many); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, total_tasks = 0;
     (void)sliced_scratch_bytes(n_chunks, chunk_bytes, &slice_bytes, &total_tasks, nbytes);
     const uint64_t groups = (n_chunks + 31) / 32;
@@ -422,6 +428,14 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     bool first_workers_first = false;
     if (fine && 20 * groups >= 117ull * (uint64_t)sm_count) { warps = MAX_WARPS; first_workers_first = groups < 8ull * sm_count; }
     else if (!fine && 10 * groups >= 63ull * (uint64_t)sm_count) warps = MAX_WARPS;
+    // From twelve groups per SM on, three warps per scheduler hide the longer chains of multiply-add
+    // additions, which take a tenth of the ALU pipe's load: 917 GB/s against 884 (32 GiB in 64 KiB chunks).
+    if (groups >= (uint64_t)MANY_WARPS * (uint64_t)sm_count) {
+        kernel_many<<<(unsigned)sm_count, 32 * MANY_WARPS, MANY_WARPS * many_per_warp + smem_pad, stream>>>(
+            map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q,
+            next_slice, mid, d_one);
+        return cudaGetLastError();
+    }
     auto kernel = first_workers_first ? kernel_fwf : kernel_plain;
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
         map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
