@@ -40,7 +40,7 @@ def _root_bytes(t: torch.Tensor) -> bytes:
     (50 * (4096 + 16) + 8, 4096 + 16),   # staged path with a 16-byte remainder in every chunk
     (33 * 8192 + 4100, 8192), (3 * 65536 + 300, 65536 + 48),
     (20_000 * 4096 + 100, 4096),     # more than 592 warps: the many-chain launch shape, ragged last chunk
-    (19_000 * 4096, 4096),
+    (19_000 * 4096, 4096),    (60_000 * 4096 + 100, 4096), (57_000 * 16384, 16384),   # 12 or more groups per SM: the twelve-worker instance
 ])
 def test_hash_chunks_equals_oracle(ctx, nbytes, chunk):
     data = inputs.uniform_bytes(nbytes, seed=1, device="cuda")

@@ -37,7 +37,7 @@ def _host(t: torch.Tensor) -> np.ndarray:
     (20_000 * 4096 + 100, 4096),          # the migrating kernel (more than 296 warps), short last chunk beside it
     (19_000 * 4096, 4096),
     (9_600 * 65536, 65536),               # several slices per chunk: the carried word crosses slice borders
-    (9_600 * 65536 + 63, 65536), (9_500 * (65536 + 16), 65536 + 16),
+    (9_600 * 65536 + 63, 65536), (9_500 * (65536 + 16), 65536 + 16),    (60_000 * 4096 + 100, 4096), (57_000 * 16384, 16384),   # 12 or more groups per SM: the twelve-worker instance
 ])
 def test_leaf_hashes_equal_oracle(ctx, nbytes, chunk):
     data = inputs.uniform_bytes(nbytes, seed=6962, device="cuda")
