@@ -231,6 +231,9 @@ int iv_verify_manifest_two_level(iv_ctx *ctx, const void *d_data, uint64_t nbyte
  * the blob is copied window by window into two device windows owned by the
  * context, the copy of window w+1 overlapping the hashing of window w on a
  * second stream, then the tree is built and compared as in iv_verify_manifest.
+ * A window with few large chunks is copied and hashed in column parts (part s of
+ * every chunk while part s+1 is in flight), so that its hashing ends shortly
+ * after its last byte arrives; the results are the same.
  *
  *   h_windows      host array of n_windows HOST pointers; window w holds bytes
  *                  [w*window_bytes, min((w+1)*window_bytes, nbytes)) of the blob.

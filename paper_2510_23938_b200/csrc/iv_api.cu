@@ -44,6 +44,8 @@ struct iv_ctx {
     uint64_t slices_cap = 0;                  // bytes
 
     // streaming windows
+    uint8_t *d_columns = nullptr;             // offsets, lengths and chaining values of a window hashed in column parts
+    uint64_t columns_cap = 0;                 // bytes
     uint8_t *d_window[2] = {nullptr, nullptr};
     uint64_t window_cap = 0;
     cudaStream_t copy_stream = nullptr;
@@ -161,6 +163,41 @@ int check_manifest(const iv_manifest *m, uint64_t nbytes) {
     if (m->total_bytes != nbytes) return IV_ERR_INVALID_ARG;
     if (m->n_chunks != chunk_count(nbytes, m->chunk_bytes)) return IV_ERR_INVALID_ARG;
     if (m->n_chunks && !m->d_digests) return IV_ERR_INVALID_ARG;
+    return IV_OK;
+}
+
+// One window of a streamed blob, copied and hashed in column parts (see iv_verify_streamed).  The window has m
+// chunks of which the last may be short; it lands in ctx->d_window[b], its digests at d_digests.
+int hash_window_in_columns(iv_ctx *ctx, const void *h_window, uint64_t bytes, uint64_t chunk, uint64_t m, uint32_t parts,
+                           int b, uint8_t *d_digests, cudaStream_t stream) {
+    const uint64_t part = (chunk / parts) & ~4095ull;              // a whole number of blocks, at least 64 KiB
+    const uint64_t whole = bytes / chunk;                          // m or m - 1
+    const uint64_t need = 2 * 8 * m * parts + sizeof(iv_sha_state) * m + 64;
+    int rc = grow(ctx, &ctx->d_columns, &ctx->columns_cap, need, 1);
+    if (rc != IV_OK) return rc;
+    uint64_t *d_off = reinterpret_cast<uint64_t *>(ctx->d_columns);
+    uint64_t *d_len = d_off + m * parts;
+    iv_sha_state *d_states = reinterpret_cast<iv_sha_state *>(d_len + m * parts);
+    IV_TRY(ctx, ivk::launch_column_ranges(m, bytes, chunk, part, parts, d_off, d_len, stream, &ctx->launches));
+    IV_TRY(ctx, cudaMemsetAsync(d_states, 0, sizeof(iv_sha_state) * m, stream));
+    uint8_t *dst = ctx->d_window[b];
+    const uint8_t *src = static_cast<const uint8_t *>(h_window);
+    for (uint32_t s = 0; s < parts; ++s) {
+        const uint64_t lo = (uint64_t)s * part;
+        const uint64_t width = (s + 1 == parts) ? chunk - lo : part;
+        if (whole)
+            IV_TRY(ctx, cudaMemcpy2DAsync(dst + lo, chunk, src + lo, chunk, width, whole, cudaMemcpyHostToDevice,
+                                          ctx->copy_stream));
+        if (s == 0 && whole < m)                                   // the blob's short last chunk comes with the first part
+            IV_TRY(ctx, cudaMemcpyAsync(dst + whole * chunk, src + whole * chunk, bytes - whole * chunk,
+                                        cudaMemcpyHostToDevice, ctx->copy_stream));
+        IV_TRY(ctx, cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
+        IV_TRY(ctx, cudaStreamWaitEvent(stream, ctx->ev_copied[b], 0));
+        IV_TRY(ctx, ivk::launch_hash_ragged_split(dst, d_off + (uint64_t)s * m, d_len + (uint64_t)s * m, nullptr, m, d_digests,
+                                                  ctx->d_status, ctx->d_one, d_states, s + 1 == parts ? 1 : 0, stream));
+        ++ctx->launches;
+    }
+    ctx->leaf_kernel = "hash_chunks_split_kernel (tensors)";
     return IV_OK;
 }
 
@@ -284,6 +321,7 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_slices);
     cudaFree(ctx->d_order);
     cudaFree(ctx->d_dirty_scratch);
+    cudaFree(ctx->d_columns);
     cudaFree(ctx->d_sub);
     cudaFree(ctx->d_batch);
     cudaFree(ctx->d_tree384[0]);
@@ -628,6 +666,22 @@ int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_win
         const uint64_t off = w * window_bytes;
         const uint64_t bytes = nbytes - off < window_bytes ? nbytes - off : window_bytes;
         if (w >= 2) IV_TRY(ctx, cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_hashed[b], 0));
+        {
+            // With few chunks the hashing of a window lasts as long as ONE chunk's serial chain, whatever the
+            // window's size, and it can start only when the window has arrived: the hashing runs a window
+            // behind the copies and nothing overlaps the last one.  So a window arrives in column parts (part s
+            // of every chunk, one strided copy) and part s is hashed, from the chaining values part s - 1 left,
+            // while part s + 1 is on its way: what remains after the last byte is one part's time.
+            const uint64_t m = chunk_count(bytes, chunk);
+            const uint64_t parts = chunk / 65536 < 8 ? chunk / 65536 : 8;
+            if (parts >= 2 && chunk < (1ull << 31) && m <= 2ull * 32 * (uint64_t)ctx->sm_count && m <= ivk::kRaggedSortMax) {
+                rc = hash_window_in_columns(ctx, h_windows[w], bytes, chunk, m, (uint32_t)parts, b,
+                                            ctx->d_digests + 32 * w * chunks_per_window, stream);
+                if (rc != IV_OK) return rc;
+                IV_TRY(ctx, cudaEventRecord(ctx->ev_hashed[b], stream));
+                continue;
+            }
+        }
         IV_TRY(ctx, cudaMemcpyAsync(ctx->d_window[b], h_windows[w], bytes, cudaMemcpyHostToDevice, ctx->copy_stream));
         IV_TRY(ctx, cudaEventRecord(ctx->ev_copied[b], ctx->copy_stream));
         IV_TRY(ctx, cudaStreamWaitEvent(stream, ctx->ev_copied[b], 0));

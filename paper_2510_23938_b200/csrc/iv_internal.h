@@ -107,6 +107,10 @@ constexpr int kTreeMaxLevels = 40;
 uint64_t tree_records(uint64_t n_leaves);
 cudaError_t launch_tree_build(const uint8_t *d_leaves, uint64_t n, uint8_t *d_tree, cudaStream_t stream,
                               uint64_t *launches);
+// Offsets and lengths of the column parts of a window's m chunks (entry s * m + i = part s of chunk i): a chunk's
+// whole blocks are cut into `parts` pieces of part_bytes (a multiple of 64), the last part takes the rest.
+cudaError_t launch_column_ranges(uint64_t m, uint64_t bytes, uint64_t chunk_bytes, uint64_t part_bytes, uint32_t parts,
+                                 uint64_t *d_offsets, uint64_t *d_lengths, cudaStream_t stream, uint64_t *launches);
 cudaError_t launch_dirty_ranges(const uint64_t *d_dirty, uint64_t n_dirty, uint64_t nbytes, uint64_t chunk_bytes,
                                 uint64_t n_leaves, uint64_t *d_offsets, uint64_t *d_lengths, uint32_t *d_status,
                                 cudaStream_t stream, uint64_t *launches);

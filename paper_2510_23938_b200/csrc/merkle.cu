@@ -246,6 +246,23 @@ __global__ void batch_ranges_kernel(BlobList blobs, uint64_t n_chunks, uint64_t 
     lengths[t] = (nbytes - begin < chunk_bytes) ? (nbytes - begin) : chunk_bytes;
 }
 
+// Column parts of the chunks of one window: part s of chunk i covers bytes [s * part, (s + 1) * part) of the
+// chunk's whole 64-byte blocks, the last part everything that is left (tail and padding included).
+// Entry s * m + i; a part that finishes no chunk is a whole number of blocks.
+__global__ void column_ranges_kernel(uint64_t m, uint64_t bytes, uint64_t chunk_bytes, uint64_t part_bytes, uint32_t parts,
+                                     uint64_t *__restrict__ offsets, uint64_t *__restrict__ lengths) {
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= m * parts) return;
+    const uint64_t s = t / m, i = t - s * m;
+    const uint64_t begin = i * chunk_bytes;
+    const uint64_t len = (bytes - begin < chunk_bytes) ? (bytes - begin) : chunk_bytes;
+    const uint64_t full = len & ~63ull;
+    const uint64_t lo = s * part_bytes < full ? s * part_bytes : full;
+    const uint64_t hi = (s + 1 == parts) ? len : ((s + 1) * part_bytes < full ? (s + 1) * part_bytes : full);
+    offsets[t] = begin + lo;
+    lengths[t] = hi - lo;
+}
+
 // new leaf digests (in dirty-list order) into the leaf level of the tree
 __global__ void scatter_leaves_kernel(const uint8_t *__restrict__ fresh, const uint64_t *__restrict__ dirty,
                                       uint64_t n_dirty, uint64_t n_leaves, uint8_t *__restrict__ tree) {
@@ -455,6 +472,16 @@ cudaError_t launch_batch_ranges(const BlobList &blobs, uint64_t n_chunks, uint64
     const uint64_t total = n_chunks * blobs.count;
     batch_ranges_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(blobs, n_chunks, nbytes, chunk_bytes,
                                                                             d_offsets, d_lengths);
+    if (launches) ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_column_ranges(uint64_t m, uint64_t bytes, uint64_t chunk_bytes, uint64_t part_bytes, uint32_t parts,
+                                 uint64_t *d_offsets, uint64_t *d_lengths, cudaStream_t stream, uint64_t *launches) {
+    const uint64_t total = m * parts;
+    if (total == 0) return cudaSuccess;
+    column_ranges_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(m, bytes, chunk_bytes, part_bytes, parts,
+                                                                             d_offsets, d_lengths);
     if (launches) ++*launches;
     return cudaGetLastError();
 }

@@ -410,6 +410,45 @@ def test_streamed_verification_equals_resident(ctx, pinned):
         ctx.verify_streamed(host, chunk + 1, host.numel(), manifest, res, idx)
 
 
+@pytest.mark.parametrize("chunk,n_chunks,short_by,window_chunks,pinned", [
+    (131072, 37, 1000, 8, True),            # two column parts per chunk, five windows, short last chunk
+    (1 << 20, 19, 77, 4, True),             # eight parts, a last chunk that ends inside a block
+    (1 << 20, 19, 77, 19, False),           # one window, pageable host memory
+    (5 * 65536 + 64, 11, 0, 3, True),       # a chunk size that is no multiple of 4 KiB: the last part is longer
+    (200_008, 9, 199_990, 4, True),         # no multiple of 16; the short last chunk has 18 bytes
+    (1 << 20, 1, 0, 1, True), (1 << 20, 1, (1 << 20) - 64, 1, True), (1 << 20, 2, (1 << 20) - 1, 2, True),
+])
+def test_streamed_windows_hashed_in_column_parts(ctx, chunk, n_chunks, short_by, window_chunks, pinned):
+    """Chunks of 128 KiB and more with few chains per window take the column-part path of the streamed
+    verification (strided copies, resumed chaining values): digests, root and the located damage equal the oracle's."""
+    nbytes = chunk * n_chunks - short_by
+    host = inputs.uniform_bytes(nbytes, seed=33 + n_chunks)
+    manifest, digests, root = _manifest_from_oracle(ctx, host.numpy(), chunk)
+    src = host.pin_memory() if pinned else host
+    res = binding.new_result("cuda")
+    idx = torch.zeros(8, dtype=torch.int64, device="cuda")
+    for _ in range(2):                                       # twice: the window buffers and states are reused
+        ctx.verify_streamed(src, window_chunks * chunk, nbytes, manifest, res, idx)
+        torch.cuda.synchronize()
+        r = binding.read_result(res)
+        assert r == {"status": 0, "root_ok": True, "n_mismatch": 0, "root": root}
+        assert np.array_equal(_host(ctx.last_digests(n_chunks)), digests)
+    # one flipped bit in a middle part of a chunk and one in the very last byte
+    bad = host.clone()
+    hits = sorted({min(nbytes - 1, (n_chunks // 2) * chunk + chunk // 2 + 5), nbytes - 1})
+    for off in hits:
+        bad[off] ^= 0x40
+    ctx.verify_streamed(bad.pin_memory() if pinned else bad, window_chunks * chunk, nbytes, manifest, res, idx)
+    torch.cuda.synchronize()
+    r = binding.read_result(res)
+    want_idx = sorted({off // chunk for off in hits})
+    assert (not r["root_ok"]) and r["n_mismatch"] == len(want_idx)
+    assert [int(v) for v in idx[:len(want_idx)].cpu()] == want_idx
+    want = oracle.hash_chunks(bad.numpy(), chunk, nthreads=oracle.host_threads())
+    assert np.array_equal(_host(ctx.last_digests(n_chunks)), want) and r["root"] == oracle.merkle_root(want)
+    assert ctx.device_status() == 0
+
+
 # ------------------------------------------------------------------------------------------ a6
 
 def test_hash_ragged_edge_lengths_and_alignments(ctx):
