@@ -170,7 +170,7 @@ int check_manifest(const iv_manifest *m, uint64_t nbytes) {
 // chunks of which the last may be short; it lands in ctx->d_window[b], its digests at d_digests.
 int hash_window_in_columns(iv_ctx *ctx, const void *h_window, uint64_t bytes, uint64_t chunk, uint64_t m, uint32_t parts,
                            int b, uint8_t *d_digests, cudaStream_t stream) {
-    const uint64_t part = (chunk / parts) & ~4095ull;              // a whole number of blocks, at least 64 KiB
+    const uint64_t part = (chunk / parts) & ~4095ull;              // a whole number of blocks, at least 16 KiB
     const uint64_t whole = bytes / chunk;                          // m or m - 1
     const uint64_t need = 2 * 8 * m * parts + sizeof(iv_sha_state) * m + 64;
     int rc = grow(ctx, &ctx->d_columns, &ctx->columns_cap, need, 1);
@@ -673,7 +673,7 @@ int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_win
             // of every chunk, one strided copy) and part s is hashed, from the chaining values part s - 1 left,
             // while part s + 1 is on its way: what remains after the last byte is one part's time.
             const uint64_t m = chunk_count(bytes, chunk);
-            const uint64_t parts = chunk / 65536 < 8 ? chunk / 65536 : 8;
+            const uint64_t parts = chunk / 16384 < 8 ? chunk / 16384 : 8;       // parts of at least 16 KiB
             if (parts >= 2 && chunk < (1ull << 31) && m <= 2ull * 32 * (uint64_t)ctx->sm_count && m <= ivk::kRaggedSortMax) {
                 rc = hash_window_in_columns(ctx, h_windows[w], bytes, chunk, m, (uint32_t)parts, b,
                                             ctx->d_digests + 32 * w * chunks_per_window, stream);

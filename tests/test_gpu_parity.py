@@ -411,7 +411,9 @@ def test_streamed_verification_equals_resident(ctx, pinned):
 
 
 @pytest.mark.parametrize("chunk,n_chunks,short_by,window_chunks,pinned", [
-    (131072, 37, 1000, 8, True),            # two column parts per chunk, five windows, short last chunk
+    (32768, 40, 100, 16, True),             # two column parts of 16 KiB per chunk
+    (65536, 64, 0, 64, True), (3 * 16384 + 4096 + 48, 21, 5, 5, False),   # four parts; three parts, odd chunk size
+    (131072, 37, 1000, 8, True),            # eight column parts per chunk, five windows, short last chunk
     (1 << 20, 19, 77, 4, True),             # eight parts, a last chunk that ends inside a block
     (1 << 20, 19, 77, 19, False),           # one window, pageable host memory
     (5 * 65536 + 64, 11, 0, 3, True),       # a chunk size that is no multiple of 4 KiB: the last part is longer
@@ -419,7 +421,7 @@ def test_streamed_verification_equals_resident(ctx, pinned):
     (1 << 20, 1, 0, 1, True), (1 << 20, 1, (1 << 20) - 64, 1, True), (1 << 20, 2, (1 << 20) - 1, 2, True),
 ])
 def test_streamed_windows_hashed_in_column_parts(ctx, chunk, n_chunks, short_by, window_chunks, pinned):
-    """Chunks of 128 KiB and more with few chains per window take the column-part path of the streamed
+    """Chunks of 32 KiB and more with few chains per window take the column-part path of the streamed
     verification (strided copies, resumed chaining values): digests, root and the located damage equal the oracle's."""
     nbytes = chunk * n_chunks - short_by
     host = inputs.uniform_bytes(nbytes, seed=33 + n_chunks)
