@@ -32,35 +32,11 @@
 #include "iv_internal.h"
 #include "rfc6962_dev.cuh"
 #include "sha256_dev.cuh"
+#include "slice_queue_dev.cuh"
 #include "tma_dev.cuh"
 
 namespace ivk {
 namespace {
-
-struct SliceQueue {
-    unsigned long long head;   // next ticket to hand to a worker
-    unsigned long long tail;   // next ticket a finished slice pushes its group under
-};
-
-// slot[t] = group + 1 once ticket t has been pushed, 0 before.  The first `groups` tickets are
-// pre-filled with the groups in order; every group starts at slice 0.
-__global__ void slice_queue_init(uint32_t *__restrict__ slot, uint64_t total_tasks, uint64_t groups,
-                                 SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice) {
-    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total_tasks; i += stride)
-        slot[i] = i < groups ? (uint32_t)i + 1u : 0u;
-    for (uint64_t g = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += stride) next_slice[g] = 0u;
-    if (blockIdx.x == 0 && threadIdx.x == 0) { q->head = 0ull; q->tail = groups; }
-}
-
-__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v) {
-    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 
 // A scheduler's second worker takes a task only when one lies in the FIFO unclaimed: the first
 // workers (one per scheduler) are served first, so no scheduler idles while another runs two

@@ -129,6 +129,13 @@ cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_man
                                   uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
                                   const uint32_t *d_status, cudaStream_t stream, uint64_t *launches);
 
+// hash_chunks_pairs.cu -----------------------------------------------------
+// Between few and many chains (2 x SMs < groups of 32 chains < about 3 x SMs): the 2 x SMs producer/consumer
+// warp pairs as persistent workers on the slice FIFO.  d_scratch as for launch_hash_chunks_sliced.
+cudaError_t launch_hash_chunks_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
+                                     uint8_t *d_digests, uint32_t *d_status, void *d_scratch, const uint32_t *d_one,
+                                     int sm_count, cudaStream_t stream);
+
 // hash_sha384.cu -----------------------------------------------------------
 // SHA-384 variant: 48-byte chunk digests and the tree with SHA-384 parents.
 cudaError_t launch_hash_chunks_sha384(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,

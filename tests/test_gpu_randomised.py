@@ -70,7 +70,8 @@ def test_chunk_digests_and_roots_of_random_shapes(ctx, block):
 
 
 def test_migrating_kernel_on_random_large_shapes(ctx):
-    """More than 296 warps of chains with chunk sizes that are multiples of 16 bytes and at least 4 KiB."""
+    """More than 296 warps of chains with chunk sizes that are multiples of 16 bytes and at least 4 KiB: the
+    shapes of the two kernels that hand chains from worker to worker through the slice FIFO."""
     rng = np.random.default_rng(77)
     for _ in range(6):
         chunk = 16 * int(rng.integers(256, 6_000))
@@ -80,7 +81,7 @@ def test_migrating_kernel_on_random_large_shapes(ctx):
         data = inputs.uniform_bytes(nbytes, seed=nbytes, device="cuda")
         host = _host(data)
         got = ctx.hash_chunks(data, chunk)
-        assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel"
+        assert ctx.last_leaf_kernel in ("hash_chunks_sliced_kernel", "hash_chunks_pairs_kernel")
         assert np.array_equal(_host(got), oracle.hash_chunks(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk)
         got = ctx.hash_chunks_rfc6962(data, chunk)
         assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel"
