@@ -259,10 +259,8 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
         // Many chains of sliceable size: chains migrate between schedulers (two launches: queue set-up + workers).
         if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
             if (launches) ++*launches;
-            // Just above 2 x SMs groups the 2 x SMs two-warp pairs, shared by all groups through the FIFO, still
-            // beat one whole-compression warp per group: 570 GB/s flat against 1.345 GB/s per group (measured
-            // crossover at 424 groups = 2.865 x SMs for chunks of 64 KiB to 4 MiB).
-            if (warps * 1000ull < 2865ull * (uint64_t)sm_count) {
+            // just above 2 x SMs groups: the two-warp pairs as workers on the slice FIFO
+            if (hash_chunks_wants_pairs(d_data, chunk_bytes, n_chunks, sm_count)) {
                 *kernel_used = "hash_chunks_pairs_kernel";
                 return launch_hash_chunks_pairs(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
                                                 d_slice_scratch, d_one, sm_count, stream);

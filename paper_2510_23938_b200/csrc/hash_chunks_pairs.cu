@@ -15,6 +15,7 @@
 // barrier phases carry over from task to task (every task drains what it requested).  All waits are
 // bounded.
 #include "iv_internal.h"
+#include "rfc6962_dev.cuh"
 #include "sha256_dev.cuh"
 #include "sha256_split_dev.cuh"
 #include "slice_queue_dev.cuh"
@@ -25,7 +26,8 @@ namespace {
 
 constexpr unsigned long long kTaskDone = ~0ull, kTaskFailed = ~0ull - 1;
 
-template <int SEG, int STAGES, int NSLOT, int MODE, int PAIR>
+// PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash), as in the migrating kernel.
+template <int SEG, int STAGES, int NSLOT, int MODE, int PAIR, bool PREFIX>
 __global__ void __launch_bounds__(64)
 hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
                          uint8_t *__restrict__ digests, uint32_t *__restrict__ status, uint64_t slice_bytes,
@@ -111,7 +113,11 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
         const uint64_t warp_full_bytes = __shfl_sync(0xffffffffu, full_bytes, 0);
         const bool last_slice = hi_full >= warp_full_bytes;
         const uint32_t my_data = (uint32_t)((my_hi - my_lo) >> 6);            // whole data blocks in this slice
-        const uint32_t my_tail = (valid && last_slice) ? (uint32_t)((((len + 8) >> 6) + 1) - (full_bytes >> 6)) : 0u;
+        // blocks after the whole data blocks: the message's remainder and padding (the prefixed message is one
+        // byte longer, and its block j ends one byte before data block j does)
+        const uint32_t my_tail = !(valid && last_slice) ? 0u
+                                 : PREFIX ? ((len + 1 - full_bytes) + 9 <= 64 ? 1u : 2u)
+                                          : (uint32_t)((((len + 8) >> 6) + 1) - (full_bytes >> 6));
         const uint32_t my_total = my_data + my_tail;
         const uint32_t warp_total = __shfl_sync(0xffffffffu, my_total, 0);
         const uint32_t warp_data = __shfl_sync(0xffffffffu, my_data, 0);
@@ -137,6 +143,8 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
                 }
             }
             uint32_t w[16], raw[16], tw[32];
+            uint32_t carry = 0u;        // PREFIX: the data word before the block; byte 3 of 0 is the prefix itself
+            if (PREFIX && my_lo > 0 && my_data > 0) carry = __ldg(reinterpret_cast<const uint32_t *>(p) - 1);
             int in_stage = 0;
             bool tail_built = false;
             auto fetch = [&](int blk_in_stage) {
@@ -152,11 +160,19 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
             uint32_t next_seg = STAGES;
             for (uint32_t blk = 0; blk < warp_total && !failed; ++blk) {
                 if (blk < my_data) {
+                    if (PREFIX) {
+                        w[0] = shifted_word(raw[0], carry);
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) w[k] = bswap32(raw[k]);
+                        for (int k = 1; k < 16; ++k) w[k] = shifted_word(raw[k], raw[k - 1]);
+                        carry = raw[15];
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) w[k] = bswap32(raw[k]);
+                    }
                 } else if (blk < my_total) {
                     if (!tail_built) {
-                        (void)sha256_build_tail(data + begin + full_bytes, (uint32_t)(len & 63u), len, tw);
+                        if (PREFIX) (void)prefixed_tail(data + begin, 0x00, full_bytes, len + 1, tw);
+                        else (void)sha256_build_tail(data + begin + full_bytes, (uint32_t)(len & 63u), len, tw);
                         tail_built = true;
                     }
                     const int t = (int)(blk - my_data);
@@ -248,14 +264,22 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
 
 }  // namespace
 
+bool hash_chunks_wants_pairs(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count) {
+    // 570 GB/s flat for the pairs against 1.345 GB/s per group for one whole-compression warp per group:
+    // measured crossover at 424 groups = 2.865 x SMs, for chunks of 64 KiB to 4 MiB
+    return hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count) &&
+           ((n_chunks + 31) / 32) * 1000ull < 2865ull * (uint64_t)sm_count;
+}
+
 cudaError_t launch_hash_chunks_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
                                      uint8_t *d_digests, uint32_t *d_status, void *d_scratch, const uint32_t *d_one,
-                                     int sm_count, cudaStream_t stream) {
+                                     int sm_count, cudaStream_t stream, bool zero_prefix) {
     constexpr int SEG = 512, STAGES = 3, NSLOT = 3, MODE = 3, PAIR = 2;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
-    auto kernel = hash_chunks_pairs_kernel<SEG, STAGES, NSLOT, MODE, PAIR>;
-    static bool configured[kMaxDevices] = {};
-    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
+    auto kernel = zero_prefix ? hash_chunks_pairs_kernel<SEG, STAGES, NSLOT, MODE, PAIR, true>
+                              : hash_chunks_pairs_kernel<SEG, STAGES, NSLOT, MODE, PAIR, false>;
+    static bool configured[2][kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured[zero_prefix ? 1 : 0]); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, total_tasks = 0;
     (void)sliced_scratch_bytes(n_chunks, chunk_bytes, &slice_bytes, &total_tasks, nbytes);
     const uint64_t groups = (n_chunks + 31) / 32;

@@ -135,8 +135,13 @@ cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, u
                                        const char **kernel_used) {
     if (n_chunks == 0) return cudaSuccess;
     if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
-        // many chains that do not divide evenly over the schedulers: the migrating kernel, prefixed
         if (launches) *launches += 2;
+        if (hash_chunks_wants_pairs(d_data, chunk_bytes, n_chunks, sm_count)) {
+            if (kernel_used) *kernel_used = "hash_chunks_pairs_kernel";
+            return launch_hash_chunks_pairs(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_slice_scratch,
+                                            d_one, sm_count, stream, true);
+        }
+        // many chains that do not divide evenly over the schedulers: the migrating kernel, prefixed
         if (kernel_used) *kernel_used = "hash_chunks_sliced_kernel";
         uint64_t covered = 0;
         cudaError_t e = launch_hash_chunks_sliced(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,

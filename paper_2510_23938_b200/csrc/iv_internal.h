@@ -132,9 +132,10 @@ cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_man
 // hash_chunks_pairs.cu -----------------------------------------------------
 // Between few and many chains (2 x SMs < groups of 32 chains < about 3 x SMs): the 2 x SMs producer/consumer
 // warp pairs as persistent workers on the slice FIFO.  d_scratch as for launch_hash_chunks_sliced.
+bool hash_chunks_wants_pairs(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count);
 cudaError_t launch_hash_chunks_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
                                      uint8_t *d_digests, uint32_t *d_status, void *d_scratch, const uint32_t *d_one,
-                                     int sm_count, cudaStream_t stream);
+                                     int sm_count, cudaStream_t stream, bool zero_prefix = false);
 
 // hash_sha384.cu -----------------------------------------------------------
 // SHA-384 variant: 48-byte chunk digests and the tree with SHA-384 parents.

@@ -84,7 +84,7 @@ def test_migrating_kernel_on_random_large_shapes(ctx):
         assert ctx.last_leaf_kernel in ("hash_chunks_sliced_kernel", "hash_chunks_pairs_kernel")
         assert np.array_equal(_host(got), oracle.hash_chunks(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk)
         got = ctx.hash_chunks_rfc6962(data, chunk)
-        assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel"
+        assert ctx.last_leaf_kernel in ("hash_chunks_sliced_kernel", "hash_chunks_pairs_kernel")
         assert np.array_equal(_host(got), oracle.hash_chunks_rfc6962(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk)
         got = ctx.hash_chunks_sha384(data, chunk)
         assert np.array_equal(_host(got), oracle.hash_chunks_sha384(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk)
