@@ -13,6 +13,7 @@
 // The two rings are handed over through mbarriers (full / empty per slot); all waits are bounded.
 // The chain's critical path per block drops from the whole compression to the rounds alone.
 #include "iv_internal.h"
+#include "rfc6962_dev.cuh"
 #include "sha256_dev.cuh"
 #include "tma_dev.cuh"
 #include "sha256_split_dev.cuh"
@@ -36,7 +37,8 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
 //                 stage; the block is read as 17 aligned words and the byte shift is folded into the
 //                 endian-swap PRMT.
 // PAIR: blocks handed over per W+K slot (1 or 2); with 2 the barrier traffic per block halves.
-template <int SEG, int STAGES, int NSLOT, int MODE, bool RAGGED, int PAIR = 1>
+// PREFIX (chunks only): message i is 0x00 || chunk i, the RFC 6962 leaf hash.
+template <int SEG, int STAGES, int NSLOT, int MODE, bool RAGGED, int PAIR = 1, bool PREFIX = false>
 __global__ void __launch_bounds__(64)
 hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                          uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
@@ -96,7 +98,8 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     }
     // SHA-256 blocks of this lane's message, padding included.  For chunks lane 0 holds the longest
     // message of the warp; for tensors the maximum is taken.
-    const uint64_t my_total = !valid ? 0 : (finishing ? ((len + 8) >> 6) + 1 : (len >> 6));
+    static_assert(!(PREFIX && RAGGED), "the prefixed leaf hash is for chunks");
+    const uint64_t my_total = !valid ? 0 : (finishing ? ((len + (PREFIX ? 1 : 0) + 8) >> 6) + 1 : (len >> 6));
     const uint64_t warp_total = RAGGED ? warp_max_u64(my_total) : __shfl_sync(0xffffffffu, my_total, 0);
 
     if (warp == 1) {
@@ -129,6 +132,7 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
             if ((uint64_t)s < nseg) issue(s, s);
 
         uint32_t w[16], raw[17], tw[32];
+        uint32_t carry = 0u;                          // PREFIX: the data word before the block (byte 3 of 0 = the prefix)
         int stage = 0, in_stage = 0;
         uint32_t dparity = 0;
         bool failed = false, tail_built = false;
@@ -153,11 +157,19 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
         uint32_t eparity = 1;                         // first pass over the slots finds them empty
         for (uint64_t blk = 0; blk < warp_total && !failed; ++blk) {
             if (blk < my_full) {
+                if (PREFIX) {
+                    w[0] = shifted_word(raw[0], carry);
 #pragma unroll
-                for (int k = 0; k < 16; ++k) w[k] = RAGGED ? __byte_perm(raw[k], raw[k + 1], sel) : bswap32(raw[k]);
+                    for (int k = 1; k < 16; ++k) w[k] = shifted_word(raw[k], raw[k - 1]);
+                    carry = raw[15];
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) w[k] = RAGGED ? __byte_perm(raw[k], raw[k + 1], sel) : bswap32(raw[k]);
+                }
             } else if (blk < my_total) {
                 if (!tail_built) {
-                    (void)sha256_build_tail(p + full_bytes, (uint32_t)(len & 63u), done_before + len, tw);
+                    if (PREFIX) (void)prefixed_tail(p, 0x00, full_bytes, len + 1, tw);
+                    else (void)sha256_build_tail(p + full_bytes, (uint32_t)(len & 63u), done_before + len, tw);
                     tail_built = true;
                 }
                 const int t = (int)(blk - my_full);
@@ -243,15 +255,16 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
 
 cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status,
-                                     const uint32_t *d_one, cudaStream_t stream) {
+                                     const uint32_t *d_one, cudaStream_t stream, bool zero_prefix) {
     // 512-byte segments, three data stages, three W+K slots of two blocks each (two blocks per hand-over
     // halve the barrier traffic: +1 % over four single-block slots; 104 KB per CTA, two CTAs per SM); the additions that close the two state
     // recurrences stay three-input ALU adds, the others go to the FMA pipe (placement 3, the fastest measured).
     constexpr int SEG = 512, STAGES = 3, NSLOT = 3, MODE = 3, PAIR = 2;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
-    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false, PAIR>;
-    static bool configured[kMaxDevices] = {};
-    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
+    auto kernel = zero_prefix ? hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false, PAIR, true>
+                              : hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false, PAIR, false>;
+    static bool configured[2][kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured[zero_prefix ? 1 : 0]); e0 != cudaSuccess) return e0;
     const uint64_t blocks = (n_chunks + 31) / 32;
     if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
     kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,

@@ -134,6 +134,13 @@ cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, u
                                        void *d_slice_scratch, cudaStream_t stream, uint64_t *launches,
                                        const char **kernel_used) {
     if (n_chunks == 0) return cudaSuccess;
+    const bool aligned = ((reinterpret_cast<uintptr_t>(d_data) & 15u) == 0) && (chunk_bytes % 16u == 0);
+    if (aligned && chunk_bytes >= 4096 && (n_chunks + 31) / 32 <= 2ull * (uint64_t)sm_count) {
+        // few chains: the two-warp kernel, prefixed
+        if (launches) ++*launches;
+        if (kernel_used) *kernel_used = "hash_chunks_split_kernel";
+        return launch_hash_chunks_split(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one, stream, true);
+    }
     if (d_slice_scratch && hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count)) {
         if (launches) *launches += 2;
         if (hash_chunks_wants_pairs(d_data, chunk_bytes, n_chunks, sm_count)) {

@@ -43,7 +43,7 @@ bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint6
 // (schedule producer + round consumer), for launches with few chains.
 cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status,
-                                     const uint32_t *d_one, cudaStream_t stream);
+                                     const uint32_t *d_one, cudaStream_t stream, bool zero_prefix = false);
 
 // hash_chunks_sliced.cu -----------------------------------------------------
 // Same result for many chunks of at least 32 KiB (16-byte aligned): chunks are cut into slices

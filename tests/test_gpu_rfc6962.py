@@ -46,6 +46,8 @@ def test_leaf_hashes_equal_oracle(ctx, nbytes, chunk):
     groups = -(-binding.n_chunks(nbytes, chunk) // 32)
     if chunk >= 4096 and chunk % 16 == 0 and 296 < groups < 424:
         assert ctx.last_leaf_kernel == "hash_chunks_pairs_kernel"
+    if chunk >= 4096 and chunk % 16 == 0 and groups <= 296:
+        assert ctx.last_leaf_kernel == "hash_chunks_split_kernel"
     want = oracle.hash_chunks_rfc6962(_host(data), chunk, nthreads=oracle.host_threads())
     assert got.shape == want.shape
     assert np.array_equal(_host(got), want)
