@@ -10,10 +10,11 @@
 // global memory between slices, so the groups take turns on the pairs and all of them advance at
 // 2 x SMs / G of the two-warp rate -- more than one warp each could give them as long as G < 3.05 x SMs.
 //
-// Both warps of a pair work on the same task: lane 0 of the consumer takes the ticket and hands the
-// task to the producer through shared memory at a CTA barrier.  The data ring, the W+K ring and their
-// barrier phases carry over from task to task (every task drains what it requested).  All waits are
-// bounded.
+// Both warps of a pair work on the same task.  The producer, which runs up to six blocks ahead of the
+// consumer, takes the tickets: while the consumer finishes a slice the producer already waits for the next
+// group, starts its copies and forms its first blocks; it hands the task to the consumer through a small ring
+// in shared memory (one mbarrier per entry).  The data ring, the W+K ring and their barrier phases carry over
+// from task to task (every task drains what it requested).  All waits are bounded.
 #include "iv_internal.h"
 #include "rfc6962_dev.cuh"
 #include "sha256_dev.cuh"
@@ -42,7 +43,10 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     constexpr uint32_t kWkSlot = PAIR * kWkBlock;
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ __align__(8) uint64_t bars[STAGES + 2 * NSLOT];
-    __shared__ unsigned long long s_task[2];
+    constexpr int kTaskRing = 8;                          // more than the producer's largest lead in blocks
+    static_assert(NSLOT * PAIR < kTaskRing, "a task has at least one block");
+    __shared__ unsigned long long s_task[kTaskRing];
+    __shared__ __align__(8) uint64_t task_bars[kTaskRing];
     __shared__ uint32_t s_failed;
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;    // warp 0 consumer, warp 1 producer
@@ -53,6 +57,7 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     const uint32_t bar_empty = bar_full + 8 * NSLOT;
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES + 2 * NSLOT; ++s) tma::mbar_init(bar_data + 8 * s, 1);
+        for (int s = 0; s < kTaskRing; ++s) tma::mbar_init(tma::smem_u32(&task_bars[s]), 1);
         tma::fence_barrier_init();
         s_failed = 0u;
     }
@@ -68,32 +73,38 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     bool failed = false;
 
     for (uint32_t turn = 0;; ++turn) {
-        // ---- the consumer's lane 0 takes a ticket and waits for the group that is pushed under it
-        if (threadIdx.x == 0) {
-            unsigned long long task = kTaskDone;
-            if (*reinterpret_cast<volatile uint32_t *>(&s_failed)) {
-                task = kTaskFailed;
-            } else {
-                const unsigned long long t = atomicAdd(&q->head, 1ull);
-                if (t < total_tasks) {
-                    uint32_t entry = ld_acquire_u32(slot + t);
-                    if (entry == 0) {
-                        const long long t0 = clock64();
-                        unsigned ns = 64;
-                        while ((entry = ld_acquire_u32(slot + t)) == 0) {
-                            if (clock64() - t0 > 8000000000ll) break;       // about four seconds: give up
-                            __nanosleep(ns);
-                            if (ns < 2048) ns *= 2;
+        // ---- the producer's lane 0 takes a ticket and waits for the group that is pushed under it
+        unsigned long long task = kTaskDone;
+        const uint32_t task_bar = tma::smem_u32(&task_bars[turn % kTaskRing]);
+        if (warp == 1) {
+            if (lane == 0) {
+                if (*reinterpret_cast<volatile uint32_t *>(&s_failed)) {
+                    task = kTaskFailed;
+                } else {
+                    const unsigned long long t = atomicAdd(&q->head, 1ull);
+                    if (t < total_tasks) {
+                        uint32_t entry = ld_acquire_u32(slot + t);
+                        if (entry == 0) {
+                            const long long t0 = clock64();
+                            unsigned ns = 64;
+                            while ((entry = ld_acquire_u32(slot + t)) == 0) {
+                                if (clock64() - t0 > 8000000000ll) break;       // about four seconds: give up
+                                __nanosleep(ns);
+                                if (ns < 2048) ns *= 2;
+                            }
                         }
+                        if (entry == 0) task = kTaskFailed;
+                        else task = ((unsigned long long)(entry - 1u) << 32) | __ldcg(next_slice + (entry - 1u));
                     }
-                    if (entry == 0) task = kTaskFailed;
-                    else task = ((unsigned long long)(entry - 1u) << 32) | __ldcg(next_slice + (entry - 1u));
                 }
+                s_task[turn % kTaskRing] = task;
+                tma::mbar_arrive(task_bar);        // releases the task (and, through the acquire above, the parked values)
             }
-            s_task[turn & 1u] = task;
+            task = __shfl_sync(0xffffffffu, task, 0);
+        } else {
+            if (!tma::mbar_wait_bounded(task_bar, (turn / kTaskRing) & 1u)) { failed = true; break; }
+            task = *reinterpret_cast<volatile unsigned long long *>(&s_task[turn % kTaskRing]);
         }
-        __syncthreads();           // hands the task to both warps; also orders the parked values after the acquire
-        const unsigned long long task = s_task[turn & 1u];
         if (task == kTaskDone) break;
         if (task == kTaskFailed) { failed = true; break; }
         const uint64_t g = task >> 32;
