@@ -276,10 +276,10 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
 }  // namespace
 
 bool hash_chunks_wants_pairs(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count) {
-    // 570 GB/s flat for the pairs against 1.345 GB/s per group for one whole-compression warp per group:
-    // measured crossover at 424 groups = 2.865 x SMs, for chunks of 64 KiB to 4 MiB
+    // 580 GB/s flat for the pairs against 1.345 GB/s per group for one whole-compression warp per group:
+    // measured crossover at 431 groups = 2.91 x SMs, for chunks of 64 KiB to 4 MiB
     return hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count) &&
-           ((n_chunks + 31) / 32) * 1000ull < 2865ull * (uint64_t)sm_count;
+           ((n_chunks + 31) / 32) * 100ull < 291ull * (uint64_t)sm_count;
 }
 
 cudaError_t launch_hash_chunks_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
