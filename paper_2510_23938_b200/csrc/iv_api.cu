@@ -673,7 +673,7 @@ int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_win
             // of every chunk, one strided copy) and part s is hashed, from the chaining values part s - 1 left,
             // while part s + 1 is on its way: what remains after the last byte is one part's time.
             const uint64_t m = chunk_count(bytes, chunk);
-            const uint64_t parts = chunk / 16384 < 8 ? chunk / 16384 : 8;       // parts of at least 16 KiB
+            const uint64_t parts = chunk / 16384 < 16 ? chunk / 16384 : 16;     // parts of at least 16 KiB
             if (parts >= 2 && chunk < (1ull << 31) && m <= 2ull * 32 * (uint64_t)ctx->sm_count && m <= ivk::kRaggedSortMax) {
                 rc = hash_window_in_columns(ctx, h_windows[w], bytes, chunk, m, (uint32_t)parts, b,
                                             ctx->d_digests + 32 * w * chunks_per_window, stream);
