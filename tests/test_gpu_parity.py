@@ -420,7 +420,7 @@ def test_streamed_verification_equals_resident(ctx, pinned):
     (32768, 40, 100, 16, True),             # two column parts of 16 KiB per chunk
     (65536, 64, 0, 64, True), (3 * 16384 + 4096 + 48, 21, 5, 5, False),   # four parts; three parts, odd chunk size
     (131072, 37, 1000, 8, True),            # eight column parts per chunk, five windows, short last chunk
-    (1 << 20, 19, 77, 4, True),             # eight parts, a last chunk that ends inside a block
+    (1 << 20, 19, 77, 4, True),             # sixteen parts, a last chunk that ends inside a block
     (1 << 20, 19, 77, 19, False),           # one window, pageable host memory
     (5 * 65536 + 64, 11, 0, 3, True),       # a chunk size that is no multiple of 4 KiB: the last part is longer
     (200_008, 9, 199_990, 4, True),         # no multiple of 16; the short last chunk has 18 bytes
