@@ -589,7 +589,7 @@ def main():
                          "separately named leaf definition; not the default)")
     ap.add_argument("--variant", default="sha256", choices=["sha256", "rfc6962", "sha384"],
                     help="sha256 = the default path; rfc6962 = 0x00/0x01-prefixed tree (verification in that mode); "
-                         "sha384 = SHA-384 leaves and tree (hash + root, no manifest compare). Not the graded line.")
+                         "sha384 = SHA-384 leaves and tree (hash + root). Not the graded line.")
     ap.add_argument("--dist-backend", default="nccl", help="torch.distributed backend for --gpus > 1")
     ap.add_argument("--same-device", action="store_true",
                     help="put every rank on cuda:0 (only to check the multi-rank logic on a one-GPU box, with gloo)")

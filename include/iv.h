@@ -321,6 +321,26 @@ int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint
 int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
                           void *cuda_stream);
 
+/* iv_verify_manifest for this variant: the same steps over 48-byte records.  The manifest holds the
+ * SHA-384 chunk digests (device) and the root of the SHA-384 tree; fields, index list, errors and
+ * asynchrony as for iv_manifest / iv_verify_result / iv_verify_manifest. */
+typedef struct iv_manifest_sha384 {
+    uint64_t total_bytes;
+    uint64_t chunk_bytes;
+    uint64_t n_chunks;
+    const uint8_t *d_digests; /* DEVICE: n_chunks * 48 bytes */
+    uint8_t root[48];
+} iv_manifest_sha384;
+typedef struct iv_verify_result_sha384 {
+    uint32_t status;
+    uint32_t root_ok;
+    uint64_t n_mismatch;
+    uint8_t root[48];
+} iv_verify_result_sha384;
+int iv_verify_manifest_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
+                              const iv_manifest_sha384 *h_manifest, iv_verify_result_sha384 *d_result,
+                              uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------
  * RFC 6962 section 2.1 mode -- the Merkle Tree Hash the paper cites for its tree,
  * with that RFC's domain separation, over SHA-256 with the chunks as entries:

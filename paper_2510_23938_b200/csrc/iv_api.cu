@@ -44,6 +44,8 @@ struct iv_ctx {
     uint64_t slices_cap = 0;                  // bytes
 
     // streaming windows
+    uint8_t *d_digests384 = nullptr;          // chunk digests of iv_verify_manifest_sha384, then its 48-byte root
+    uint64_t digests384_cap = 0;              // records of 48 bytes
     uint8_t *d_columns = nullptr;             // offsets, lengths and chaining values of a window hashed in column parts
     uint64_t columns_cap = 0;                 // bytes
     uint8_t *d_window[2] = {nullptr, nullptr};
@@ -322,6 +324,7 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_order);
     cudaFree(ctx->d_dirty_scratch);
     cudaFree(ctx->d_columns);
+    cudaFree(ctx->d_digests384);
     cudaFree(ctx->d_sub);
     cudaFree(ctx->d_batch);
     cudaFree(ctx->d_tree384[0]);
@@ -765,6 +768,34 @@ int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leave
     if (rc != IV_OK) return rc;
     IV_TRY(ctx, ivk::launch_merkle_root_sha384(d_leaves, n_leaves, d_root, ctx->d_tree384[0], ctx->d_tree384[1],
                                                static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
+    return IV_OK;
+}
+
+int iv_verify_manifest_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest_sha384 *m,
+                              iv_verify_result_sha384 *d_result, uint64_t *d_mismatch_idx, uint64_t idx_cap,
+                              void *cuda_stream) {
+    if (!ctx || !d_result || (idx_cap && !d_mismatch_idx)) return IV_ERR_INVALID_ARG;
+    if (!m || m->chunk_bytes == 0 || m->total_bytes != nbytes) return IV_ERR_INVALID_ARG;
+    const uint64_t n = chunk_count(nbytes, m->chunk_bytes);
+    if (m->n_chunks != n || (n && !m->d_digests) || (nbytes && !d_data)) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int rc = grow(ctx, &ctx->d_digests384, &ctx->digests384_cap, n + 2, 48);      // digests, then the root
+    if (rc != IV_OK) return rc;
+    if ((rc = ensure_variant_tree_scratch(ctx, (n + 1) / 2 + 1)) != IV_OK) return rc;
+    if ((rc = grow(ctx, &ctx->d_words, &ctx->words_cap, (n + 31) / 32 + 1, sizeof(uint32_t))) != IV_OK) return rc;
+    uint8_t *d_root = ctx->d_digests384 + 48 * (n + 1);
+    IV_TRY(ctx, ivk::launch_hash_chunks_sha384(static_cast<const uint8_t *>(d_data), nbytes, m->chunk_bytes, n,
+                                               ctx->d_digests384, ctx->sm_count, stream, &ctx->launches));
+    ctx->leaf_kernel = "hash_chunks_sha384_kernel";
+    IV_TRY(ctx, ivk::launch_merkle_root_sha384(ctx->d_digests384, n, d_root, ctx->d_tree384[0], ctx->d_tree384[1], stream,
+                                               &ctx->launches));
+    ivk::RootBytes384 expect;
+    std::memcpy(expect.b, m->root, 48);
+    IV_TRY(ctx, ivk::launch_verify_compare_sha384(ctx->d_digests384, m->d_digests, n, d_root, expect, d_result,
+                                                  d_mismatch_idx, idx_cap, ctx->d_words,
+                                                  ctx->d_tickets + ivk::kMerkleMaxPasses, ctx->d_status, stream,
+                                                  &ctx->launches));
     return IV_OK;
 }
 

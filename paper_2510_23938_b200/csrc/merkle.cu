@@ -288,22 +288,27 @@ __global__ void empty_root_kernel(uint8_t *d_root) {
 // words into the ascending index list with a block-wide exclusive scan.
 // ---------------------------------------------------------------------------
 
+// REC: bytes per digest record (32 for SHA-256, 48 for SHA-384).
+template <int REC>
 __device__ __forceinline__ bool digest_differs(const uint8_t *a, const uint8_t *b, bool aligned) {
-    if (aligned) {
-        const uint4 a0 = __ldg(reinterpret_cast<const uint4 *>(a)), a1 = __ldg(reinterpret_cast<const uint4 *>(a) + 1);
-        const uint4 b0 = __ldg(reinterpret_cast<const uint4 *>(b)), b1 = __ldg(reinterpret_cast<const uint4 *>(b) + 1);
-        return ((a0.x ^ b0.x) | (a0.y ^ b0.y) | (a0.z ^ b0.z) | (a0.w ^ b0.w) |
-                (a1.x ^ b1.x) | (a1.y ^ b1.y) | (a1.z ^ b1.z) | (a1.w ^ b1.w)) != 0u;
-    }
     uint32_t diff = 0;
-    for (int i = 0; i < 32; ++i) diff |= (uint32_t)(a[i] ^ b[i]);
+    if (aligned) {
+#pragma unroll
+        for (int q = 0; q < REC / 16; ++q) {
+            const uint4 x = __ldg(reinterpret_cast<const uint4 *>(a) + q), y = __ldg(reinterpret_cast<const uint4 *>(b) + q);
+            diff |= (x.x ^ y.x) | (x.y ^ y.y) | (x.z ^ y.z) | (x.w ^ y.w);
+        }
+        return diff != 0u;
+    }
+    for (int i = 0; i < REC; ++i) diff |= (uint32_t)(a[i] ^ b[i]);
     return diff != 0u;
 }
 
+template <int REC, class Result, class Root>
 __global__ void __launch_bounds__(kThreads)
 verify_compare_kernel(const uint8_t *__restrict__ digests, const uint8_t *__restrict__ manifest, uint64_t n,
-                      const uint8_t *__restrict__ d_root, RootBytes manifest_root,
-                      iv_verify_result *__restrict__ result, uint64_t *__restrict__ idx_out, uint64_t idx_cap,
+                      const uint8_t *__restrict__ d_root, Root manifest_root,
+                      Result *__restrict__ result, uint64_t *__restrict__ idx_out, uint64_t idx_cap,
                       uint32_t *__restrict__ words, uint32_t *ticket, const uint32_t *__restrict__ dev_status) {
     __shared__ uint32_t s_last;
     __shared__ uint32_t s_warp_sum[kThreads / 32];
@@ -315,7 +320,7 @@ verify_compare_kernel(const uint8_t *__restrict__ digests, const uint8_t *__rest
     const uint64_t warps_total = (uint64_t)gridDim.x * (kThreads / 32);
     for (uint64_t wi = (uint64_t)blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); wi < n_words; wi += warps_total) {
         const uint64_t i = wi * 32 + lane;
-        const bool bad = (i < n) && digest_differs(digests + 32 * i, manifest + 32 * i, aligned);
+        const bool bad = (i < n) && digest_differs<REC>(digests + (uint64_t)REC * i, manifest + (uint64_t)REC * i, aligned);
         const uint32_t mask = __ballot_sync(0xffffffffu, bad);
         if (lane == 0) words[wi] = mask;
     }
@@ -363,7 +368,7 @@ verify_compare_kernel(const uint8_t *__restrict__ digests, const uint8_t *__rest
     }
     if (threadIdx.x == 0) {
         uint32_t diff = 0;
-        for (int i = 0; i < 32; ++i) {
+        for (int i = 0; i < REC; ++i) {
             const uint8_t r = d_root[i];
             result->root[i] = r;
             diff |= (uint32_t)(r ^ manifest_root.b[i]);
@@ -528,7 +533,23 @@ cudaError_t launch_verify_compare(const uint8_t *d_digests, const uint8_t *d_man
     uint64_t blocks = (n_words + (kThreads / 32) - 1) / (kThreads / 32);
     if (blocks == 0) blocks = 1;
     if (blocks > 1184) blocks = 1184;
-    verify_compare_kernel<<<(unsigned)blocks, kThreads, 0, stream>>>(
+    verify_compare_kernel<32, iv_verify_result, RootBytes><<<(unsigned)blocks, kThreads, 0, stream>>>(
+        d_digests, d_manifest_digests, n, d_root, manifest_root, d_result, d_mismatch_idx, idx_cap,
+        d_words, d_ticket, d_status);
+    if (launches) ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_verify_compare_sha384(const uint8_t *d_digests, const uint8_t *d_manifest_digests,
+                                         uint64_t n, const uint8_t *d_root, RootBytes384 manifest_root,
+                                         iv_verify_result_sha384 *d_result, uint64_t *d_mismatch_idx,
+                                         uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
+                                         const uint32_t *d_status, cudaStream_t stream, uint64_t *launches) {
+    const uint64_t n_words = (n + 31) / 32;
+    uint64_t blocks = (n_words + (kThreads / 32) - 1) / (kThreads / 32);
+    if (blocks == 0) blocks = 1;
+    if (blocks > 1184) blocks = 1184;
+    verify_compare_kernel<48, iv_verify_result_sha384, RootBytes384><<<(unsigned)blocks, kThreads, 0, stream>>>(
         d_digests, d_manifest_digests, n, d_root, manifest_root, d_result, d_mismatch_idx, idx_cap,
         d_words, d_ticket, d_status);
     if (launches) ++*launches;

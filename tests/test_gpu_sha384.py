@@ -87,3 +87,34 @@ def test_sha384_chunks_then_root_repeated_calls(ctx):
     # a smaller tree after a larger one reuses the level buffers
     assert _host(ctx.merkle_root_sha384(leaves[:5])).tobytes() == oracle.merkle_root_sha384(want_leaves[:5])
     assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("nbytes,chunk", [((8 << 20) + 300, 4096), (64 << 20, 64 << 10), (100_003, 1001), (5000, 8192)])
+def test_verification_against_a_sha384_manifest_from_the_oracle(ctx, nbytes, chunk):
+    """Manifest = the oracle's SHA-384 chunk digests and root: clean data passes, flipped bits are located in
+    ascending order with the exact count, the recomputed root is the oracle's root of the damaged blob."""
+    data = inputs.uniform_bytes(nbytes, seed=3840, device="cuda")
+    digests = oracle.hash_chunks_sha384(_host(data), chunk, nthreads=oracle.host_threads())
+    root = oracle.merkle_root_sha384(digests)
+    d_digests = torch.from_numpy(digests).cuda()
+    n = digests.shape[0]
+    idx = torch.zeros(4, dtype=torch.int64, device="cuda")
+    r = ctx.verify_manifest_sha384(data, nbytes, chunk, d_digests, root, idx)
+    assert r == {"status": 0, "root_ok": True, "n_mismatch": 0, "root": root}
+    bad = data.clone()
+    hits = sorted({inputs.flip_position(s, nbytes) for s in range(11, 18)})
+    for off, bit in hits:
+        bad[off] ^= (1 << bit)
+    want = oracle.hash_chunks_sha384(_host(bad), chunk, nthreads=oracle.host_threads())
+    want_idx = [i for i in range(n) if bytes(want[i]) != bytes(digests[i])]
+    assert want_idx == sorted({off // chunk for off, _ in hits})
+    r = ctx.verify_manifest_sha384(bad, nbytes, chunk, d_digests, root, idx)
+    assert (not r["root_ok"]) and r["n_mismatch"] == len(want_idx) and r["root"] == oracle.merkle_root_sha384(want)
+    assert [int(v) for v in idx[:min(4, len(want_idx))].cpu()] == want_idx[:4]
+    # manifest-side damage: one digest of the manifest changed, the data clean
+    d_digests[n // 2, 7] ^= 1
+    r = ctx.verify_manifest_sha384(data, nbytes, chunk, d_digests, root, idx)
+    assert r["root_ok"] and r["n_mismatch"] == 1 and int(idx[0]) == n // 2
+    with pytest.raises(binding.IvError):
+        ctx.verify_manifest_sha384(data, nbytes + 1, chunk, d_digests, root, idx)
+    assert ctx.device_status() == 0
