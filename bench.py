@@ -7,16 +7,22 @@ Merkle root, comparison with the manifest (`iv_verify_manifest`; for the ragged 
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl ours|reference]
 
-Multi-GPU runs are launched with torch.distributed.run, one rank per GPU; the ranks' blobs are the
-shards of one blob (weak scaling): every rank verifies its shard and the global root is built from an
-all-gather of a few 32-byte tree nodes per rank (the path's only exchange).
+`--gpus N` with N > 1 starts N ranks by itself (one per GPU, torch.distributed.run on 127.0.0.1)
+unless a launcher has already set WORLD_SIZE.  The ranks' blobs are the shards of one blob (weak
+scaling): every rank verifies its shard, the global root is built from an all-gather of a few
+32-byte tree nodes per rank and the mismatch counts are all-reduced (the path's only exchanges).
+The default single-GPU run also reports, in a `secondary` object, the 16 GB configuration (device
+resident, streamed, per-tensor digests) and the small configuration (one by one and as a batch).
 `--impl reference` times the CPU oracle (the plain restatement of the method) on the host cores.
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -35,8 +41,18 @@ MIB = 1 << 20
 # 6 SHF + 4 LOP3 + 4 IADD3, 48 schedule steps of 6 SHF + 2 LOP3 + 2 IADD3, 16 PRMT, 8 adds)
 # against 148 SMs x 64 INT32 lanes x the maximum SM clock.
 INT_OPS_PER_BYTE = 1400.0 / 64.0
+INT_OPS_PER_BYTE_SHA512 = 3568.0 / 128.0      # SHA-384 / SHA-512: 80 rounds and 64 schedule steps on 64-bit words
 INT_LANES_PER_SM = 64
 SM_COUNT = 148
+SM_HZ = 1.965e9
+PEAK_GBS = SM_COUNT * INT_LANES_PER_SM * SM_HZ / INT_OPS_PER_BYTE / 1e9
+# Cycles ONE chain needs per 64-byte block when its warps have their SM schedulers to themselves: the
+# two-warp kernel as measured on the 16 GB configuration (leaf-kernel time x clock / blocks per chunk),
+# and the issue floor of the round function (10 SHF/LOP3 per round on a 16-lane pipe, two cycles each).
+SPLIT_CYCLES_PER_BLOCK = 1965.0
+ISSUE_FLOOR_CYCLES_PER_BLOCK = 1280.0
+# DRAM read+write bytes per byte hashed, from the ncu captures summarised under profiles/.
+TRAFFIC_FACTOR = {"hash_chunks_sliced_kernel": 1.0034, "hash_chunks_split_kernel": 1.001}
 
 CONFIGS = {
     1: dict(name="config1: 64 MiB uniform random bytes, 64 KiB chunks, 1024 leaves", kind="uniform",
@@ -124,12 +140,21 @@ def _physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
+def _measured_peak(key):
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f).get(key)
+    except Exception:
+        return None
+
+
 # --------------------------------------------------------------------------------------------
 # workloads
 
 def build_workload(cfg_id: int, device, seed: int, nbytes_override=None, chunk_override=None):
     from paper_2510_23938_b200 import inputs
     cfg = dict(CONFIGS[cfg_id])
+    cfg["id"] = cfg_id
     if nbytes_override or chunk_override:
         if nbytes_override and "nbytes" in cfg:
             cfg["nbytes"] = int(nbytes_override) & ~1
@@ -174,6 +199,107 @@ def pick_config(requested: int | None, device) -> tuple[int, str | None]:
 
 
 # --------------------------------------------------------------------------------------------
+# timing
+
+def time_steps(step, steps: int, warmup: int, flush, gpu_index: int, dist=None):
+    """`warmup` untimed calls of step(), then `steps` timed ones (CUDA events on the current stream, the
+    region bracketed by synchronisation and, with several ranks, barriers).  With `flush` (a device buffer
+    larger than L2) the buffer is rewritten before every timed step and the steps are timed one by one.
+    Returns (total milliseconds, maximum over ranks; the clock record of the timed region)."""
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    with ClockSampler(gpu_index) as clocks:
+        for k in range(steps):
+            if flush is not None:
+                flush.fill_(k & 0xFF)
+            starts[k].record(stream)
+            step()
+            ends[k].record(stream)
+        torch.cuda.synchronize()
+    if flush is not None:
+        total_ms = float(sum(s.elapsed_time(e) for s, e in zip(starts, ends)))
+    else:
+        total_ms = float(starts[0].elapsed_time(ends[-1]))
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64)
+        if dist.get_backend() == "nccl":
+            t = t.to(torch.device("cuda", torch.cuda.current_device()))
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        dist.barrier()
+    return total_ms, clocks.summary()
+
+
+def roofline_of(kernel_name: str, nbytes: int, hash_ms: float, chains: int, tree_ms=None, cmp_ms=None):
+    achieved = nbytes / (hash_ms * 1e-3) / 1e9
+    factor = TRAFFIC_FACTOR.get(kernel_name.split(" ")[0])
+    split = kernel_name.startswith("hash_chunks_split_kernel")
+    chain_bound = chains * 64 * SM_HZ / SPLIT_CYCLES_PER_BLOCK / 1e9
+    floor_bound = chains * 64 * SM_HZ / ISSUE_FLOOR_CYCLES_PER_BLOCK / 1e9
+    return {
+        "bound": "alu", "kernel": kernel_name,
+        "achieved": round(achieved, 2), "peak": round(PEAK_GBS, 1), "unit": "GB/s",
+        "frac": round(achieved / PEAK_GBS, 4),
+        "traffic": int(factor * nbytes) if factor else None,
+        "traffic_source": ("ncu dram bytes of a smaller capture of the same kernel, scaled by bytes hashed "
+                           "(profiles/)") if factor else None,
+        "algorithmic_bytes": nbytes, "int32_ops_per_byte": INT_OPS_PER_BYTE,
+        # what the chain count allows: chains x 64 B x f / (cycles one chain needs per block)
+        "chain_count_bound_gbs": round(min(chain_bound, PEAK_GBS), 1),
+        "chain_count_bound_at_issue_floor_gbs": round(min(floor_bound, PEAK_GBS), 1),
+        "cycles_per_block_assumed": SPLIT_CYCLES_PER_BLOCK if split else None,
+        "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1.965 GHz / 21.875 INT32 ops per byte",
+        "hbm_peak_gbs_measured": _measured_peak("hbm_gbs"),
+        "launch_ms": round(hash_ms, 4), "tree_ms": tree_ms, "compare_ms": cmp_ms,
+        "chains": chains,
+    }
+
+
+def measure_verify(ctx, wl, device, steps, warmup, gpu_index, flush=None, dist=None, extra_step=None):
+    """The default path on a device-resident blob: `iv_verify_manifest` per step, the manifest made from the
+    blob itself beforehand.  Returns the figures of one JSON object plus the manifest pieces."""
+    from paper_2510_23938_b200 import binding
+    data, nbytes, chunk = wl["data"], wl["nbytes"], wl["chunk"]
+    n_units = binding.n_chunks(nbytes, chunk)
+    man_digests = ctx.hash_chunks(data, chunk)
+    man_root = bytes(ctx.merkle_root(man_digests).cpu().numpy().tobytes())
+    manifest = ctx.make_manifest(nbytes, chunk, man_digests, man_root)
+    result = binding.new_result(device)
+    idx = torch.zeros(64, dtype=torch.int64, device=device)
+
+    def step():
+        ctx.verify_manifest(data, manifest, result, idx)
+        if extra_step is not None:
+            extra_step(result)
+
+    ctx.set_timing(True)
+    launches0 = ctx.kernel_launches
+    total_ms, clocks = time_steps(step, steps, warmup, flush, gpu_index, dist)
+    launches = (ctx.kernel_launches - launches0) * steps // (steps + warmup)
+    ctx.set_timing(False)
+    k = min(steps, 64)
+    hash_ms = float(np.mean([ctx.phase_times(j)[0] for j in range(k)]))
+    tree_ms = float(np.mean([ctx.phase_times(j)[1] for j in range(k)]))
+    cmp_ms = float(np.mean([ctx.phase_times(j)[2] for j in range(k)]))
+    # the benchmark number counts only if the timed launches verified the blob: read the last step's result
+    r = binding.read_result(result)
+    status = ctx.device_status()
+    ok = bool(r["root_ok"] and r["n_mismatch"] == 0 and r["status"] == 0 and status == 0 and r["root"] == man_root)
+    ms_per_step = total_ms / steps
+    return {
+        "ms_per_step": ms_per_step, "gbs": nbytes / (ms_per_step * 1e-3) / 1e9, "clocks": clocks, "launches": int(launches),
+        "roofline": roofline_of(ctx.last_leaf_kernel, nbytes, hash_ms, n_units, tree_ms, cmp_ms),
+        "verified_ok": ok, "man_digests": man_digests, "man_root": man_root, "manifest": manifest, "n_units": n_units,
+    }
+
+
+# --------------------------------------------------------------------------------------------
 # our arm
 
 def run_ours(args):
@@ -183,14 +309,20 @@ def run_ours(args):
     world = _env_int("WORLD_SIZE", 1)
     rank = _env_int("RANK", 0)
     local_rank = _env_int("LOCAL_RANK", 0)
+    if args.gpus != world:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    if not args.same_device and torch.cuda.device_count() < _env_int("LOCAL_WORLD_SIZE", world):
+        raise SystemExit(f"bench.py: {world} ranks need {world} GPUs, {torch.cuda.device_count()} visible "
+                         "(--same-device puts every rank on cuda:0 to check the multi-rank logic)")
     if rank == 0 and iv_build.is_stale():
         iv_build.build()
     if args.same_device:                     # checking the multi-rank logic on a box with one GPU (with gloo)
         local_rank = 0
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
+    gpu_index = _physical_gpu_index(local_rank)
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -209,169 +341,134 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     ragged = wl["kind"] == "ragged"
-    if ragged:
-        d_off = torch.from_numpy(wl["offsets"]).to(device)
-        d_len = torch.from_numpy(wl["lengths"]).to(device)
-        n_units = int(d_off.numel())
-        digests = torch.empty((n_units, 32), dtype=torch.uint8, device=device)
-        root = torch.empty(32, dtype=torch.uint8, device=device)
+    copies = args.batch if (not ragged and args.batch and args.batch > 1) else 1
+    plain = (not ragged) and copies == 1 and args.variant == "sha256" and not args.two_level
+    # L2 (126 MB): every workload but config 1 is far larger than L2; config 1 gets a flush between steps.
+    flush = torch.empty(256 * MIB, dtype=torch.uint8, device=device) if nbytes < 512 * MIB else None
+    shard_plan, parallelism, verified_ok, extra = None, f"independent blob per GPU x{world}", None, {}
 
-        def step():
-            ctx.hash_ragged(data, d_off, d_len, out=digests)
-            ctx.merkle_root(digests, out=root)
-    else:
-        n_units = binding.n_chunks(nbytes, chunk)
-        two_level = args.two_level
-        variant = args.variant
-        if variant == "rfc6962":
-            man_digests = ctx.hash_chunks_rfc6962(data, chunk)
-            man_root = bytes(ctx.merkle_root_rfc6962(man_digests).cpu().numpy().tobytes())
-        else:
-            man_digests = ctx.hash_chunks_two_level(data, chunk, two_level) if two_level else ctx.hash_chunks(data, chunk)
-            man_root = bytes(ctx.merkle_root(man_digests).cpu().numpy().tobytes())
-        manifest = ctx.make_manifest(nbytes, chunk, man_digests, man_root)
-        result = binding.new_result(device)
-        idx = torch.zeros(64, dtype=torch.int64, device=device)
-
+    if plain:
         # Several GPUs: the ranks' blobs are the shards of ONE blob of world x nbytes.  Each step then also
-        # builds the global root: local digests -> k levels -> all-gather of the few level-k nodes (32 bytes
-        # each, the path's only exchange) -> root, on every rank.
-        shard_plan = None
-        if world > 1 and args.variant == "sha256":
+        # builds the global root (local digests -> k levels -> all-gather of the few level-k nodes, 32 bytes
+        # each -> root, on every rank) and all-reduces the mismatch count: the path's only exchanges.
+        n_units = binding.n_chunks(nbytes, chunk)
+        extra_step = None
+        if world > 1:
             from paper_2510_23938_b200 import sharded
             shard_plan = sharded.plan_shards(world * n_units, world, min_nodes_per_rank=64)
             lo, hi = shard_plan.leaf_ranges[rank]
             if hi - lo != n_units or nbytes % chunk:
                 shard_plan = None                       # uneven cut: fall back to independent blobs
+        if shard_plan is not None:
+            state = {}
 
-        batch_blobs = None
-        if args.batch and args.batch > 1:
-            from paper_2510_23938_b200 import inputs as _inputs
-            batch_blobs = [data]
-            for k in range(1, args.batch):
-                off, bit = _inputs.flip_position(1 + k, nbytes)
-                bad = data.clone()
-                bad[off] ^= (1 << bit)
-                batch_blobs.append(bad)
-            batch_results = torch.zeros((args.batch, 48), dtype=torch.uint8, device=device)
-            batch_idx = torch.zeros((args.batch, 8), dtype=torch.int64, device=device)
-
-        def step():
-            if batch_blobs is not None:
-                ctx.verify_manifest_batch(batch_blobs, manifest, batch_results, batch_idx)
-                return
-            if variant == "sha384":
-                ctx.merkle_root_sha384(ctx.hash_chunks_sha384(data, chunk))
-            elif variant == "rfc6962":
-                ctx.verify_manifest_rfc6962(data, manifest, result, idx)
-            elif two_level:
-                ctx.verify_manifest_two_level(data, manifest, two_level, result, idx)
-            else:
-                ctx.verify_manifest(data, manifest, result, idx)
-            if shard_plan is not None:
-                sharded.sharded_root(ctx, ctx.last_digests(n_units), shard_plan, rank)
+            def extra_step(result):
+                state["root"] = sharded.sharded_root(ctx, ctx.last_digests(n_units), shard_plan, rank)
+                state["bad"] = sharded.count_mismatches(result[8:16].view(torch.int64), device)
+        m = measure_verify(ctx, wl, device, args.steps, args.warmup, gpu_index, flush, dist, extra_step)
+        total_ms, clocks, launches = m["ms_per_step"] * args.steps, m["clocks"], m["launches"]
+        roofline, verified_ok, man_digests = m["roofline"], m["verified_ok"], m["man_digests"]
         if shard_plan is not None:
             global_root = sharded.sharded_root(ctx, man_digests, shard_plan, rank)
-    torch.cuda.synchronize()
-    setup_s = time.time() - t_setup
-
-    # L2 (126 MB): every workload but config 1 is far larger than L2; config 1 gets a flush between steps.
-    flush = torch.empty(256 * MIB, dtype=torch.uint8, device=device) if nbytes < 512 * MIB else None
-
-    ctx.set_timing(True)
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    launches0 = ctx.kernel_launches
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    with ClockSampler(_physical_gpu_index(local_rank)) as clocks:
-        for k in range(args.steps):
-            if flush is not None:
-                flush.fill_(k & 0xFF)
-            starts[k].record(stream)
-            step()
-            ends[k].record(stream)
-        torch.cuda.synchronize()
-    launches = ctx.kernel_launches - launches0
-    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
-    total_ms = float(sum(step_ms)) if flush is not None else float(starts[0].elapsed_time(ends[-1]))
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-        dist.barrier()
-    ctx.set_timing(False)
-
-    # dominant kernel: the leaf-hashing launch, timed by the library's own events inside the timed steps
-    if not ragged and args.variant == "sha384":
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        ctx.hash_chunks_sha384(data, chunk)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        hash_ms, tree_ms, cmp_ms = float(e0.elapsed_time(e1)), None, None
-    elif ragged or (args.batch and args.batch > 1):
-        hash_ms = None
+            verified_ok = bool(verified_ok and torch.equal(state["root"], global_root) and int(state["bad"].item()) == 0)
+            parallelism = (f"one blob of {world} shards, global root by all-gather of {shard_plan.n_nodes} "
+                           f"level-{shard_plan.level} nodes, mismatch count all-reduced")
+            extra["global_root"] = bytes(global_root.cpu().numpy().tobytes()).hex()
     else:
-        hash_ms = float(np.mean([ctx.phase_times(k)[0] for k in range(min(args.steps, 64))]))
-        tree_ms = float(np.mean([ctx.phase_times(k)[1] for k in range(min(args.steps, 64))]))
-        cmp_ms = float(np.mean([ctx.phase_times(k)[2] for k in range(min(args.steps, 64))]))
+        if ragged:
+            d_off = torch.from_numpy(wl["offsets"]).to(device)
+            d_len = torch.from_numpy(wl["lengths"]).to(device)
+            n_units = int(d_off.numel())
+            digests = torch.empty((n_units, 32), dtype=torch.uint8, device=device)
+            root = torch.empty(32, dtype=torch.uint8, device=device)
 
-    if not ragged and args.batch and args.batch > 1:
-        hash_ms, tree_ms, cmp_ms = total_ms / args.steps / args.batch, None, None   # whole step per copy (no phase events here)
-        out_batch = [r for r in binding.read_results(batch_results)]
-    if ragged:
-        # time the hashing launch alone, same launch configuration, for the roofline line
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        ctx.hash_ragged(data, d_off, d_len, out=digests)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        hash_ms, tree_ms, cmp_ms = float(e0.elapsed_time(e1)), None, None
+            def step():
+                ctx.hash_ragged(data, d_off, d_len, out=digests)
+                ctx.merkle_root(digests, out=root)
+        else:
+            n_units = binding.n_chunks(nbytes, chunk)
+            two_level, variant = args.two_level, args.variant
+            if variant == "rfc6962":
+                man_digests = ctx.hash_chunks_rfc6962(data, chunk)
+                man_root = bytes(ctx.merkle_root_rfc6962(man_digests).cpu().numpy().tobytes())
+            elif variant in ("sha384", "sha512"):
+                man_digests, man_root = None, None
+            else:
+                man_digests = ctx.hash_chunks_two_level(data, chunk, two_level) if two_level else ctx.hash_chunks(data, chunk)
+                man_root = bytes(ctx.merkle_root(man_digests).cpu().numpy().tobytes())
+            if man_digests is not None:
+                manifest = ctx.make_manifest(nbytes, chunk, man_digests, man_root)
+            result = binding.new_result(device)
+            idx = torch.zeros(64, dtype=torch.int64, device=device)
+            if copies > 1:
+                from paper_2510_23938_b200 import inputs as _inputs
+                batch_blobs = [data]
+                for k in range(1, copies):
+                    off, bit = _inputs.flip_position(1 + k, nbytes)
+                    bad = data.clone()
+                    bad[off] ^= (1 << bit)
+                    batch_blobs.append(bad)
+                batch_results = torch.zeros((copies, 48), dtype=torch.uint8, device=device)
+                batch_idx = torch.zeros((copies, 8), dtype=torch.int64, device=device)
+
+            def step():
+                if copies > 1:
+                    ctx.verify_manifest_batch(batch_blobs, manifest, batch_results, batch_idx)
+                elif variant == "sha384":
+                    ctx.merkle_root_sha384(ctx.hash_chunks_sha384(data, chunk))
+                elif variant == "sha512":
+                    ctx.merkle_root_sha512(ctx.hash_chunks_sha512(data, chunk))
+                elif variant == "rfc6962":
+                    ctx.verify_manifest_rfc6962(data, manifest, result, idx)
+                else:
+                    ctx.verify_manifest_two_level(data, manifest, two_level, result, idx)
+        ctx.set_timing(True)
+        launches0 = ctx.kernel_launches
+        total_ms, clocks = time_steps(step, args.steps, args.warmup, flush, gpu_index, dist)
+        launches = (ctx.kernel_launches - launches0) * args.steps // (args.steps + args.warmup)
+        ctx.set_timing(False)
+        tree_ms = cmp_ms = None
+        if ragged or (not ragged and args.variant in ("sha384", "sha512")):
+            # time the hashing launch alone, same launch configuration, for the roofline line
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            if ragged:
+                ctx.hash_ragged(data, d_off, d_len, out=digests)
+            elif args.variant == "sha384":
+                ctx.hash_chunks_sha384(data, chunk)
+            else:
+                ctx.hash_chunks_sha512(data, chunk)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            hash_ms = float(e0.elapsed_time(e1))
+            verified_ok = ctx.device_status() == 0
+        elif copies > 1:
+            hash_ms = total_ms / args.steps / copies          # whole step per copy (no phase events here)
+            out_batch = binding.read_results(batch_results)
+            verified_ok = bool(ctx.device_status() == 0 and out_batch[0]["root_ok"] and out_batch[0]["n_mismatch"] == 0
+                               and all((not r["root_ok"]) and r["n_mismatch"] == 1 for r in out_batch[1:]))
+        else:
+            k = min(args.steps, 64)
+            hash_ms = float(np.mean([ctx.phase_times(j)[0] for j in range(k)]))
+            tree_ms = float(np.mean([ctx.phase_times(j)[1] for j in range(k)]))
+            cmp_ms = float(np.mean([ctx.phase_times(j)[2] for j in range(k)]))
+            r = binding.read_result(result)
+            verified_ok = bool(r["root_ok"] and r["n_mismatch"] == 0 and r["status"] == 0 and ctx.device_status() == 0)
+        roofline = roofline_of(ctx.last_leaf_kernel, nbytes, hash_ms, n_units, tree_ms, cmp_ms)
+    torch.cuda.synchronize()
+    setup_s = time.time() - t_setup - total_ms * 1e-3
 
     ms_per_step = total_ms / args.steps
-    copies = args.batch if (not ragged and args.batch and args.batch > 1) else 1
     value = world * copies * nbytes / (ms_per_step * 1e-3) / 1e9
-
-    peak_gbs = SM_COUNT * INT_LANES_PER_SM * 1.965e9 / INT_OPS_PER_BYTE / 1e9
-    achieved = nbytes / (hash_ms * 1e-3) / 1e9
-    # DRAM traffic per launch: ncu measured dram read+write = 1.0034 x the bytes hashed for the sliced kernel
-    # (2 GiB capture) and 1.001 x for the two-warp kernel (config 2 capture); both scale with the bytes.
-    kernel_name = ctx.last_leaf_kernel
-    traffic_factor = {"hash_chunks_sliced_kernel": 1.0034, "hash_chunks_split_kernel": 1.001}.get(kernel_name)
-    # what the chain count allows: chains x 64 B x f / (cycles one chain needs per block when it has a
-    # scheduler to itself: 2,000 for the two-warp kernel)
-    chain_bound = n_units * 64 * 1.965e9 / 2000.0 / 1e9
-    roofline = {
-        "bound": "alu", "kernel": kernel_name,
-        "achieved": round(achieved, 2), "peak": round(peak_gbs, 1), "unit": "GB/s",
-        "frac": round(achieved / peak_gbs, 4),
-        "traffic": int(traffic_factor * nbytes) if traffic_factor else None,
-        "traffic_source": ("ncu dram bytes of a smaller capture of the same kernel, scaled by bytes hashed "
-                           "(profiles/)") if traffic_factor else None,
-        "algorithmic_bytes": nbytes, "int32_ops_per_byte": INT_OPS_PER_BYTE,
-        "chain_count_bound_gbs": round(min(chain_bound, peak_gbs), 1),
-        "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1.965 GHz / 21.875 INT32 ops per byte",
-        "hbm_peak_gbs_measured": _measured_peak("hbm_gbs"),
-        "launch_ms": round(hash_ms, 4), "tree_ms": tree_ms, "compare_ms": cmp_ms,
-        "chains": n_units,
-    }
-
     out = {
         "metric": "GB/s verified (SHA-256 chunks + Merkle root + manifest compare) at 1 B200",
-        "value": round(value, 3), "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u32", "data": "synthetic",
+        "value": round(value, 3) if verified_ok else None, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u32", "data": "synthetic", "verified_ok": verified_ok,
         "config": {"workload": wl["name"], "bytes_per_gpu": nbytes, "chunk_bytes": chunk, "units": n_units,
                    "l2": "inputs larger than L2" if flush is None else "L2 flushed between steps (256 MiB write)",
-                   "parallelism": (f"independent blob per GPU x{world}" if world == 1 or ragged or shard_plan is None else
-                                   f"one blob of {world} shards, global root by all-gather of "
-                                   f"{shard_plan.n_nodes} level-{shard_plan.level} nodes"),
-                   "setup_s": round(setup_s, 1)},
-        "clocks": clocks.summary(), "gpu_launches": int(launches), "roofline": roofline,
+                   "parallelism": parallelism, "setup_s": round(setup_s, 1), **extra},
+        "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline,
     }
     if fallback:
         out["config"]["fallback"] = fallback
@@ -379,14 +476,16 @@ def run_ours(args):
         out["config"]["batch"] = (f"{copies} copies verified in one pass (iv_verify_manifest_batch); mismatches per copy: "
                                   f"{[r['n_mismatch'] for r in out_batch]}; roofline figures are per whole step")
     if not ragged and args.variant != "sha256":
-        out["config"]["variant"] = {"rfc6962": "RFC 6962 section 2.1 mode: leaf = SHA-256(0x00 || chunk), node = "
-                                               "SHA-256(0x01 || left || right); verification in that mode",
-                                    "sha384": "SHA-384 leaves and tree (hash + root, no manifest compare)"}[args.variant]
-        if args.variant == "sha384":
-            sha384_peak = SM_COUNT * INT_LANES_PER_SM * 1.965e9 / (3568.0 / 128.0) / 1e9
-            out["metric"] = "GB/s hashed (SHA-384 chunks + Merkle root) at 1 B200"
-            out["roofline"].update({"peak": round(sha384_peak, 1), "frac": round(achieved / sha384_peak, 4),
-                                    "int32_ops_per_byte": 3568.0 / 128.0, "chain_count_bound_gbs": None,
+        wide = args.variant in ("sha384", "sha512")
+        out["config"]["variant"] = ("RFC 6962 section 2.1 mode: leaf = SHA-256(0x00 || chunk), node = SHA-256(0x01 || left || "
+                                    "right); verification in that mode" if not wide else
+                                    f"{args.variant.upper()} leaves and tree (hash + root, no manifest compare)")
+        if wide:
+            peak = SM_COUNT * INT_LANES_PER_SM * SM_HZ / INT_OPS_PER_BYTE_SHA512 / 1e9
+            out["metric"] = f"GB/s hashed ({args.variant.upper()} chunks + Merkle root) at 1 B200"
+            out["roofline"].update({"peak": round(peak, 1), "frac": round(roofline["achieved"] / peak, 4),
+                                    "int32_ops_per_byte": INT_OPS_PER_BYTE_SHA512, "chain_count_bound_gbs": None,
+                                    "chain_count_bound_at_issue_floor_gbs": None,
                                     "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1.965 GHz / 27.875 INT32 ops per byte"})
     if not ragged and args.two_level:
         out["config"]["leaf_definition"] = (f"TWO-LEVEL (not the default): chunk digest = Merkle root over SHA-256 of "
@@ -394,15 +493,20 @@ def run_ours(args):
         out["roofline"]["chains"] = binding.n_chunks(nbytes, args.two_level)
         out["roofline"]["note"] = "launch_ms covers piece hashing + the levels up to chunk digests"
 
-    if rank == 0 and not ragged and not args.no_e2e and not args.two_level and copies == 1 and args.variant == "sha256":
-        out["e2e"] = measure_e2e(ctx, wl, device, args)
+    if rank == 0 and plain and not args.no_e2e:
+        out["e2e"] = measure_e2e(ctx, wl, device, args.steps)
     elif rank == 0:
         out["e2e"] = None
-    if rank == 0 and world == 1 and not args.no_cpu and not (not ragged and args.two_level) and copies == 1 \
-            and args.variant == "sha256":
+    if rank == 0 and world == 1 and not args.no_cpu and (plain or ragged):
         out["cpu_baseline"] = measure_cpu_baseline(ctx, wl, device, oracle, ragged,
                                                    None if ragged else man_digests,
                                                    (d_off, d_len, digests) if ragged else None)
+    want_secondary = args.secondary if args.secondary is not None else (
+        args.config is None and cfg_id == 4 and not args.nbytes and not args.chunk)
+    if rank == 0 and world == 1 and plain and want_secondary:
+        del data, wl, man_digests, m
+        torch.cuda.empty_cache()
+        out["secondary"] = measure_secondary(ctx, device, gpu_index, args)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
@@ -411,15 +515,7 @@ def run_ours(args):
     ctx.close()
 
 
-def _measured_peak(key):
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            return json.load(f).get(key)
-    except Exception:
-        return None
-
-
-def measure_e2e(ctx, wl, device, args):
+def measure_e2e(ctx, wl, device, steps):
     """Same metric through iv_verify_streamed: the blob starts in pinned HOST memory, every step copies it
     to the device in 4 GiB windows (overlapped with hashing) and reads the verification result back."""
     from paper_2510_23938_b200 import binding
@@ -457,7 +553,7 @@ def measure_e2e(ctx, wl, device, args):
     result = binding.new_result(device)
     idx = torch.zeros(64, dtype=torch.int64, device=device)
     stream = torch.cuda.current_stream()
-    steps = max(1, min(args.steps, 3))
+    steps = max(1, min(steps, 3))
     ok = True
     for _ in range(1):
         ctx.verify_streamed(windows, window, e_nbytes, manifest, result, idx)
@@ -468,7 +564,7 @@ def measure_e2e(ctx, wl, device, args):
     for _ in range(steps):
         ctx.verify_streamed(windows, window, e_nbytes, manifest, result, idx)
         host_result = binding.read_result(result)          # device -> host read of the step's result
-        ok &= host_result["root_ok"] and host_result["n_mismatch"] == 0
+        ok &= host_result["root_ok"] and host_result["n_mismatch"] == 0 and host_result["status"] == 0
     e1.record(stream)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
@@ -482,7 +578,7 @@ def measure_e2e(ctx, wl, device, args):
     torch.cuda.synchronize()
     link_gbs = ring[0].numel() / (e0.elapsed_time(e1) * 1e-3) / 1e9
     del dst
-    return {"value": round(e_nbytes / (ms * 1e-3) / 1e9, 3), "unit": "GB/s", "ms_per_step": round(ms, 3),
+    return {"value": round(e_nbytes / (ms * 1e-3) / 1e9, 3) if ok else None, "unit": "GB/s", "ms_per_step": round(ms, 3),
             "h2d_copy_alone_gbs": round(link_gbs, 2),
             "steps": steps, "h2d_bytes_per_step": int(e_nbytes), "d2h_bytes_per_step": 48,
             "api": "iv_verify_streamed, pinned host windows of %d MiB, two device windows" % (window // MIB),
@@ -527,6 +623,92 @@ def measure_cpu_baseline(ctx, wl, device, oracle, ragged, man_digests, ragged_st
         sample = f"first {ns} chunks ({nb / 1e9:.2f} GB) of the same blob, verified against the GPU's digests and root"
     return {"value": round(nb / dt / 1e9, 3), "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample,
             "seconds": round(dt, 2), "gpu_matches_oracle_on_sample": parity}
+
+
+def measure_secondary(ctx, device, gpu_index, args):
+    """The other named configurations, for the record beside the headline: the 16 GB weight file (device
+    resident, streamed from pinned host memory, and its per-tensor digests) and the 64 MiB blob (alone, and
+    with its three tampered copies verified as one batch).  Each timed region lasts at least a second so that
+    the clock sampler sees it."""
+    from paper_2510_23938_b200 import binding, inputs
+    out = {}
+    stream = torch.cuda.current_stream()
+
+    def steps_for(ms_per_step, floor):
+        return max(floor, int(math.ceil(1000.0 / max(ms_per_step, 1e-3))))
+
+    # ---- 16 GB weight file
+    wl = build_workload(3, device, seed=1000)
+    data, nbytes, chunk = wl["data"], wl["nbytes"], wl["chunk"]
+    m = measure_verify(ctx, wl, device, steps_for(66.0, args.steps), 3, gpu_index)
+    rf = m["roofline"]
+    blocks_per_chain = (chunk + 8) // 64 + 1
+    c3 = {"workload": wl["name"], "bytes": nbytes, "chunk_bytes": chunk, "chains": m["n_units"],
+          "value": round(m["gbs"], 3) if m["verified_ok"] else None, "unit": "GB/s", "verified_ok": m["verified_ok"],
+          "ms_per_step": round(m["ms_per_step"], 4), "leaf_kernel": rf["kernel"], "leaf_kernel_ms": rf["launch_ms"],
+          "frac": rf["frac"], "peak": rf["peak"],
+          "cycles_per_block_measured": round(rf["launch_ms"] * 1e-3 * SM_HZ / blocks_per_chain, 1),
+          "chain_count_bound_gbs": rf["chain_count_bound_gbs"],
+          "chain_count_bound_at_issue_floor_gbs": rf["chain_count_bound_at_issue_floor_gbs"],
+          "target_70pct_of_roofline": "not met and not reachable with leaf = SHA-256(4 MiB chunk): 3,830 serial chains bound "
+                                      "the launch at 44 % of the roofline even at the issue floor of 1,280 cycles per block",
+          "clocks": m["clocks"]}
+    e2e = measure_e2e(ctx, wl, device, 3)
+    c3["streamed"] = {k: e2e.get(k) for k in ("value", "unit", "ms_per_step", "h2d_copy_alone_gbs", "verified_ok", "api")}
+    # per-tensor digests of the same file: one iv_hash_ragged call over its 291 tensors
+    table = wl["table"]
+    offs = torch.tensor([o for _, o, _ in table], dtype=torch.int64, device=device)
+    lens = torch.tensor([ln for _, _, ln in table], dtype=torch.int64, device=device)
+    tens = torch.empty((len(table), 32), dtype=torch.uint8, device=device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(gpu_index) as clocks:
+        e0.record(stream)
+        ctx.hash_ragged(data, offs, lens, out=tens)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    longest = int(lens.max().item())
+    seconds = e0.elapsed_time(e1) * 1e-3
+    c3["per_tensor"] = {"seconds": round(seconds, 3), "n_tensors": len(table), "bytes": int(lens.sum().item()),
+                        "longest_bytes": longest, "leaf_kernel": ctx.last_leaf_kernel,
+                        "bound_seconds": round(longest / 64 * SPLIT_CYCLES_PER_BLOCK / SM_HZ, 3),
+                        "bound": "longest_bytes / 64 x cycles per block of one chain / SM clock (one tensor is one serial chain)",
+                        "device_status": ctx.device_status(), "clocks": clocks.summary()}
+    out["config3"] = c3
+    del data, wl, m, tens
+    torch.cuda.empty_cache()
+
+    # ---- 64 MiB blob, alone and with its three tampered copies as one batch
+    wl = build_workload(1, device, seed=1000)
+    data, nbytes, chunk = wl["data"], wl["nbytes"], wl["chunk"]
+    flush = torch.empty(256 * MIB, dtype=torch.uint8, device=device)
+    m = measure_verify(ctx, wl, device, steps_for(1.1, args.steps), 3, gpu_index, flush)
+    c1 = {"workload": wl["name"], "bytes": nbytes, "chunk_bytes": chunk, "chains": m["n_units"],
+          "value": round(m["gbs"], 3) if m["verified_ok"] else None, "unit": "GB/s", "verified_ok": m["verified_ok"],
+          "ms_per_step": round(m["ms_per_step"], 4), "leaf_kernel": m["roofline"]["kernel"],
+          "leaf_kernel_ms": m["roofline"]["launch_ms"], "frac": m["roofline"]["frac"],
+          "chain_count_bound_gbs": m["roofline"]["chain_count_bound_gbs"], "l2": "flushed between steps (256 MiB write)",
+          "clocks": m["clocks"]}
+    blobs, want_idx = [data], [[]]
+    for k in (2, 3, 4):
+        off, bit = inputs.flip_position(k, nbytes)
+        bad = data.clone()
+        bad[off] ^= (1 << bit)
+        blobs.append(bad)
+        want_idx.append([off // chunk])
+    results = torch.zeros((4, 48), dtype=torch.uint8, device=device)
+    bidx = torch.full((4, 8), -1, dtype=torch.int64, device=device)
+    total_ms, clocks = time_steps(lambda: ctx.verify_manifest_batch(blobs, m["manifest"], results, bidx),
+                                  steps_for(1.3, args.steps), 3, flush, gpu_index)
+    n_steps = steps_for(1.3, args.steps)
+    rs = binding.read_results(results)
+    got_idx = [[int(v) for v in bidx[b, :rs[b]["n_mismatch"]].cpu()] for b in range(4)]
+    ok = bool(ctx.device_status() == 0 and got_idx == want_idx and rs[0]["root_ok"] and not any(r["root_ok"] for r in rs[1:]))
+    c1["batch_of_4"] = {"value": round(4 * nbytes / (total_ms / n_steps * 1e-3) / 1e9, 3) if ok else None, "unit": "GB/s",
+                        "ms_per_step": round(total_ms / n_steps, 4), "chains": 4 * m["n_units"], "verified_ok": ok,
+                        "mismatch_idx": got_idx, "api": "iv_verify_manifest_batch: the blob and its three tampered copies, "
+                                                        "one hashing launch", "clocks": clocks}
+    out["config1"] = c1
+    return out
 
 
 # --------------------------------------------------------------------------------------------
@@ -575,6 +757,22 @@ def run_reference(args):
     }), flush=True)
 
 
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(args) -> int:
+    """`--gpus N` without a launcher: start N ranks of this script with torch.distributed.run, one per GPU."""
+    if not args.same_device and torch.cuda.device_count() < args.gpus:
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} needs {args.gpus} GPUs, {torch.cuda.device_count()} visible\n")
+        return 2
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.run(cmd).returncode
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -587,9 +785,9 @@ def main():
     ap.add_argument("--two-level", type=int, default=None, metavar="SUB_BYTES",
                     help="two-level leaves: chunk digest = Merkle root over SHA-256 of SUB_BYTES pieces (a different, "
                          "separately named leaf definition; not the default)")
-    ap.add_argument("--variant", default="sha256", choices=["sha256", "rfc6962", "sha384"],
+    ap.add_argument("--variant", default="sha256", choices=["sha256", "rfc6962", "sha384", "sha512"],
                     help="sha256 = the default path; rfc6962 = 0x00/0x01-prefixed tree (verification in that mode); "
-                         "sha384 = SHA-384 leaves and tree (hash + root). Not the graded line.")
+                         "sha384 / sha512 = those leaves and tree (hash + root). Not the graded line.")
     ap.add_argument("--dist-backend", default="nccl", help="torch.distributed backend for --gpus > 1")
     ap.add_argument("--same-device", action="store_true",
                     help="put every rank on cuda:0 (only to check the multi-rank logic on a one-GPU box, with gloo)")
@@ -598,10 +796,15 @@ def main():
                          "pass with iv_verify_manifest_batch; value counts all copies' bytes")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--secondary", dest="secondary", action="store_true", default=None,
+                    help="also measure the 16 GB and the 64 MiB configurations (default: on for the default workload)")
+    ap.add_argument("--no-secondary", dest="secondary", action="store_false")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     else:
         run_ours(args)
 

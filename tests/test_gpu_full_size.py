@@ -1,11 +1,11 @@
 """Parity at the full sizes of the named configurations, in the launch configuration bench.py times.
 
 The blobs are built by bench.py's own workload builder and hashed through the same entry points the
-benchmark calls.  Configurations 2 and 3 are checked completely (the oracle hashes the whole blob on the
-host cores); configurations 4 and 5 are too large for that, so the oracle recomputes sampled outputs one
-by one (first, last, window borders, random picks; the longest tensors), and the rest is covered by
-properties that hold at any size: a flipped bit is found at its chunk, the streamed digests equal the
-resident ones, and the tree kernel is checked against the oracle on seeded leaves of the same count."""
+benchmark calls.  Every configuration is checked completely: the blob goes to the host window by window through a
+pinned staging buffer, the oracle hashes every chunk (every tensor) on the host cores, and every digest,
+the root, and the count and indices of seeded bit flips are compared bit for bit.  Manifests are built
+from the ORACLE's digests and root, never from the library's own output.  The RFC 6962 and SHA-384
+variants at the largest size stay sampled."""
 import numpy as np
 import pytest
 import torch
@@ -46,6 +46,37 @@ def _oracle_digests_of_device_blob(data: torch.Tensor, chunk: int, piece: int = 
     return np.concatenate(out)
 
 
+class _Stager:
+    """Device bytes -> a numpy view of a reused pinned host buffer (valid until the next call)."""
+
+    def __init__(self, capacity: int):
+        self.buf = torch.empty(capacity, dtype=torch.uint8, pin_memory=True)
+
+    def __call__(self, t: torch.Tensor) -> np.ndarray:
+        n = t.numel()
+        self.buf[:n].copy_(t)
+        torch.cuda.synchronize()
+        return self.buf[:n].numpy()
+
+
+def _oracle_tensor_digests(data: torch.Tensor, offs: np.ndarray, lens: np.ndarray, stage: _Stager) -> np.ndarray:
+    """Oracle digests of tensors laid out in ascending offset order, over consecutive runs of tensors that fit
+    the staging buffer."""
+    cap, n = stage.buf.numel(), len(lens)
+    want = np.zeros((n, 32), dtype=np.uint8)
+    threads = oracle.host_threads()
+    k = 0
+    while k < n:
+        j = k + 1
+        while j < n and int(offs[j] + lens[j] - offs[k]) <= cap:
+            j += 1
+        lo, hi = int(offs[k]), int(offs[j - 1] + lens[j - 1])
+        assert hi - lo <= cap
+        want[k:j] = oracle.hash_ragged(stage(data[lo:hi]), offs[k:j] - lo, lens[k:j], nthreads=threads)
+        k = j
+    return want
+
+
 @pytest.mark.parametrize("cfg_id", [2, 3])
 def test_weight_file_configurations_completely(ctx, cfg_id):
     _need((4 if cfg_id == 2 else 20) * GIB)
@@ -71,84 +102,106 @@ def test_weight_file_configurations_completely(ctx, cfg_id):
     r = binding.read_result(res)
     assert (not r["root_ok"]) and r["n_mismatch"] == 1 and int(idx[0]) == n - 1
     data[data.numel() - 2] ^= 0x10
-    # per-tensor digests of the same file (sampled: the oracle hashes every tensor below 40 MB and the two largest)
+    # per-tensor digests of the same file: every tensor against the oracle
     table = wl["table"]
     offs = np.array([o for _, o, _ in table], dtype=np.int64)
     lens = np.array([ln for _, _, ln in table], dtype=np.int64)
     tens = ctx.hash_ragged(data, torch.from_numpy(offs).cuda(), torch.from_numpy(lens).cuda())
-    pick = [k for k in range(len(table)) if lens[k] < 40e6] + list(np.argsort(lens)[-2:])
-    for k in pick:
-        piece = _host(data[offs[k]:offs[k] + lens[k]])
-        assert _host(tens[k]).tobytes() == oracle.sha256(piece), table[k][0]
+    assert ctx.device_status() == 0
+    want_t = _oracle_tensor_digests(data, offs, lens, _Stager(2 * GIB))
+    bad = np.nonzero((_host(tens) != want_t).any(axis=1))[0]
+    assert bad.size == 0, [table[k][0] for k in bad[:8]]
     del data, wl
     torch.cuda.empty_cache()
 
 
-def test_largest_configuration_sampled(ctx):
-    """112 GiB, 4 MiB chunks: the launch the benchmark times (sliced kernel, tiled copies)."""
+def test_largest_configuration_completely(ctx):
+    """112 GiB, 4 MiB chunks: the launch the benchmark times (sliced kernel, tiled copies, first workers
+    first), every one of its 28,672 digests against the oracle."""
     _need(125 * GIB)
     wl = bench.build_workload(4, torch.device("cuda", 0), seed=1000)
     data, chunk = wl["data"], wl["chunk"]
-    n = binding.n_chunks(data.numel(), chunk)
+    nbytes = data.numel()
+    n = binding.n_chunks(nbytes, chunk)
     assert n == 28_672
     got = ctx.hash_chunks(data, chunk)
     assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel" and ctx.device_status() == 0
+    host_got = _host(got)
+
+    # the oracle over the whole blob, one 4 GiB window at a time
+    window = 4 * GIB
+    stage = _Stager(window)
+    threads = oracle.host_threads()
+    want = np.concatenate([oracle.hash_chunks(stage(data[off:off + window]), chunk, nthreads=threads)
+                           for off in range(0, nbytes, window)])
+    assert want.shape == (n, 32)
+    bad = np.nonzero((host_got != want).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} digests differ from the oracle, first at chunk {bad[:8]}"
+    want_root = oracle.merkle_root(want)
+    assert _host(ctx.merkle_root(got)).tobytes() == want_root
+    assert _host(ctx.merkle_root(ctx.merkle_levels(got, 9))).tobytes() == want_root
+    assert _host(ctx.tree_build(got)[-1]).tobytes() == want_root
+
+    # verification against the ORACLE's manifest: clean, then three seeded flipped bits
+    manifest = ctx.make_manifest(nbytes, chunk, torch.from_numpy(want).cuda(), want_root)
+    res = binding.new_result("cuda")
+    idx = torch.full((8,), -1, dtype=torch.int64, device="cuda")
+    ctx.verify_manifest(data, manifest, res, idx)
+    assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel"
+    r = binding.read_result(res)
+    assert r["status"] == 0 and r["root_ok"] and r["n_mismatch"] == 0 and r["root"] == want_root
+    flips = [inputs.flip_position(seed, nbytes) for seed in (2, 3, 4)]
+    for off, bit in flips:
+        data[off] ^= (1 << bit)
+    touched = sorted({off // chunk for off, _ in flips})
+    tampered = want.copy()
+    for c in touched:
+        d = oracle.sha256(stage(data[c * chunk:(c + 1) * chunk]))
+        assert d != want[c].tobytes()
+        tampered[c] = np.frombuffer(d, dtype=np.uint8)
+    ctx.verify_manifest(data, manifest, res, idx)
+    r = binding.read_result(res)
+    assert r["status"] == 0 and (not r["root_ok"]) and r["n_mismatch"] == len(touched)
+    assert [int(v) for v in idx[:len(touched)].cpu()] == touched
+    assert r["root"] == oracle.merkle_root(tampered)
+    assert np.array_equal(_host(ctx.last_digests(n)), tampered)
+    for off, bit in flips:
+        data[off] ^= (1 << bit)
+
+    # the same launch shape in the RFC 6962 mode and with SHA-384 digests (sampled)
     rng = np.random.default_rng(4)
     sample = sorted(set([0, 1, 31, 32, 1023, 1024, 1025, 14_335, 14_336, n - 33, n - 32, n - 2, n - 1]
                         + [int(v) for v in rng.integers(0, n, size=40)]))
-    host_got = _host(got)
-    for i in sample:
-        want = oracle.sha256(_host(data[i * chunk:(i + 1) * chunk]))
-        assert host_got[i].tobytes() == want, i
-    # the tree over these digests by two independent routes of the library, and against the oracle on the
-    # sampled structure: the oracle root over the GPU digests is NOT used; the tree kernel's parity at this
-    # leaf count is pinned on seeded leaves in test_gpu_parity
-    root = _host(ctx.merkle_root(got)).tobytes()
-    assert _host(ctx.merkle_root(ctx.merkle_levels(got, 9))).tobytes() == root
-    assert _host(ctx.tree_build(got)[-1]).tobytes() == root
-    # the same launch shape in the RFC 6962 mode (prefixed leaf hashes through the migrating kernel)
     got6962 = _host(ctx.hash_chunks_rfc6962(data, chunk))
     assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel" and ctx.device_status() == 0
     for i in sample[::3]:
-        want = oracle.hash_chunks_rfc6962(_host(data[i * chunk:(i + 1) * chunk]), chunk)[0]
-        assert got6962[i].tobytes() == want.tobytes(), i
+        w = oracle.hash_chunks_rfc6962(stage(data[i * chunk:(i + 1) * chunk]), chunk)[0]
+        assert got6962[i].tobytes() == w.tobytes(), i
     del got6962
-    # and with SHA-384 digests
     got384 = _host(ctx.hash_chunks_sha384(data, chunk))
     assert ctx.device_status() == 0
     for i in sample[1::3]:
-        assert got384[i].tobytes() == oracle.sha384(_host(data[i * chunk:(i + 1) * chunk])), i
+        assert got384[i].tobytes() == oracle.sha384(stage(data[i * chunk:(i + 1) * chunk])), i
     del got384
-    # a flipped bit is found at its chunk, nothing else changes
-    manifest = ctx.make_manifest(data.numel(), chunk, got.clone(), root)
-    off, bit = inputs.flip_position(7, data.numel())
-    data[off] ^= (1 << bit)
-    res = binding.new_result("cuda")
-    idx = torch.zeros(4, dtype=torch.int64, device="cuda")
-    ctx.verify_manifest(data, manifest, res, idx)
-    r = binding.read_result(res)
-    assert (not r["root_ok"]) and r["n_mismatch"] == 1 and int(idx[0]) == off // chunk
-    flipped = oracle.sha256(_host(data[(off // chunk) * chunk:(off // chunk + 1) * chunk]))
-    assert _host(ctx.last_digests(n))[off // chunk].tobytes() == flipped
-    data[off] ^= (1 << bit)
-    # streamed from pinned host windows (a ring of two 4 GiB windows read as windows 0 and 1 of the blob):
-    # the digests of those windows equal the resident ones
-    window = 4 * GIB
+
+    # streamed from pinned host windows (a ring of two 4 GiB windows read as windows 0 and 1 of the blob),
+    # against the oracle's digests of those windows
     ring = [torch.empty(window, dtype=torch.uint8, pin_memory=True) for _ in range(2)]
     for w in range(2):
         ring[w].copy_(data[w * window:(w + 1) * window])
     per = window // chunk
-    sub_manifest = ctx.make_manifest(2 * window, chunk, got[:2 * per].clone(),
-                                     _host(ctx.merkle_root(got[:2 * per].contiguous())).tobytes())
+    sub_manifest = ctx.make_manifest(2 * window, chunk, torch.from_numpy(want[:2 * per].copy()).cuda(),
+                                     oracle.merkle_root(want[:2 * per]))
     ctx.verify_streamed(ring, window, 2 * window, sub_manifest, res, idx)
     r = binding.read_result(res)
-    assert r["root_ok"] and r["n_mismatch"] == 0
-    del data, wl, ring
+    assert r["status"] == 0 and r["root_ok"] and r["n_mismatch"] == 0
+    del data, wl, ring, stage
     torch.cuda.empty_cache()
 
 
-def test_ragged_configuration_sampled(ctx):
-    """10,000 tensors, log-uniform 4 KiB .. 64 MiB, packed at 2-byte alignment (about 69 GB)."""
+def test_ragged_configuration_completely(ctx):
+    """10,000 tensors, log-uniform 4 KiB .. 64 MiB, packed at 2-byte alignment (about 69 GB): every tensor
+    digest and the root over them against the oracle."""
     _need(75 * GIB)
     wl = bench.build_workload(5, torch.device("cuda", 0), seed=1000)
     data, offs, lens = wl["data"], wl["offsets"], wl["lengths"]
@@ -156,15 +209,11 @@ def test_ragged_configuration_sampled(ctx):
     got = ctx.hash_ragged(data, torch.from_numpy(offs).cuda(), torch.from_numpy(lens).cuda())
     assert ctx.last_leaf_kernel.startswith("hash_chunks_split_kernel") and ctx.device_status() == 0
     host_got = _host(got)
-    order = np.argsort(lens)
-    rng = np.random.default_rng(5)
-    sample = set(int(k) for k in order[:20]) | set(int(k) for k in order[-6:]) | {0, 1, 9_998, 9_999}
-    sample |= set(int(k) for k in rng.integers(0, 10_000, size=150) if lens[k] < 8e6)
-    for k in sorted(sample):
-        want = oracle.sha256(_host(data[offs[k]:offs[k] + lens[k]]))
-        assert host_got[k].tobytes() == want, (k, int(lens[k]))
-    # the root over the tensor digests in index order, against the oracle on the same count of seeded leaves
-    leaves = inputs.uniform_bytes(32 * 10_000, seed=55, device="cuda")
-    assert _host(ctx.merkle_root(leaves)).tobytes() == oracle.merkle_root(_host(leaves))
-    del data, wl
+    stage = _Stager(4 * GIB)
+    want = _oracle_tensor_digests(data, offs, lens, stage)
+    bad = np.nonzero((host_got != want).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} tensor digests differ from the oracle, first at {bad[:8]}"
+    # the root over the tensor digests in index order
+    assert _host(ctx.merkle_root(got)).tobytes() == oracle.merkle_root(want)
+    del data, wl, stage
     torch.cuda.empty_cache()
