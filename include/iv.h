@@ -77,6 +77,21 @@ uint64_t iv_kernel_launches(const iv_ctx *ctx);
  * Static text, never freed. */
 const char *iv_last_leaf_kernel(const iv_ctx *ctx);
 
+/* Where that kernel has several launch shapes (the many-chain kernel: workers per SM and the order in
+ * which they are served), the one the last call ran in; "" otherwise.  Static text. */
+const char *iv_last_leaf_instance(const iv_ctx *ctx);
+
+/* Self-test of the bounded waits (a diagnostic; the paper has no counterpart).  Every wait inside the
+ * library's kernels -- for a bulk copy, for a hand-over between warps -- gives up after a fixed number of
+ * SM clocks (about two seconds), sets the device status to 1 and lets the kernel return, so that a lost
+ * copy can never hang the GPU.  This call runs that path on purpose: one warp waits, with the same wait
+ * routine and a limit of limit_cycles SM clocks (1 .. 4e9), on a barrier that nobody arrives at, gives
+ * up, sets the status word and returns.  Afterwards iv_device_status reports 1 (and clears it), and the
+ * context works as before.
+ *   h_waited_cycles   optional host pointer; when given, the call waits for the stream and stores the
+ *                     SM clocks the warp spent waiting (>= limit_cycles) */
+int iv_selftest_wait_timeout(iv_ctx *ctx, uint64_t limit_cycles, uint64_t *h_waited_cycles, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------
  * Leaf hashing -- Algorithm 1, "chunk_count <- ceil(|M| / C)" and
  * "H_i = GPU_HASH(M_i)" with GPU_HASH = SHA-256 (FIPS 180-4 section 6.2).
@@ -114,8 +129,8 @@ int iv_merkle_root(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint
  * d_nodes[n] -> d_out[n_out], n_out = n halved (rounding up) `levels` times.  Node j
  * of the result is the root of the aligned run of 2^levels inputs starting at
  * j * 2^levels, which is also a node of the whole tree -- the building block for
- * the paper's multi-GPU scheme ("global Merkle trees from distributed hash
- * computations", section "Multi-GPU Deployment Architectures"): every GPU
+ * the paper's multi-GPU scheme (section "Multi-GPU Deployment Architectures",
+ * a global tree built from the hashes computed on each device): every GPU
  * reduces its aligned range of leaves to such nodes, the nodes are gathered, and
  * iv_merkle_root over them gives the global root.
  *   d_out, out_cap   receives n_out records; out_cap (in records) must be >= n_out;
@@ -127,7 +142,7 @@ int iv_merkle_levels(iv_ctx *ctx, const uint8_t *d_nodes, uint64_t n, uint32_t l
 
 /* ---------------------------------------------------------------------------
  * Incremental re-verification -- the paper's hierarchical / differential
- * verification ("incremental verification for model updates": when fine-tuning
+ * verification (section "Version Management and Incremental Verification": when fine-tuning
  * or an update touches some chunks, only those leaves and their paths to the
  * root are recomputed).
  *
@@ -186,7 +201,7 @@ int iv_verify_manifest(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
                        const iv_manifest *h_manifest, iv_verify_result *d_result,
                        uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream);
 
-/* Batch verification -- the paper's "multiple models can be verified simultaneously": n_blobs blobs of
+/* Batch verification -- the paper's batch processing (section "Scalability Analysis"): n_blobs blobs of
  * the same size (copies, replicas, variants that share a manifest) are verified against ONE manifest in
  * one pass; all their chunks are independent chains of a single hashing launch, which is what fills the
  * GPU when one blob alone has few chunks.
@@ -204,8 +219,8 @@ const uint8_t *iv_ctx_digests(const iv_ctx *ctx);
 
 /* ---------------------------------------------------------------------------
  * Two-level leaves -- a SEPARATELY NAMED mode whose digests differ from
- * iv_hash_chunks (the paper speaks of verification "at multiple levels of
- * granularity").  The digest of chunk i is the Merkle root (this library's tree
+ * iv_hash_chunks (the paper's hierarchical verification at several
+ * granularities).  The digest of chunk i is the Merkle root (this library's tree
  * rule) over the SHA-256 digests of its sub_bytes-sized pieces:
  *     D_i = root( SHA-256(piece_0), SHA-256(piece_1), ... )   pieces of chunk i.
  * A chunk is then no longer one serial SHA-256 chain but chunk_bytes/sub_bytes
@@ -269,8 +284,8 @@ int iv_set_timing(iv_ctx *ctx, int enabled);
 int iv_phase_times(iv_ctx *ctx, uint32_t calls_back, float *h_ms);
 
 /* ---------------------------------------------------------------------------
- * Per-tensor digests -- the paper's batch verification ("verification of
- * dozens of models concurrently", one digest per payload): digest k =
+ * Per-tensor digests -- the paper's batch verification (section "Scalability
+ * Analysis": many payloads per launch, one digest per payload): digest k =
  * SHA-256(d_base[offset_k .. offset_k + length_k)).
  *
  *   d_offsets, d_lengths   n uint64 each, DEVICE memory; any byte alignment of
@@ -283,8 +298,8 @@ int iv_hash_ragged(iv_ctx *ctx, const void *d_base, const uint64_t *d_offsets,
                    void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
- * Resumable per-tensor digests -- the paper's multi-pass processing ("hash state
- * is maintained across passes to ensure cryptographic continuity"): a tensor
+ * Resumable per-tensor digests -- the paper's multi-pass processing (section
+ * "Memory Scalability Considerations", the hash state carried from pass to pass): a tensor
  * that is larger than a resident window, or that spans two windows, is hashed
  * part by part.
  *
@@ -392,14 +407,14 @@ int iv_merkle_root_noalloc(const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *
  * Roofline probe (a measurement aid; the paper has no counterpart).  Runs a
  * register-only microbenchmark on every SM and reports, from the SM cycle
  * counter, how many lane-operations of one instruction kind an SM retires per
- * clock -- the denominator of the integer roofline -- or, for IV_PROBE_SHA256,
- * how many message bytes per clock per SM the compression function alone
- * sustains.  Synchronous; allocates and frees a few KB of device memory.
+ * clock -- the denominator of the integer roofline -- or, for the kinds that run
+ * SHA-256 (6, 7, 13, 14), how many message bytes per clock per SM that part of the
+ * compression function alone sustains.  Synchronous; allocates and frees a few KB of device memory.
  *
  *   warps_per_block, blocks_per_sm   launch shape (blocks = blocks_per_sm * SM count)
  *   active_lanes                     1..32 lanes of each warp that do work
- *   iters                            loop trips (128 operations each; one compression
- *                                    each for IV_PROBE_SHA256)
+ *   iters                            loop trips (128 operations each; one 64-byte block
+ *                                    each for the SHA-256 kinds)
  *   h_out[0]                         lane-ops (or bytes) per clock per SM
  *   h_out[1]                         mean cycles per block
  */
@@ -411,26 +426,14 @@ typedef enum iv_probe_kind {
     IV_PROBE_IMAD = 4,   /* integer multiply-add */
     IV_PROBE_MIXED = 5,  /* LOP3 and IMAD interleaved 1:1 */
     IV_PROBE_SHA256 = 6,     /* full SHA-256 compressions, registers only */
-    IV_PROBE_SHA256_FMA = 7, /* the same with every addition issued as a multiply-add (FMA pipe) */
+    IV_PROBE_SHA256_SCHED_FMA = 7, /* the same with the message schedule's additions as multiply-adds (FMA pipe) */
     IV_PROBE_LAT_IADD3 = 8,  /* kinds 8..11: ONE dependent chain per thread; with one warp per SM,   */
     IV_PROBE_LAT_LOP3 = 9,   /* 32 / h_out[0] is the dependent-issue latency of the instruction in   */
     IV_PROBE_LAT_SHF = 10,   /* clocks                                                               */
     IV_PROBE_LAT_IMAD = 11,
     IV_PROBE_LAT_CROSS = 12, /* one chain alternating LOP3 (ALU pipe) and IMAD (FMA pipe) */
-    IV_PROBE_ROUNDS_M0 = 13, /* kinds 13..16: the 64 rounds alone (W + K from shared memory), one   */
-    IV_PROBE_ROUNDS_M1 = 14, /* block per trip, for the four placements of the additions; reported  */
-    IV_PROBE_ROUNDS_M2 = 15, /* as message bytes per clock per SM                                    */
-    IV_PROBE_ROUNDS_M3 = 16,
-    IV_PROBE_SCHEDULE = 17,  /* the message schedule + round constants alone, one block per trip */
-    IV_PROBE_ROUNDS_M4 = 18,
-    IV_PROBE_ROUNDS_M5 = 19,
-    IV_PROBE_SHA256_ADD2 = 20, /* kinds 20..22: full compressions with the additions placed as the */
-    IV_PROBE_SHA256_ADD3 = 21, /* library's addition placements 2, 3 and 4                          */
-    IV_PROBE_SHA256_ADD4 = 22,
-    IV_PROBE_ROUNDS_M3_HANDSHAKE = 23, /* kind 16 plus the consumer's per-block hand-over (barrier wait, arrival, feed-forward) */
-    IV_PROBE_SHA256_STREAM = 24, /* full compressions of a message that does not depend on the chaining value */
-    IV_PROBE_SHA256_ADD6 = 25,   /* full compressions, the schedule's plain shifts as multiply-high (FMA pipe) */
-    IV_PROBE_SHA256_ADD7 = 26    /* full compressions, the schedule's shifts and rotations as multiply-adds (FMA pipe) */
+    IV_PROBE_ROUNDS = 13,    /* the 64 rounds alone, W + K from shared memory: the consumer half of the two-warp kernel */
+    IV_PROBE_SCHEDULE = 14   /* the message schedule + round constants alone: its producer half */
 } iv_probe_kind;
 int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t blocks_per_sm,
                  uint32_t active_lanes, uint32_t iters, double *h_out);

@@ -28,7 +28,7 @@ EXPORTS = (
     "iv_create", "iv_destroy", "iv_strerror", "iv_last_cuda_error", "iv_kernel_launches",
     "iv_hash_chunks", "iv_merkle_root", "iv_verify_manifest", "iv_ctx_digests",
     "iv_verify_streamed", "iv_hash_ragged", "iv_set_timing", "iv_phase_times", "iv_probe_alu", "iv_device_status",
-    "iv_merkle_root_noalloc", "iv_last_leaf_kernel", "iv_merkle_levels",
+    "iv_merkle_root_noalloc", "iv_last_leaf_kernel", "iv_last_leaf_instance", "iv_selftest_wait_timeout", "iv_merkle_levels",
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
     "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update", "iv_verify_manifest_batch",
     "iv_hash_chunks_sha384", "iv_merkle_root_sha384", "iv_verify_manifest_sha384",
@@ -143,6 +143,10 @@ def load_library() -> ctypes.CDLL:
     lib.iv_merkle_root_noalloc.restype = i32
     lib.iv_last_leaf_kernel.argtypes = [vp]
     lib.iv_last_leaf_kernel.restype = ctypes.c_char_p
+    lib.iv_last_leaf_instance.argtypes = [vp]
+    lib.iv_last_leaf_instance.restype = ctypes.c_char_p
+    lib.iv_selftest_wait_timeout.argtypes = [vp, u64, ctypes.POINTER(u64), vp]
+    lib.iv_selftest_wait_timeout.restype = i32
     lib.iv_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.iv_device_status.restype = i32
     lib.iv_probe_alu.argtypes = [vp, i32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
@@ -234,11 +238,13 @@ class Context:
         self._check(rc, "iv_hash_chunks")
         return out[:got.value]
 
-    def hash_chunks_two_level(self, data: torch.Tensor, chunk_bytes: int, sub_bytes: int, stream=None) -> torch.Tensor:
+    def hash_chunks_two_level(self, data: torch.Tensor, chunk_bytes: int, sub_bytes: int, stream=None,
+                              out: torch.Tensor | None = None) -> torch.Tensor:
         """iv_hash_chunks_two_level: digest i = Merkle root over the SHA-256 digests of chunk i's sub_bytes pieces."""
         nb = _nbytes(data)
         n = n_chunks(nb, chunk_bytes) if chunk_bytes > 0 else 0
-        out = torch.empty((n, 32), dtype=torch.uint8, device=data.device)
+        if out is None:
+            out = torch.empty((n, 32), dtype=torch.uint8, device=data.device)
         got = ctypes.c_uint64(0)
         rc = self._lib.iv_hash_chunks_two_level(self._h, _dev_ptr(data), nb, chunk_bytes, sub_bytes, _dev_ptr(out), n,
                                                 ctypes.byref(got), _stream_ptr(stream))
@@ -263,21 +269,24 @@ class Context:
         self._check(rc, "iv_merkle_root")
         return out
 
-    def hash_chunks_sha384(self, data: torch.Tensor, chunk_bytes: int, stream=None) -> torch.Tensor:
+    def hash_chunks_sha384(self, data: torch.Tensor, chunk_bytes: int, stream=None,
+                           out: torch.Tensor | None = None) -> torch.Tensor:
         """iv_hash_chunks_sha384: (n, 48) uint8 SHA-384 digests of the chunks of `data`."""
         nb = _nbytes(data)
         n = n_chunks(nb, chunk_bytes) if chunk_bytes > 0 else 0
-        out = torch.empty((n, 48), dtype=torch.uint8, device=data.device)
+        if out is None:
+            out = torch.empty((n, 48), dtype=torch.uint8, device=data.device)
         got = ctypes.c_uint64(0)
         rc = self._lib.iv_hash_chunks_sha384(self._h, _dev_ptr(data), nb, chunk_bytes, _dev_ptr(out), n,
                                              ctypes.byref(got), _stream_ptr(stream))
         self._check(rc, "iv_hash_chunks_sha384")
         return out[:got.value]
 
-    def merkle_root_sha384(self, leaves: torch.Tensor, stream=None) -> torch.Tensor:
+    def merkle_root_sha384(self, leaves: torch.Tensor, stream=None, out: torch.Tensor | None = None) -> torch.Tensor:
         """iv_merkle_root_sha384: 48-byte root of (n, 48) leaf digests."""
         n = leaves.numel() // 48
-        out = torch.empty(48, dtype=torch.uint8, device=leaves.device)
+        if out is None:
+            out = torch.empty(48, dtype=torch.uint8, device=leaves.device)
         rc = self._lib.iv_merkle_root_sha384(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
         self._check(rc, "iv_merkle_root_sha384")
         return out
@@ -298,26 +307,29 @@ class Context:
         r = VerifyResult384.from_buffer_copy(bytes(result.cpu().numpy().tobytes()))
         return {"status": int(r.status), "root_ok": bool(r.root_ok), "n_mismatch": int(r.n_mismatch), "root": bytes(r.root)}
 
-    def hash_chunks_rfc6962(self, data: torch.Tensor, chunk_bytes: int, stream=None) -> torch.Tensor:
+    def hash_chunks_rfc6962(self, data: torch.Tensor, chunk_bytes: int, stream=None,
+                            out: torch.Tensor | None = None) -> torch.Tensor:
         """iv_hash_chunks_rfc6962: (n, 32) uint8 leaf hashes SHA-256(0x00 || chunk)."""
         nb = _nbytes(data)
         n = n_chunks(nb, chunk_bytes) if chunk_bytes > 0 else 0
-        out = torch.empty((n, 32), dtype=torch.uint8, device=data.device)
+        if out is None:
+            out = torch.empty((n, 32), dtype=torch.uint8, device=data.device)
         got = ctypes.c_uint64(0)
         rc = self._lib.iv_hash_chunks_rfc6962(self._h, _dev_ptr(data), nb, chunk_bytes, _dev_ptr(out), n,
                                               ctypes.byref(got), _stream_ptr(stream))
         self._check(rc, "iv_hash_chunks_rfc6962")
         return out[:got.value]
 
-    def merkle_root_rfc6962(self, leaves: torch.Tensor, stream=None) -> torch.Tensor:
+    def merkle_root_rfc6962(self, leaves: torch.Tensor, stream=None, out: torch.Tensor | None = None) -> torch.Tensor:
         """iv_merkle_root_rfc6962: 32-byte root with 0x01-prefixed nodes over (n, 32) leaf hashes."""
         n = leaves.numel() // 32
-        out = torch.empty(32, dtype=torch.uint8, device=leaves.device)
+        if out is None:
+            out = torch.empty(32, dtype=torch.uint8, device=leaves.device)
         rc = self._lib.iv_merkle_root_rfc6962(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
         self._check(rc, "iv_merkle_root_rfc6962")
         return out
 
-    def merkle_levels(self, nodes: torch.Tensor, levels: int, stream=None) -> torch.Tensor:
+    def merkle_levels(self, nodes: torch.Tensor, levels: int, stream=None, out: torch.Tensor | None = None) -> torch.Tensor:
         """iv_merkle_levels: the (ceil(n / 2^levels), 32) nodes `levels` levels above `nodes`."""
         n = nodes.numel() // 32
         n_out = n
@@ -325,7 +337,8 @@ class Context:
             if n_out <= 1:
                 break
             n_out = (n_out + 1) // 2
-        out = torch.empty((n_out, 32), dtype=torch.uint8, device=nodes.device)
+        if out is None:
+            out = torch.empty((n_out, 32), dtype=torch.uint8, device=nodes.device)
         got = ctypes.c_uint64(0)
         rc = self._lib.iv_merkle_levels(self._h, _dev_ptr(nodes), n, levels, _dev_ptr(out), n_out,
                                         ctypes.byref(got), _stream_ptr(stream))
@@ -333,11 +346,14 @@ class Context:
         assert got.value == n_out
         return out
 
-    def tree_build(self, leaves: torch.Tensor, stream=None) -> torch.Tensor:
+    def tree_records(self, n_leaves: int) -> int:
+        return int(self._lib.iv_tree_records(n_leaves))
+
+    def tree_build(self, leaves: torch.Tensor, stream=None, out: torch.Tensor | None = None) -> torch.Tensor:
         """iv_tree_build: the retained tree (iv_tree_records(n), 32) of the (n, 32) leaf digests; root = tree[-1]."""
         n = leaves.numel() // 32
         records = int(self._lib.iv_tree_records(n))
-        tree = torch.empty((records, 32), dtype=torch.uint8, device=leaves.device)
+        tree = torch.empty((records, 32), dtype=torch.uint8, device=leaves.device) if out is None else out
         rc = self._lib.iv_tree_build(self._h, _dev_ptr(leaves), n, _dev_ptr(tree), records, _stream_ptr(stream))
         self._check(rc, "iv_tree_build")
         return tree
@@ -433,17 +449,27 @@ class Context:
     def last_leaf_kernel(self) -> str:
         return self._lib.iv_last_leaf_kernel(self._h).decode()
 
+    @property
+    def last_leaf_instance(self) -> str:
+        return self._lib.iv_last_leaf_instance(self._h).decode()
+
+    def selftest_wait_timeout(self, limit_cycles: int, stream=None) -> int:
+        """iv_selftest_wait_timeout: a warp waits `limit_cycles` SM clocks on a barrier nobody arrives at, gives
+        up and sets the device status to 1; returns the clocks it waited (synchronises the stream)."""
+        waited = ctypes.c_uint64(0)
+        rc = self._lib.iv_selftest_wait_timeout(self._h, int(limit_cycles), ctypes.byref(waited), _stream_ptr(stream))
+        self._check(rc, "iv_selftest_wait_timeout")
+        return int(waited.value)
+
     def device_status(self) -> int:
         """iv_device_status: waits for the device, returns and clears the device-side status word."""
         st = ctypes.c_uint32(0)
         self._check(self._lib.iv_device_status(self._h, ctypes.byref(st)), "iv_device_status")
         return int(st.value)
 
-    PROBE_KINDS = {"iadd3": 0, "lop3": 1, "shf": 2, "prmt": 3, "imad": 4, "mixed": 5, "sha256": 6, "sha256_fma": 7,
+    PROBE_KINDS = {"iadd3": 0, "lop3": 1, "shf": 2, "prmt": 3, "imad": 4, "mixed": 5, "sha256": 6, "sha256_sched_fma": 7,
                    "lat_iadd3": 8, "lat_lop3": 9, "lat_shf": 10, "lat_imad": 11, "lat_cross": 12,
-                   "rounds_m0": 13, "rounds_m1": 14, "rounds_m2": 15, "rounds_m3": 16, "schedule": 17, "rounds_m4": 18, "rounds_m5": 19,
-                   "sha256_add2": 20, "sha256_add3": 21, "sha256_add4": 22, "rounds_m3_handshake": 23,
-                   "sha256_stream": 24, "sha256_add6": 25, "sha256_add7": 26}
+                   "rounds": 13, "schedule": 14}
 
     def probe_alu(self, kind: str, warps_per_block: int = 4, blocks_per_sm: int = 1, active_lanes: int = 32,
                   iters: int = 2000) -> tuple[float, float]:

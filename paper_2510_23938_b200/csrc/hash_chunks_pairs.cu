@@ -28,7 +28,7 @@ namespace {
 constexpr unsigned long long kTaskDone = ~0ull, kTaskFailed = ~0ull - 1;
 
 // PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash), as in the migrating kernel.
-template <int SEG, int STAGES, int NSLOT, int MODE, int PAIR, bool PREFIX>
+template <int SEG, int STAGES, int NSLOT, int PAIR, bool PREFIX>
 __global__ void __launch_bounds__(64)
 hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
                          uint8_t *__restrict__ digests, uint32_t *__restrict__ status, uint64_t slice_bytes,
@@ -237,7 +237,7 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
                     failed = !tma::mbar_wait_bounded(bar_full + 8 * wslot, fparity);     // uniform: one barrier word
                     if (failed) break;
                 }
-                rounds64<MODE>(v, wk_base + wslot * kWkSlot + in_slot * kWkBlock, one);
+                rounds64(v, wk_base + wslot * kWkSlot + in_slot * kWkBlock, one);
                 const bool slot_done = in_slot == PAIR - 1 || blk + 1 == warp_total;
                 if (slot_done) {
                     __syncwarp();                          // all 32 lanes have their values in registers
@@ -285,10 +285,10 @@ bool hash_chunks_wants_pairs(const uint8_t *d_data, uint64_t chunk_bytes, uint64
 cudaError_t launch_hash_chunks_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
                                      uint8_t *d_digests, uint32_t *d_status, void *d_scratch, const uint32_t *d_one,
                                      int sm_count, cudaStream_t stream, bool zero_prefix) {
-    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, MODE = 3, PAIR = 2;
+    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, PAIR = 2;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
-    auto kernel = zero_prefix ? hash_chunks_pairs_kernel<SEG, STAGES, NSLOT, MODE, PAIR, true>
-                              : hash_chunks_pairs_kernel<SEG, STAGES, NSLOT, MODE, PAIR, false>;
+    auto kernel = zero_prefix ? hash_chunks_pairs_kernel<SEG, STAGES, NSLOT, PAIR, true>
+                              : hash_chunks_pairs_kernel<SEG, STAGES, NSLOT, PAIR, false>;
     static bool configured[2][kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured[zero_prefix ? 1 : 0]); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, total_tasks = 0;

@@ -17,14 +17,13 @@
 // come, warps 4..7 take a task only when one lies in the FIFO unclaimed.  The schedulers left
 // with one group finish early and then take over what remains of the others.
 //
-// Data movement, TILED = false: the staged kernel's per-lane bulk copies (TMA, 1-D) into a
-// lane-interleaved shared-memory ring.  TILED = true: the blob is described to the TMA unit as a
-// 2-D tensor [chunk][byte] with the chunk size as row pitch, and ONE tiled copy of a 32-row x
-// 128-byte box brings the next two blocks of all 32 chains (instead of 32 copies issued one
-// lane after the other).  The box lands row-major, one 128-byte row per lane, with the 128-byte
-// swizzle (16-byte piece c of row r sits at piece c ^ (r mod 8)), so the lanes' 128-bit loads of
-// the same piece hit eight different bank groups.  Either way completion is counted by one
-// mbarrier per stage and the next block is in registers before the current block's rounds.
+// Data movement: the blob is described to the TMA unit as a 2-D tensor [chunk][byte] with the chunk
+// size as row pitch, and ONE tiled copy of a 32-row x 128-byte box brings the next two blocks of all
+// 32 chains (instead of 32 copies issued one lane after the other).  The box lands row-major, one
+// 128-byte row per lane, with the 128-byte swizzle (16-byte piece c of row r sits at piece
+// c ^ (r mod 8)), so the lanes' 128-bit loads of the same piece hit eight different bank groups.
+// Completion is counted by one mbarrier per stage and the next block is in registers before the
+// current block's rounds.
 #include <cuda.h>          // CUtensorMap (types only; the encoder is fetched through the runtime)
 
 #include <cstring>
@@ -71,7 +70,7 @@ __device__ __forceinline__ void tiled_g2s(uint32_t dst, const CUtensorMap *map, 
 // byte before data block j followed by its first 63 bytes; the word before the block is carried in a
 // register, at the start of a later slice it is read back from the blob.
 // ADD: where the additions of the compression go (see sha256_compress).
-template <int SEG, int STAGES, int MAX_WARPS, bool TILED, bool PREFIX, bool FWF, int ADD>
+template <int SEG, int STAGES, int MAX_WARPS, bool PREFIX, bool FWF, int ADD>
 __global__ void __launch_bounds__(32 * MAX_WARPS)
 hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
@@ -82,16 +81,16 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
     // schedule's additions to the FMA pipe (placement 2) lengthens the dependency chains and needs three warps
     // per scheduler to pay (launcher below).
     const uint32_t one = __ldg(one_ptr);
-    static_assert(!TILED || SEG == 256, "a tiled stage is two boxes of 32 rows x 128 bytes");
-    constexpr uint32_t kLaneStride = TILED ? 128 : SEG + 16;
-    constexpr uint32_t kStageBytes = TILED ? 8192 : 32 * kLaneStride;
+    static_assert(SEG == 256, "a stage is two boxes of 32 rows x 128 bytes");
+    constexpr uint32_t kLaneStride = 128;
+    constexpr uint32_t kStageBytes = 8192;
     constexpr int kBlocksPerSeg = SEG / 64;
     extern __shared__ __align__(128) uint8_t ring[];
     __shared__ __align__(8) uint64_t bars[MAX_WARPS][STAGES];
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
     // tiled boxes must start on a 1024-byte boundary (the swizzle pattern repeats every 8 rows)
-    const uint32_t ring0 = TILED ? ((tma::smem_u32(ring) + 1023u) & ~1023u) : tma::smem_u32(ring);
+    const uint32_t ring0 = (tma::smem_u32(ring) + 1023u) & ~1023u;
     const uint32_t ring_warp = ring0 + warp * (STAGES * kStageBytes);
     const uint32_t ring_base = ring_warp + lane * kLaneStride;
     const uint32_t swz = (lane & 7u) * 16u;
@@ -171,38 +170,24 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
         auto issue = [&](uint64_t seg, int stg) {
             const uint64_t off = seg * SEG;
             const uint32_t bar = bar_base + 8 * stg;
-            if (TILED) {
-                // one or two boxes of 32 chains x 128 bytes; a box always delivers its 4096 bytes
-                // (rows or bytes outside the tensor arrive as zeros and are never hashed)
-                if (lane == 0) {
-                    const uint32_t boxes = (warp_bytes - off > 128) ? 2u : 1u;
-                    tma::mbar_arrive_expect_tx(bar, boxes * 4096u);
-                    const uint32_t x = (uint32_t)(lo + off), y = (uint32_t)(g * 32);
-                    tiled_g2s(ring_warp + stg * kStageBytes, &tmap, x, y, bar);
-                    if (boxes == 2) tiled_g2s(ring_warp + stg * kStageBytes + 4096u, &tmap, x + 128u, y, bar);
-                }
-            } else {
-                const uint32_t bytes = off < my_bytes ? (uint32_t)((my_bytes - off < SEG) ? (my_bytes - off) : SEG) : 0u;
-                const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
-                if (lane == 0) tma::mbar_arrive_expect_tx(bar, total);
-                if (bytes) tma::bulk_g2s(ring_base + stg * kStageBytes, p + off, bytes, bar);
+            // one or two boxes of 32 chains x 128 bytes; a box always delivers its 4096 bytes
+            // (rows or bytes outside the tensor arrive as zeros and are never hashed)
+            if (lane == 0) {
+                const uint32_t boxes = (warp_bytes - off > 128) ? 2u : 1u;
+                tma::mbar_arrive_expect_tx(bar, boxes * 4096u);
+                const uint32_t x = (uint32_t)(lo + off), y = (uint32_t)(g * 32);
+                tiled_g2s(ring_warp + stg * kStageBytes, &tmap, x, y, bar);
+                if (boxes == 2) tiled_g2s(ring_warp + stg * kStageBytes + 4096u, &tmap, x + 128u, y, bar);
             }
         };
         auto fetch = [&](int stg, int blk_in_stage) {
-            if (TILED) {
-                // block b of the stage: box b / 2, 16-byte pieces 4 (b mod 2) .. +3 of this lane's row
-                const uint32_t row = ring_base + stg * kStageBytes + (uint32_t)(blk_in_stage >> 1) * 4096u;
-                const uint32_t c0 = (uint32_t)(blk_in_stage & 1) * 64u;
+            // block b of the stage: box b / 2, 16-byte pieces 4 (b mod 2) .. +3 of this lane's row
+            const uint32_t row = ring_base + stg * kStageBytes + (uint32_t)(blk_in_stage >> 1) * 4096u;
+            const uint32_t c0 = (uint32_t)(blk_in_stage & 1) * 64u;
 #pragma unroll
-                for (int qd = 0; qd < 4; ++qd)
-                    tma::ld_shared_v4(row + ((c0 + 16u * qd) ^ swz), raw[4 * qd], raw[4 * qd + 1], raw[4 * qd + 2],
-                                      raw[4 * qd + 3]);
-            } else {
-                const uint32_t src = ring_base + stg * kStageBytes + 64 * blk_in_stage;
-#pragma unroll
-                for (int qd = 0; qd < 4; ++qd)
-                    tma::ld_shared_v4(src + 16 * qd, raw[4 * qd], raw[4 * qd + 1], raw[4 * qd + 2], raw[4 * qd + 3]);
-            }
+            for (int qd = 0; qd < 4; ++qd)
+                tma::ld_shared_v4(row + ((c0 + 16u * qd) ^ swz), raw[4 * qd], raw[4 * qd + 1], raw[4 * qd + 2],
+                                  raw[4 * qd + 3]);
         };
 
         // prologue: request the first STAGES segments into the stages that follow the ring position
@@ -215,7 +200,6 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
             }
         }
         // block and segment counts of a slice fit 32 bits (a slice is at most 1/256 of a chunk beyond 4 MiB)
-        const uint32_t my_blocks = (uint32_t)(my_bytes >> 6);
         const uint32_t warp_blocks = (uint32_t)(warp_bytes >> 6);
         const uint32_t nseg32 = (uint32_t)nseg;
         int in_stage = 0;
@@ -247,13 +231,13 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
                     if (failed) break;
                 }
             }
-            // With tiled copies every lane of a group has the same number of blocks (lanes beyond the blob's
-            // last chunk hash the zeros their rows were filled with and store nothing), and a fetch past the
-            // last block reads ring memory that is never used: neither needs a branch.  Measured: the loop
-            // without the two branches and with 32-bit counters is 1.7 % faster on the 112 GiB launch and 3.3 %
-            // where every scheduler runs a single group.
-            if (TILED || blk + 1 < warp_blocks) fetch(stage, in_stage);
-            if (TILED || blk < my_blocks) sha256_compress<ADD>(st, w, one);
+            // Every lane of a group has the same number of blocks (lanes beyond the blob's last chunk hash the
+            // zeros their rows were filled with and store nothing), and a fetch past the last block reads ring
+            // memory that is never used: neither needs a branch.  Measured: the loop without the two branches
+            // and with 32-bit counters is 1.7 % faster on the 112 GiB launch and 3.3 % where every scheduler
+            // runs a single group.
+            fetch(stage, in_stage);
+            sha256_compress<ADD>(st, w, one);
         }
         if (failed) break;
 
@@ -360,19 +344,20 @@ bool make_chunk_tensor_map(CUtensorMap *map, const uint8_t *d_data, uint64_t chu
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool TILED, bool PREFIX>
+thread_local const char *t_instance = "";
+
+template <bool PREFIX>
 cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
                           const uint32_t *d_one, int sm_count, cudaStream_t stream) {
     // Three instances: up to eight workers per SM with three stages each (arrival order or first workers
     // first), and twelve workers with two stages each for launches that keep all of them busy.
     constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8, MANY_STAGES = 2, MANY_WARPS = 12;
-    constexpr size_t smem_per_warp = TILED ? (size_t)STAGES * 8192 : (size_t)STAGES * 32 * (SEG + 16);
-    constexpr size_t many_per_warp = TILED ? (size_t)MANY_STAGES * 8192 : (size_t)MANY_STAGES * 32 * (SEG + 16);
-    constexpr size_t smem_pad = TILED ? 1024 : 0;
-    auto kernel_plain = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX, false, 0>;
-    auto kernel_fwf = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, TILED, PREFIX, true, 0>;
-    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, TILED, PREFIX, false, 2>;
+    constexpr size_t smem_per_warp = (size_t)STAGES * 8192, many_per_warp = (size_t)MANY_STAGES * 8192;
+    constexpr size_t smem_pad = 1024;
+    auto kernel_plain = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, false, 0>;
+    auto kernel_fwf = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, true, 0>;
+    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, PREFIX, false, 2>;
     static bool configured[kMaxDevices] = {}, configured_fwf[kMaxDevices] = {}, configured_many[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel_plain, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
     if (cudaError_t e0 = ensure_dynamic_smem(kernel_fwf, MAX_WARPS * smem_per_warp + smem_pad, configured_fwf); e0 != cudaSuccess) return e0;
@@ -407,12 +392,15 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     // From twelve groups per SM on, three warps per scheduler hide the longer chains of multiply-add
     // additions, which take a tenth of the ALU pipe's load: 917 GB/s against 884 (32 GiB in 64 KiB chunks).
     if (groups >= (uint64_t)MANY_WARPS * (uint64_t)sm_count) {
+        t_instance = "12 workers per SM";
         kernel_many<<<(unsigned)sm_count, 32 * MANY_WARPS, MANY_WARPS * many_per_warp + smem_pad, stream>>>(
             map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q,
             next_slice, mid, d_one);
         return cudaGetLastError();
     }
     auto kernel = first_workers_first ? kernel_fwf : kernel_plain;
+    t_instance = first_workers_first ? "8 workers per SM, first workers first"
+                                     : (warps == 4 ? "4 workers per SM" : "8 workers per SM, arrival order");
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
         map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
         mid, d_one);
@@ -421,8 +409,11 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
 
 }  // namespace
 
-// Returns how many chunks (from the front of the blob) the launch covers: with the tiled copies only whole
-// chunks can be described to the TMA unit, so a short last chunk is left to the caller (*covered = n - 1).
+const char *sliced_instance_name() { return t_instance; }
+
+// Returns in *covered how many chunks (from the front of the blob) the launch hashes: only whole chunks can be
+// described to the TMA unit, so a short last chunk is left to the caller (*covered = n - 1), and so is the
+// whole blob (*covered = 0, nothing launched) if the tensor map cannot be made.
 cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                       uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
                                       const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *covered,
@@ -430,19 +421,14 @@ cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, ui
     const uint64_t whole = nbytes / chunk_bytes;          // n_chunks or n_chunks - 1
     alignas(64) CUtensorMap map;
     std::memset(&map, 0, sizeof map);
-    if (whole > 0 && make_chunk_tensor_map(&map, d_data, chunk_bytes, whole)) {
-        *covered = whole;
-        const uint64_t bytes = whole * chunk_bytes;
-        return zero_prefix ? launch_sliced<true, true>(map, d_data, bytes, chunk_bytes, whole, d_digests, d_status,
-                                                       d_scratch, d_one, sm_count, stream)
-                           : launch_sliced<true, false>(map, d_data, bytes, chunk_bytes, whole, d_digests, d_status,
-                                                        d_scratch, d_one, sm_count, stream);
-    }
-    *covered = n_chunks;
-    return zero_prefix ? launch_sliced<false, true>(map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
-                                                    d_scratch, d_one, sm_count, stream)
-                       : launch_sliced<false, false>(map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status,
-                                                     d_scratch, d_one, sm_count, stream);
+    *covered = 0;
+    if (whole == 0 || !make_chunk_tensor_map(&map, d_data, chunk_bytes, whole)) return cudaSuccess;
+    *covered = whole;
+    const uint64_t bytes = whole * chunk_bytes;
+    return zero_prefix ? launch_sliced<true>(map, d_data, bytes, chunk_bytes, whole, d_digests, d_status, d_scratch, d_one,
+                                             sm_count, stream)
+                       : launch_sliced<false>(map, d_data, bytes, chunk_bytes, whole, d_digests, d_status, d_scratch, d_one,
+                                              sm_count, stream);
 }
 
 }  // namespace ivk

@@ -38,7 +38,7 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
 //                 endian-swap PRMT.
 // PAIR: blocks handed over per W+K slot (1 or 2); with 2 the barrier traffic per block halves.
 // PREFIX (chunks only): message i is 0x00 || chunk i, the RFC 6962 leaf hash.
-template <int SEG, int STAGES, int NSLOT, int MODE, bool RAGGED, int PAIR = 1, bool PREFIX = false>
+template <int SEG, int STAGES, int NSLOT, bool RAGGED, int PAIR = 1, bool PREFIX = false>
 __global__ void __launch_bounds__(64)
 hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                          uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
@@ -224,7 +224,7 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
             if (failed) break;
         }
         const uint32_t src = wk_base + slot * kWkSlot + in_slot * kWkBlock;
-        rounds64<MODE>(v, src, one);
+        rounds64(v, src, one);
         const bool slot_done = in_slot == PAIR - 1 || blk + 1 == warp_total;
         if (slot_done) {
             __syncwarp();                              // all 32 lanes have their values in registers
@@ -259,10 +259,10 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
     // 512-byte segments, three data stages, three W+K slots of two blocks each (two blocks per hand-over
     // halve the barrier traffic: +1 % over four single-block slots; 104 KB per CTA, two CTAs per SM); the additions that close the two state
     // recurrences stay three-input ALU adds, the others go to the FMA pipe (placement 3, the fastest measured).
-    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, MODE = 3, PAIR = 2;
+    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, PAIR = 2;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
-    auto kernel = zero_prefix ? hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false, PAIR, true>
-                              : hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, false, PAIR, false>;
+    auto kernel = zero_prefix ? hash_chunks_split_kernel<SEG, STAGES, NSLOT, false, PAIR, true>
+                              : hash_chunks_split_kernel<SEG, STAGES, NSLOT, false, PAIR, false>;
     static bool configured[2][kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured[zero_prefix ? 1 : 0]); e0 != cudaSuccess) return e0;
     const uint64_t blocks = (n_chunks + 31) / 32;
@@ -275,9 +275,9 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
 cudaError_t launch_hash_ragged_split(const uint8_t *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
                                      const uint32_t *d_order, uint64_t n, uint8_t *d_digests, uint32_t *d_status,
                                      const uint32_t *d_one, iv_sha_state *d_states, int finish, cudaStream_t stream) {
-    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, MODE = 3, PAIR = 2;
+    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, PAIR = 2;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 32) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
-    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, MODE, true, PAIR>;
+    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, true, PAIR>;
     static bool configured[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
     const uint64_t blocks = (n + 31) / 32;

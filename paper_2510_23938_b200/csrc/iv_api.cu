@@ -12,6 +12,7 @@ struct iv_ctx {
     int last_cuda_error = 0;
     uint64_t launches = 0;
     const char *leaf_kernel = "";             // name of the leaf-hashing kernel the last call launched
+    const char *leaf_instance = "";           // and, where that kernel has several launch shapes, which one
 
     // small fixed block: tickets, work-queue counter, root
     uint32_t *d_tickets = nullptr;            // kMerkleMaxPasses + 1 words
@@ -130,6 +131,11 @@ int ensure_variant_tree_scratch(iv_ctx *ctx, uint64_t records) {
     return IV_OK;
 }
 
+// After a leaf-hashing launch: which launch shape the kernel ran in, for the kernels that have several.
+void note_leaf_instance(iv_ctx *ctx) {
+    ctx->leaf_instance = std::strcmp(ctx->leaf_kernel, "hash_chunks_sliced_kernel") == 0 ? ivk::sliced_instance_name() : "";
+}
+
 // Leaf hashing with the scratch the launch shape needs.
 int hash_leaves(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n,
                 uint8_t *d_digests, cudaStream_t stream) {
@@ -142,6 +148,7 @@ int hash_leaves(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t ch
     }
     IV_TRY(ctx, ivk::launch_hash_chunks(d_data, nbytes, chunk_bytes, n, d_digests, ctx->sm_count, ctx->d_status,
                                         ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel));
+    note_leaf_instance(ctx);
     return IV_OK;
 }
 
@@ -157,6 +164,7 @@ int hash_leaves_rfc6962(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uin
     }
     IV_TRY(ctx, ivk::launch_hash_chunks_rfc6962(d_data, nbytes, chunk_bytes, n, d_digests, ctx->sm_count, ctx->d_status,
                                                 ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel));
+    note_leaf_instance(ctx);
     return IV_OK;
 }
 
@@ -350,6 +358,22 @@ int iv_last_cuda_error(const iv_ctx *ctx) { return ctx ? ctx->last_cuda_error : 
 uint64_t iv_kernel_launches(const iv_ctx *ctx) { return ctx ? ctx->launches : 0; }
 
 const char *iv_last_leaf_kernel(const iv_ctx *ctx) { return ctx ? ctx->leaf_kernel : ""; }
+
+const char *iv_last_leaf_instance(const iv_ctx *ctx) { return ctx ? ctx->leaf_instance : ""; }
+
+int iv_selftest_wait_timeout(iv_ctx *ctx, uint64_t limit_cycles, uint64_t *h_waited_cycles, void *cuda_stream) {
+    if (!ctx || limit_cycles == 0 || limit_cycles > 4000000000ull) return IV_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    IV_TRY(ctx, ivk::launch_wait_timeout_selftest(limit_cycles, ctx->d_status, ctx->d_queue, stream, &ctx->launches));
+    if (h_waited_cycles) {
+        unsigned long long waited = 0;
+        IV_TRY(ctx, cudaMemcpyAsync(&waited, ctx->d_queue, sizeof waited, cudaMemcpyDeviceToHost, stream));
+        IV_TRY(ctx, cudaStreamSynchronize(stream));
+        *h_waited_cycles = waited;
+    }
+    return IV_OK;
+}
 
 int iv_device_status(iv_ctx *ctx, uint32_t *h_status) {
     if (!ctx || !h_status) return IV_ERR_INVALID_ARG;
@@ -846,7 +870,7 @@ int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t block
     if (!ctx || !h_out || warps_per_block == 0 || warps_per_block > 32 || blocks_per_sm == 0 ||
         blocks_per_sm > 32 || active_lanes == 0 || active_lanes > 32 || iters == 0)
         return IV_ERR_INVALID_ARG;
-    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_SHA256_ADD7) return IV_ERR_INVALID_ARG;
+    if (kind < IV_PROBE_IADD3 || kind > IV_PROBE_SCHEDULE) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     const unsigned blocks = blocks_per_sm * (unsigned)ctx->sm_count;
     unsigned long long *d_cycles = nullptr;
@@ -869,7 +893,7 @@ int iv_probe_alu(iv_ctx *ctx, int kind, uint32_t warps_per_block, uint32_t block
         for (unsigned b = 0; b < blocks; ++b) sum += (double)h_cycles[b];
         const double mean = sum / blocks;
         double per_thread = (double)ivk::probe_ops_per_thread(kind, iters);
-        if (kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_FMA || kind >= IV_PROBE_ROUNDS_M0) per_thread *= 64.0;       // bytes per compression
+        if (ivk::probe_counts_blocks(kind)) per_thread *= 64.0;       // bytes per compression
         h_out[0] = (double)blocks_per_sm * warps_per_block * active_lanes * per_thread / mean;
         h_out[1] = mean;
     } else {

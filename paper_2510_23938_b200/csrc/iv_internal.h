@@ -57,6 +57,9 @@ cudaError_t launch_hash_chunks_sliced(const uint8_t *d_data, uint64_t nbytes, ui
                                       uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
                                       const uint32_t *d_one, int sm_count, cudaStream_t stream, uint64_t *covered,
                                       bool zero_prefix = false);
+// Which instance of the sliced kernel the calling host thread's last launch_hash_chunks_sliced picked
+// (worker count and service order); static text.
+const char *sliced_instance_name();
 
 // The same two-warp kernel for tensors at any alignment; message k of the launch is tensor d_order[k]
 // (d_order may be NULL for index order).
@@ -161,9 +164,16 @@ cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, u
 cudaError_t launch_merkle_root_rfc6962(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root, uint8_t *d_scratch_a,
                                        uint8_t *d_scratch_b, cudaStream_t stream, uint64_t *launches);
 
+// selftest.cu --------------------------------------------------------------
+// One warp waits (bounded by limit_cycles SM clocks) on a barrier nobody arrives at, then sets *d_status to
+// IVK_DEV_TIMEOUT and returns; *d_waited (may be NULL) receives the clocks it waited.
+cudaError_t launch_wait_timeout_selftest(uint64_t limit_cycles, uint32_t *d_status, unsigned long long *d_waited,
+                                         cudaStream_t stream, uint64_t *launches);
+
 // probe_alu.cu -------------------------------------------------------------
 cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t iters, uint32_t active_lanes,
                          unsigned long long *d_cycles, uint32_t *d_sink, cudaStream_t stream);
 uint64_t probe_ops_per_thread(int kind, uint32_t iters);
+bool probe_counts_blocks(int kind);   // the kind reports message bytes (one 64-byte block per trip), not instructions
 
 }  // namespace ivk

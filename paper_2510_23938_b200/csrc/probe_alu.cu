@@ -96,78 +96,21 @@ __global__ void probe_sha_kernel(uint32_t iters, uint32_t active_lanes, unsigned
     if (threadIdx.x == 0) cycles[blockIdx.x] = (unsigned long long)(t1 - t0);
 }
 
-// Register-only SHA-256 over a message that does not depend on the chaining value (as data from
-// memory does not), so the schedule of one block is free to overlap the rounds of the one before.
-__global__ void probe_sha_stream_kernel(uint32_t iters, uint32_t active_lanes, unsigned long long *cycles, uint32_t *sink) {
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t mul = sink[1] * 0x9e3779b9u;       // the host stored 1 in sink[1]
-    uint32_t st[8];
-    sha256_init(st);
-    st[0] ^= threadIdx.x + blockIdx.x * blockDim.x;
-    __syncthreads();
-    const long long t0 = clock64();
-    if (lane < active_lanes) {
-        uint32_t w[16];
-        uint32_t x = threadIdx.x;
-#pragma unroll 1
-        for (uint32_t it = 0; it < iters; ++it) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) w[i] = bswap32(x + (uint32_t)i * mul);
-            x += mul;
-            sha256_compress<0>(st, w, 1u);
-        }
-    }
-    __syncthreads();
-    const long long t1 = clock64();
-    if ((st[0] ^ st[5]) == 0x12345u) sink[0] = st[1];
-    if (threadIdx.x == 0) cycles[blockIdx.x] = (unsigned long long)(t1 - t0);
-}
-
-// The consumer half alone: 64 rounds per trip, W + K read from a (constant) shared-memory slot.
-// HANDSHAKE adds what the split kernel's consumer does around the rounds: a wait on a "full"
-// barrier (completed just before by lane 0 itself), the warp barrier, the "empty" arrival and the
-// feed-forward, so the difference to the plain kind is the cost of the hand-over.
-template <int MODE, bool HANDSHAKE = false>
+// The consumer half of the two-warp kernel alone: 64 rounds per trip, W + K read from a (constant)
+// shared-memory slot.
 __global__ void probe_rounds_kernel(uint32_t iters, uint32_t active_lanes, unsigned long long *cycles, uint32_t *sink) {
     __shared__ __align__(16) uint32_t slot[32 * 68];
-    __shared__ __align__(8) uint64_t bars[2];
-    if (threadIdx.x == 0) {
-        tma::mbar_init(tma::smem_u32(&bars[0]), 1);
-        tma::mbar_init(tma::smem_u32(&bars[1]), 1);
-        tma::fence_barrier_init();
-    }
     for (int i = threadIdx.x; i < 32 * 68; i += blockDim.x) slot[i] = i * 2654435761u;
     __syncthreads();
     const uint32_t one = sink[1];        // the host stored 1 there; the compiler cannot know
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t src = tma::smem_u32(slot) + lane * 272;
-    uint32_t v[8], st[8];
+    uint32_t v[8];
     sha256_init(v);
     v[0] ^= threadIdx.x;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) st[k] = v[k];
-    const uint32_t bar_full = tma::smem_u32(&bars[0]), bar_empty = tma::smem_u32(&bars[1]);
-    uint32_t parity = 0;
     const long long t0 = clock64();
     if (lane < active_lanes)
-        for (uint32_t it = 0; it < iters; ++it) {
-            if (HANDSHAKE) {
-                if (lane == 0) tma::mbar_arrive(bar_full);
-                if (!__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_full, parity))) break;
-                parity ^= 1u;
-            }
-            rounds64<MODE>(v, src, one);
-            if (HANDSHAKE) {
-                __syncwarp();
-                if (lane == 0) tma::mbar_arrive(bar_empty);
-                const uint32_t keep = (it < iters) ? one : 0u;
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    st[k] = padd<true>(v[k], st[k], keep);
-                    v[k] = st[k];
-                }
-            }
-        }
+        for (uint32_t it = 0; it < iters; ++it) rounds64(v, src, one);
     __syncthreads();
     const long long t1 = clock64();
     if ((v[0] ^ v[5]) == 0x12345u) sink[0] = v[1];
@@ -213,29 +156,21 @@ cudaError_t launch_probe(int kind, unsigned blocks, unsigned threads, uint32_t i
         case IV_PROBE_LAT_SHF: probe_kernel<IV_PROBE_SHF, 1><<<blocks, threads, 0, stream>>>(iters, active_lanes, 7u, sc, d_cycles, d_sink); break;
         case IV_PROBE_LAT_IMAD: probe_kernel<IV_PROBE_IMAD, 1><<<blocks, threads, 0, stream>>>(iters, active_lanes, sb, sc, d_cycles, d_sink); break;
         case IV_PROBE_LAT_CROSS: probe_kernel<IV_PROBE_LAT_CROSS, 1><<<blocks, threads, 0, stream>>>(iters, active_lanes, sb, sc, d_cycles, d_sink); break;
-        case IV_PROBE_ROUNDS_M0: probe_rounds_kernel<0><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_ROUNDS_M1: probe_rounds_kernel<1><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_ROUNDS_M2: probe_rounds_kernel<2><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_ROUNDS_M3: probe_rounds_kernel<3><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_ROUNDS_M3_HANDSHAKE: probe_rounds_kernel<3, true><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_ROUNDS_M4: probe_rounds_kernel<4><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_ROUNDS_M5: probe_rounds_kernel<5><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_ROUNDS: probe_rounds_kernel<<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_SCHEDULE: probe_schedule_kernel<<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         case IV_PROBE_SHA256: probe_sha_kernel<0><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256_FMA: probe_sha_kernel<1><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256_ADD2: probe_sha_kernel<2><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256_ADD3: probe_sha_kernel<3><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256_ADD4: probe_sha_kernel<4><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256_ADD6: probe_sha_kernel<6><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256_ADD7: probe_sha_kernel<7><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
-        case IV_PROBE_SHA256_STREAM: probe_sha_stream_kernel<<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
+        case IV_PROBE_SHA256_SCHED_FMA: probe_sha_kernel<2><<<blocks, threads, 0, stream>>>(iters, active_lanes, d_cycles, d_sink); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();
 }
 
+bool probe_counts_blocks(int kind) {
+    return kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_SCHED_FMA || kind == IV_PROBE_ROUNDS || kind == IV_PROBE_SCHEDULE;
+}
+
 uint64_t probe_ops_per_thread(int kind, uint32_t iters) {
-    if (kind == IV_PROBE_SHA256 || kind == IV_PROBE_SHA256_FMA || kind >= IV_PROBE_ROUNDS_M0) return iters;                        // compressions
+    if (probe_counts_blocks(kind)) return iters;                                      // compressions
     if (kind == IV_PROBE_LAT_CROSS) return (uint64_t)iters * kUnroll * 2;             // two instructions per trip
     if (kind >= IV_PROBE_LAT_IADD3) return (uint64_t)iters * kUnroll;                 // one dependent chain
     return (uint64_t)iters * kUnroll * kThroughputChains;                              // instructions

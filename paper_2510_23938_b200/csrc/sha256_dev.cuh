@@ -59,74 +59,30 @@ __device__ __forceinline__ uint32_t padd(uint32_t a, uint32_t b, uint32_t one) {
 
 // Where the additions of a compression go (template parameter ADD):
 //   0  left to the compiler (mostly three-input adds on the ALU pipe)
-//   1  every addition a multiply-add on the FMA pipe
-//   2  the message schedule's additions on the FMA pipe, the rounds' left to the compiler
-//   3  schedule additions and the part of T1 that does not depend on this round's e (h + K + W)
-//      on the FMA pipe; the additions that close the e and a recurrences stay three-input ALU adds
-//   4  as 3 for the rounds, the schedule left to the compiler
-//   6  schedule: the two plain shifts as multiply-high on the FMA pipe; additions left to the compiler
-//   7  schedule: shifts and rotations on the FMA pipe (x >> n = hi(x * 2^(32-n)); rotr(x, n) = that plus
-//      lo(x * 2^(32-n)), two multiply-adds instead of one funnel shift); additions left to the compiler
-__host__ __device__ constexpr bool add_sched_fma(int add) { return add == 1 || add == 2 || add == 3; }
-
-// x >> N and rotr(x, N) formed on the FMA pipe; `one` is 1 in a way the compiler cannot see.
-template <int N>
-__device__ __forceinline__ uint32_t shr_fma(uint32_t x, uint32_t one) { return __umulhi(x, one << (32 - N)); }
-template <int N>
-__device__ __forceinline__ uint32_t rotr_fma(uint32_t x, uint32_t one) {
-    const uint32_t m = one << (32 - N);
-    uint32_t r;
-    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(x), "r"(m), "r"(__umulhi(x, m)));
-    return r;
-}
+//   2  the message schedule's additions and the feed-forward on the FMA pipe, the rounds' left to the
+//      compiler; pays only with three warps per SM scheduler, which hide the longer dependency chains
 
 // One round (FIPS 180-4 section 6.2.2 step 3):
 //   T1 = h + S1(e) + Ch(e,f,g) + K + W;  d += T1;  h = T1 + S0(a) + Maj(a,b,c).
 // The caller rotates the variable names instead of moving values.
-template <int ADD>
 __device__ __forceinline__ void sha_round(uint32_t a, uint32_t b, uint32_t c, uint32_t &d, uint32_t e, uint32_t f,
-                                          uint32_t g, uint32_t &h, uint32_t k, uint32_t w, uint32_t one) {
-    if (ADD == 1) {
-        const uint32_t kw = padd<true>(w, k, one);
-        const uint32_t x = padd<true>(h, kw, one);
-        const uint32_t y = padd<true>(x, f_ch(e, f, g), one);
-        const uint32_t t1 = padd<true>(y, big_s1(e), one);
-        const uint32_t q = padd<true>(big_s0(a), f_maj(a, b, c), one);
-        d = padd<true>(d, t1, one);
-        h = padd<true>(t1, q, one);
-    } else if (ADD == 3 || ADD == 4) {
-        const uint32_t kw = padd<true>(w, k, one);
-        const uint32_t x = padd<true>(h, kw, one);
-        const uint32_t t1 = x + f_ch(e, f, g) + big_s1(e);
-        d += t1;
-        h = t1 + big_s0(a) + f_maj(a, b, c);
-    } else {
-        const uint32_t t1 = h + big_s1(e) + f_ch(e, f, g) + (k + w);
-        d += t1;
-        h = t1 + big_s0(a) + f_maj(a, b, c);
-    }
+                                          uint32_t g, uint32_t &h, uint32_t k, uint32_t w) {
+    const uint32_t t1 = h + big_s1(e) + f_ch(e, f, g) + (k + w);
+    d += t1;
+    h = t1 + big_s0(a) + f_maj(a, b, c);
 }
 
 // Message-schedule step in the rolling 16-word window (i = t mod 16):
 // W[t] = s1(W[t-2]) + W[t-7] + s0(W[t-15]) + W[t-16].
 template <int ADD>
 __device__ __forceinline__ void sha_sched(uint32_t (&w)[16], int i, uint32_t one) {
-    if (ADD == 6 || ADD == 7) {
-        const uint32_t x1 = w[(i + 14) & 15], x0 = w[(i + 1) & 15];
-        const uint32_t s1 = ADD == 7 ? xor3(rotr_fma<17>(x1, one), rotr_fma<19>(x1, one), shr_fma<10>(x1, one))
-                                     : xor3(rotr(x1, 17), rotr(x1, 19), shr_fma<10>(x1, one));
-        const uint32_t s0 = ADD == 7 ? xor3(rotr_fma<7>(x0, one), rotr_fma<18>(x0, one), shr_fma<3>(x0, one))
-                                     : xor3(rotr(x0, 7), rotr(x0, 18), shr_fma<3>(x0, one));
-        w[i & 15] = s1 + w[(i + 9) & 15] + s0 + w[i & 15];
-        return;
-    }
-    constexpr bool F = add_sched_fma(ADD);
+    constexpr bool F = ADD == 2;
     const uint32_t s = padd<F>(small_s1(w[(i + 14) & 15]), w[(i + 9) & 15], one);
     const uint32_t t = padd<F>(small_s0(w[(i + 1) & 15]), w[i & 15], one);
     w[i & 15] = padd<F>(s, t, one);
 }
 
-#define IV_ROUND(a, b, c, d, e, f, g, h, k, wv) ivk::sha_round<ADD>(a, b, c, d, e, f, g, h, k, wv, one)
+#define IV_ROUND(a, b, c, d, e, f, g, h, k, wv) ivk::sha_round(a, b, c, d, e, f, g, h, k, wv)
 
 // Eight rounds starting at a round index that is a multiple of 8 (so the
 // variable rotation returns to a..h), constants k0..k7 from FIPS 180-4 4.2.2.
@@ -147,10 +103,11 @@ __device__ __forceinline__ void sha_sched(uint32_t (&w)[16], int i, uint32_t one
     ivk::sha_sched<ADD>(w, (i) + 6, one); ivk::sha_sched<ADD>(w, (i) + 7, one)
 
 // st <- compress(st, block) where w[0..15] holds the block as big-endian words.
-// w is destroyed (it is the rolling schedule window).  ADD places the additions (see above);
+// w is destroyed (it is the rolling schedule window).  ADD places the additions (0 or 2, see above);
 // for ADD != 0 `one` must hold the value 1 in a way the compiler cannot see through.
 template <int ADD = 0>
 __device__ __forceinline__ void sha256_compress(uint32_t (&st)[8], uint32_t (&w)[16], uint32_t one = 1u) {
+    static_assert(ADD == 0 || ADD == 2, "addition placements 0 and 2 exist");
     uint32_t v[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = st[i];
@@ -171,7 +128,7 @@ __device__ __forceinline__ void sha256_compress(uint32_t (&st)[8], uint32_t (&w)
     IV_ROUNDS8(v, w, 8, 0x748f82eeu, 0x78a5636fu, 0x84c87814u, 0x8cc70208u, 0x90befffau, 0xa4506cebu, 0xbef9a3f7u, 0xc67178f2u);
 
 #pragma unroll
-    for (int i = 0; i < 8; ++i) st[i] = padd<ADD != 0 && ADD < 6>(st[i], v[i], one);
+    for (int i = 0; i < 8; ++i) st[i] = padd<ADD != 0>(st[i], v[i], one);
 }
 
 // The last block of a message whose length is a multiple of 64 bytes holds no

@@ -66,70 +66,36 @@ __device__ __forceinline__ void produce_wk(uint32_t (&w)[16], uint32_t dst, uint
     store_wk16<48>(w, dst, one);
 }
 
-// One round with kw = W[t] + K[t] already formed.  The ten SHF/LOP3 of a round must run on the
-// ALU pipe; MODE says where the additions go (`one` is a register that holds 1, so that
-// a * one + b is a real multiply-add on the FMA pipe):
-//   0  all additions left to the compiler (IADD3 on the ALU pipe)
-//   1  all additions on the FMA pipe
-//   2  the addition that closes the e -> e recurrence stays a three-input ALU add, the rest on the FMA pipe
-//   3  both recurrences (e and a) close with three-input ALU adds, the rest on the FMA pipe
-template <int MODE>
+// One round with kw = W[t] + K[t] already formed.  The ten SHF/LOP3 of a round must run on the ALU pipe.  Of
+// the additions, the two that close the state recurrences (e and a) stay three-input ALU adds; the ones that
+// feed them from values a round old go to the FMA pipe (`one` is a register that holds 1, so that
+// a * one + b is a real multiply-add there).  The fastest of the placements measured.
 __device__ __forceinline__ void round_kw(uint32_t a, uint32_t b, uint32_t c, uint32_t &d, uint32_t e, uint32_t f,
                                          uint32_t g, uint32_t &h, uint32_t kw, uint32_t one) {
-    if (MODE == 0) {
-        const uint32_t t1 = h + big_s1(e) + f_ch(e, f, g) + kw;
-        d += t1;
-        h = t1 + big_s0(a) + f_maj(a, b, c);
-    } else if (MODE == 4 || MODE == 5) {
-        // e' = (d + h + kw) + Ch + S1 closes the e recurrence with ONE three-input ALU add after S1;
-        // everything that feeds it is formed on the FMA pipe from values that are a round old.
-        const uint32_t x = padd<true>(h, kw, one);
-        const uint32_t p = padd<true>(x, d, one);
-        const uint32_t s1 = big_s1(e);
-        const uint32_t ch = f_ch(e, f, g);
-        const uint32_t q = padd<true>(big_s0(a), f_maj(a, b, c), one);
-        uint32_t t1;
-        if (MODE == 4) {
-            d = p + ch + s1;
-            t1 = padd<true>(x, ch, one);
-            t1 = padd<true>(t1, s1, one);
-        } else {
-            t1 = x + ch + s1;
-            d = p + ch + s1;
-        }
-        h = padd<true>(t1, q, one);
-    } else {
-        const uint32_t x = padd<true>(h, kw, one);
-        const uint32_t y = padd<true>(x, f_ch(e, f, g), one);
-        const uint32_t s1 = big_s1(e);
-        const uint32_t t1 = padd<true>(y, s1, one);
-        if (MODE == 1) d = padd<true>(d, t1, one);
-        else d = d + y + s1;
-        if (MODE == 3) {
-            h = t1 + big_s0(a) + f_maj(a, b, c);
-        } else {
-            const uint32_t q = padd<true>(big_s0(a), f_maj(a, b, c), one);
-            h = padd<true>(t1, q, one);
-        }
-    }
+    const uint32_t x = padd<true>(h, kw, one);
+    const uint32_t y = padd<true>(x, f_ch(e, f, g), one);
+    const uint32_t s1 = big_s1(e);
+    const uint32_t t1 = padd<true>(y, s1, one);
+    d = d + y + s1;
+    h = t1 + big_s0(a) + f_maj(a, b, c);
 }
 
 // Four rounds (T0 a multiple of 4) on W + K values already in registers.
-template <int T0, int MODE>
+template <int T0>
 __device__ __forceinline__ void rounds4(uint32_t (&v)[8], const uint32_t (&k)[4], uint32_t one) {
     constexpr int r = T0 & 7;   // 0 or 4: position in the eight-round rotation of the variable names
-    round_kw<MODE>(v[(8 - r) & 7], v[(9 - r) & 7], v[(10 - r) & 7], v[(11 - r) & 7], v[(12 - r) & 7],
+    round_kw(v[(8 - r) & 7], v[(9 - r) & 7], v[(10 - r) & 7], v[(11 - r) & 7], v[(12 - r) & 7],
                    v[(13 - r) & 7], v[(14 - r) & 7], v[(15 - r) & 7], k[0], one);
-    round_kw<MODE>(v[(7 - r) & 7], v[(8 - r) & 7], v[(9 - r) & 7], v[(10 - r) & 7], v[(11 - r) & 7],
+    round_kw(v[(7 - r) & 7], v[(8 - r) & 7], v[(9 - r) & 7], v[(10 - r) & 7], v[(11 - r) & 7],
                    v[(12 - r) & 7], v[(13 - r) & 7], v[(14 - r) & 7], k[1], one);
-    round_kw<MODE>(v[(6 - r) & 7], v[(7 - r) & 7], v[(8 - r) & 7], v[(9 - r) & 7], v[(10 - r) & 7],
+    round_kw(v[(6 - r) & 7], v[(7 - r) & 7], v[(8 - r) & 7], v[(9 - r) & 7], v[(10 - r) & 7],
                    v[(11 - r) & 7], v[(12 - r) & 7], v[(13 - r) & 7], k[2], one);
-    round_kw<MODE>(v[(5 - r) & 7], v[(6 - r) & 7], v[(7 - r) & 7], v[(8 - r) & 7], v[(9 - r) & 7],
+    round_kw(v[(5 - r) & 7], v[(6 - r) & 7], v[(7 - r) & 7], v[(8 - r) & 7], v[(9 - r) & 7],
                    v[(10 - r) & 7], v[(11 - r) & 7], v[(12 - r) & 7], k[3], one);
 }
 
 // Rounds T0 .. T0+3 with the W + K values of rounds T0+AHEAD .. fetched first (software prefetch).
-template <int T0, int MODE, int AHEAD>
+template <int T0, int AHEAD>
 __device__ __forceinline__ void rounds4_step(uint32_t (&v)[8], uint32_t (&kbuf)[16], uint32_t src, uint32_t one) {
     constexpr int TN = T0 + AHEAD;
     if (TN < 64) {
@@ -137,25 +103,24 @@ __device__ __forceinline__ void rounds4_step(uint32_t (&v)[8], uint32_t (&kbuf)[
         tma::ld_shared_v4_at<4 * (TN < 64 ? TN : 0)>(src, kbuf[o], kbuf[o + 1], kbuf[o + 2], kbuf[o + 3]);
     }
     const uint32_t k[4] = {kbuf[(T0 & 15)], kbuf[(T0 & 15) + 1], kbuf[(T0 & 15) + 2], kbuf[(T0 & 15) + 3]};
-    rounds4<T0, MODE>(v, k, one);
+    rounds4<T0>(v, k, one);
 }
 
 // All 64 rounds of one block, W[t] + K[t] read from the shared-memory slot at `src`.
-template <int MODE>
 __device__ __forceinline__ void rounds64(uint32_t (&v)[8], uint32_t src, uint32_t one) {
     constexpr int AHEAD = 12;          // W + K values are requested three groups of four rounds early
     uint32_t kbuf[16];
     tma::ld_shared_v4_at<0>(src, kbuf[0], kbuf[1], kbuf[2], kbuf[3]);
     tma::ld_shared_v4_at<16>(src, kbuf[4], kbuf[5], kbuf[6], kbuf[7]);
     tma::ld_shared_v4_at<32>(src, kbuf[8], kbuf[9], kbuf[10], kbuf[11]);
-    rounds4_step<0, MODE, AHEAD>(v, kbuf, src, one);  rounds4_step<4, MODE, AHEAD>(v, kbuf, src, one);
-    rounds4_step<8, MODE, AHEAD>(v, kbuf, src, one);  rounds4_step<12, MODE, AHEAD>(v, kbuf, src, one);
-    rounds4_step<16, MODE, AHEAD>(v, kbuf, src, one); rounds4_step<20, MODE, AHEAD>(v, kbuf, src, one);
-    rounds4_step<24, MODE, AHEAD>(v, kbuf, src, one); rounds4_step<28, MODE, AHEAD>(v, kbuf, src, one);
-    rounds4_step<32, MODE, AHEAD>(v, kbuf, src, one); rounds4_step<36, MODE, AHEAD>(v, kbuf, src, one);
-    rounds4_step<40, MODE, AHEAD>(v, kbuf, src, one); rounds4_step<44, MODE, AHEAD>(v, kbuf, src, one);
-    rounds4_step<48, MODE, AHEAD>(v, kbuf, src, one); rounds4_step<52, MODE, AHEAD>(v, kbuf, src, one);
-    rounds4_step<56, MODE, AHEAD>(v, kbuf, src, one); rounds4_step<60, MODE, AHEAD>(v, kbuf, src, one);
+    rounds4_step<0, AHEAD>(v, kbuf, src, one);  rounds4_step<4, AHEAD>(v, kbuf, src, one);
+    rounds4_step<8, AHEAD>(v, kbuf, src, one);  rounds4_step<12, AHEAD>(v, kbuf, src, one);
+    rounds4_step<16, AHEAD>(v, kbuf, src, one); rounds4_step<20, AHEAD>(v, kbuf, src, one);
+    rounds4_step<24, AHEAD>(v, kbuf, src, one); rounds4_step<28, AHEAD>(v, kbuf, src, one);
+    rounds4_step<32, AHEAD>(v, kbuf, src, one); rounds4_step<36, AHEAD>(v, kbuf, src, one);
+    rounds4_step<40, AHEAD>(v, kbuf, src, one); rounds4_step<44, AHEAD>(v, kbuf, src, one);
+    rounds4_step<48, AHEAD>(v, kbuf, src, one); rounds4_step<52, AHEAD>(v, kbuf, src, one);
+    rounds4_step<56, AHEAD>(v, kbuf, src, one); rounds4_step<60, AHEAD>(v, kbuf, src, one);
 }
 
 }  // namespace ivk

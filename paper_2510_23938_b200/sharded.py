@@ -65,6 +65,12 @@ def sharded_root(ctx, local_leaves: torch.Tensor, plan: ShardPlan, rank: int, gr
         mine[:n_mine] = nodes
     if plan.world == 1:
         gathered = [mine]
+    elif mine.is_cuda and dist.get_backend(group) == "gloo":
+        # gloo gathers host tensors only (checking the multi-rank logic without NCCL): stage through the host
+        host = mine.cpu()
+        gathered = [torch.empty_like(host) for _ in range(plan.world)]
+        dist.all_gather(gathered, host, group=group)
+        gathered = [g.to(device) for g in gathered]
     else:
         gathered = [torch.empty_like(mine) for _ in range(plan.world)]
         dist.all_gather(gathered, mine, group=group)          # the one exchange step: <= cap * 32 bytes per rank
@@ -73,9 +79,19 @@ def sharded_root(ctx, local_leaves: torch.Tensor, plan: ShardPlan, rank: int, gr
     return ctx.merkle_root(all_nodes.contiguous())
 
 
-def count_mismatches(local_count: int, device, group=None) -> int:
-    """Total number of mismatching chunks over all ranks (an 8-byte all-reduce)."""
-    t = torch.tensor([local_count], dtype=torch.int64, device=device)
+def count_mismatches(local_count, device, group=None):
+    """Total number of mismatching chunks over all ranks (an 8-byte all-reduce).
+
+    `local_count` is an int (the total comes back as an int) or a one-element int64 tensor, e.g. the
+    n_mismatch field of a verification result still on the device; then the total comes back as a
+    tensor on `device` and nothing waits for the GPU."""
+    as_tensor = isinstance(local_count, torch.Tensor)
+    t = local_count.clone().reshape(1) if as_tensor else torch.tensor([local_count], dtype=torch.int64, device=device)
     if dist.is_initialized() and dist.get_world_size(group) > 1:
-        dist.all_reduce(t, group=group)
-    return int(t.item())
+        if t.is_cuda and dist.get_backend(group) == "gloo":
+            host = t.cpu()
+            dist.all_reduce(host, group=group)
+            t = host.to(t.device)
+        else:
+            dist.all_reduce(t, group=group)
+    return t if as_tensor else int(t.item())
