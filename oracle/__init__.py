@@ -76,6 +76,15 @@ def _load():
         lib.ivo_hash_chunks_sha384.restype = ctypes.c_uint64
         lib.ivo_merkle_root_sha384.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u8p]
         lib.ivo_merkle_root_sha384.restype = None
+        lib.ivo_h0_sha512.argtypes = [u64p_]
+        lib.ivo_h0_sha512.restype = None
+        lib.ivo_sha512.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u8p]
+        lib.ivo_sha512.restype = None
+        lib.ivo_hash_chunks_sha512.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64,
+                                               ctypes.c_void_p, ctypes.c_int]
+        lib.ivo_hash_chunks_sha512.restype = ctypes.c_uint64
+        lib.ivo_merkle_root_sha512.argtypes = [ctypes.c_void_p, ctypes.c_uint64, u8p]
+        lib.ivo_merkle_root_sha512.restype = None
         lib.ivo_hash_chunks_rfc6962.argtypes = [ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64,
                                                 ctypes.c_void_p, ctypes.c_int]
         lib.ivo_hash_chunks_rfc6962.restype = ctypes.c_uint64
@@ -215,6 +224,43 @@ def merkle_root_sha384(leaves) -> bytes:
     assert arr.size % 48 == 0
     out = (ctypes.c_uint8 * 48)()
     _load().ivo_merkle_root_sha384(_ptr(arr), arr.size // 48, out)
+    return bytes(out)
+
+
+# ---------------------------------------------------------------------------------------------
+# SHA-512 variant
+
+def h0_sha512() -> np.ndarray:
+    """The SHA-512 initial value (FIPS 180-4 section 5.3.5) as derived from the first eight primes."""
+    h0 = np.zeros(8, dtype=np.uint64)
+    _load().ivo_h0_sha512(h0.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64)))
+    return h0
+
+
+def sha512(msg) -> bytes:
+    arr = _as_u8(msg)
+    out = (ctypes.c_uint8 * 64)()
+    _load().ivo_sha512(_ptr(arr), arr.size, out)
+    return bytes(out)
+
+
+def hash_chunks_sha512(data, chunk_bytes: int, nthreads: int = 1) -> np.ndarray:
+    """SHA-512 chunk digests as an (n, 64) uint8 array."""
+    arr = _as_u8(data)
+    if chunk_bytes <= 0:
+        raise ValueError("chunk_bytes must be positive")
+    n = n_chunks(arr.size, chunk_bytes)
+    out = np.zeros((n, 64), dtype=np.uint8)
+    got = _load().ivo_hash_chunks_sha512(_ptr(arr), arr.size, chunk_bytes, _ptr(out), nthreads)
+    assert got == n
+    return out
+
+
+def merkle_root_sha512(leaves) -> bytes:
+    arr = _as_u8(leaves)
+    assert arr.size % 64 == 0
+    out = (ctypes.c_uint8 * 64)()
+    _load().ivo_merkle_root_sha512(_ptr(arr), arr.size // 64, out)
     return bytes(out)
 
 

@@ -316,6 +316,7 @@ void ivo_hash_ragged(const uint8_t *base, const uint64_t *offsets, const uint64_
 
 static uint64_t g_k512[80];
 static uint64_t g_h0_384[8];
+static uint64_t g_h0_512[8];
 static pthread_once_t g_once512 = PTHREAD_ONCE_INIT;
 
 /* 256-bit unsigned integers as four 64-bit limbs, least significant first: just
@@ -391,6 +392,8 @@ static void derive_constants512(void)
         g_k512[found] = (uint64_t)scaled_root(p, 3);            /* first 64 fraction bits of the cube root */
         if (found >= 8 && found < 16)                           /* SHA-384: the 9th to 16th primes */
             g_h0_384[found - 8] = (uint64_t)scaled_root(p, 2);  /* first 64 fraction bits of the square root */
+        if (found < 8)                                          /* SHA-512 (section 5.3.5): the first eight primes */
+            g_h0_512[found] = (uint64_t)scaled_root(p, 2);
         ++found;
     }
 }
@@ -507,6 +510,94 @@ void ivo_merkle_root_sha384(const uint8_t *leaves, uint64_t n, uint8_t root_out[
         n = parents;
     }
     memcpy(root_out, level, 48);
+    free(level);
+}
+
+/* ------------------------------------------------------------------------- */
+/* SHA-512 (FIPS 180-4 sections 5.1.2, 5.3.5, 6.4): the same compression      */
+/* function, the initial value from the first eight primes, all 512 bits out. */
+/* ------------------------------------------------------------------------- */
+
+void ivo_h0_sha512(uint64_t h0_out[8])
+{
+    pthread_once(&g_once512, derive_constants512);
+    memcpy(h0_out, g_h0_512, sizeof g_h0_512);
+}
+
+void ivo_sha512(const uint8_t *msg, uint64_t len, uint8_t out[64])
+{
+    pthread_once(&g_once512, derive_constants512);
+    uint64_t hash[8];
+    memcpy(hash, g_h0_512, sizeof hash);
+
+    uint64_t full = len / 128;
+    for (uint64_t i = 0; i < full; ++i)
+        process_block512(hash, msg + 128 * i);
+
+    /* section 5.1.2: 0x80, zeros up to 112 mod 128, then the bit length as a 128-bit big-endian integer */
+    uint8_t tail[256];
+    uint64_t rem = len - 128 * full;
+    memset(tail, 0, sizeof tail);
+    if (rem) memcpy(tail, msg + 128 * full, rem);
+    tail[rem] = 0x80;
+    uint64_t tail_len = (rem + 1 + 16 <= 128) ? 128 : 256;
+    u128 bits = (u128)len * 8u;
+    for (int i = 0; i < 16; ++i)
+        tail[tail_len - 1 - i] = (uint8_t)(bits >> (8 * i));
+    for (uint64_t off = 0; off < tail_len; off += 128)
+        process_block512(hash, tail + off);
+
+    for (int i = 0; i < 8; ++i)
+        for (int b = 0; b < 8; ++b)
+            out[8 * i + b] = (uint8_t)(hash[i] >> (56 - 8 * b));
+}
+
+typedef struct {
+    const uint8_t *data;
+    uint64_t nbytes, chunk_bytes;
+    uint8_t *out;
+} chunk512_job;
+
+static void chunk512_task(void *arg, uint64_t i)
+{
+    chunk512_job *job = (chunk512_job *)arg;
+    uint64_t begin = i * job->chunk_bytes;
+    uint64_t end = begin + job->chunk_bytes;
+    if (end > job->nbytes || end < begin) end = job->nbytes;
+    ivo_sha512(job->data + begin, end - begin, job->out + 64 * i);
+}
+
+uint64_t ivo_hash_chunks_sha512(const uint8_t *data, uint64_t nbytes, uint64_t chunk_bytes,
+                                uint8_t *digests_out, int nthreads)
+{
+    if (chunk_bytes == 0 || nbytes == 0) return 0;
+    uint64_t n = nbytes / chunk_bytes + (nbytes % chunk_bytes ? 1 : 0);
+    chunk512_job job = { data, nbytes, chunk_bytes, digests_out };
+    run_tasks(chunk512_task, &job, n, nthreads);
+    return n;
+}
+
+/* The tree rule of the default path with SHA-512 as the node hash: parent = SHA-512(left || right) over
+ * exactly 128 bytes, an unpaired last node moves up unchanged, one leaf is the root, no leaf gives SHA-512(""). */
+void ivo_merkle_root_sha512(const uint8_t *leaves, uint64_t n, uint8_t root_out[64])
+{
+    if (n == 0) { ivo_sha512((const uint8_t *)"", 0, root_out); return; }
+    uint8_t *level = (uint8_t *)malloc((size_t)n * 64);
+    memcpy(level, leaves, (size_t)n * 64);
+    while (n > 1) {
+        uint64_t parents = n / 2;
+        for (uint64_t j = 0; j < parents; ++j) {
+            uint8_t node[64];
+            ivo_sha512(level + 128 * j, 128, node);
+            memcpy(level + 64 * j, node, 64);
+        }
+        if (n % 2) {
+            memmove(level + 64 * parents, level + 64 * (n - 1), 64);
+            ++parents;
+        }
+        n = parents;
+    }
+    memcpy(root_out, level, 64);
     free(level);
 }
 

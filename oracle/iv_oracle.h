@@ -80,6 +80,17 @@ uint64_t ivo_hash_chunks_sha384(const uint8_t *data, uint64_t nbytes, uint64_t c
 void ivo_merkle_root_sha384(const uint8_t *leaves, uint64_t n, uint8_t root_out[48]);
 
 /* ---------------------------------------------------------------------------
+ * SHA-512 variant: FIPS 180-4 section 6.4 with the initial value of section
+ * 5.3.5, no truncation; digests are 64 bytes.  Tree rule as above with
+ * parent = SHA-512(left || right) over exactly 128 bytes.
+ * ------------------------------------------------------------------------- */
+void ivo_h0_sha512(uint64_t h0_out[8]);
+void ivo_sha512(const uint8_t *msg, uint64_t len, uint8_t out[64]);
+uint64_t ivo_hash_chunks_sha512(const uint8_t *data, uint64_t nbytes, uint64_t chunk_bytes,
+                                uint8_t *digests_out, int nthreads);
+void ivo_merkle_root_sha512(const uint8_t *leaves, uint64_t n, uint8_t root_out[64]);
+
+/* ---------------------------------------------------------------------------
  * RFC 6962 section 2.1 mode (the paper cites RFC 6962 for its tree): the Merkle
  * Tree Hash with domain separation over SHA-256, the entries being the chunks.
  * leaf = SHA-256(0x00 || chunk), node = SHA-256(0x01 || left || right), split
