@@ -323,12 +323,18 @@ int iv_hash_ragged_update(iv_ctx *ctx, const void *d_base, const uint64_t *d_off
                           int finish, uint8_t *d_digests, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
- * SHA-384 variant -- the digest of the paper's own kernel listings (FIPS 180-4
- * section 6.5).  Chunking and tree rule as above with 48-byte records: digest i
+ * SHA-384 and SHA-512 variants -- SHA-384 is the digest of the paper's own kernel
+ * listings (FIPS 180-4 section 6.5).  Chunking and tree rule as above with 48-byte records: digest i
  * = SHA-384(chunk i); parent = SHA-384(left || right) over exactly 96 bytes, an
  * unpaired last node moves up unchanged, one leaf is its own root, zero leaves
- * give SHA-384 of the empty string.  A plain implementation (one chain per lane,
- * direct loads): it is not tuned like the SHA-256 path.
+ * give SHA-384 of the empty string.  The SHA-512 entry points (FIPS 180-4 section
+ * 6.4, initial value of section 5.3.5, no truncation) are the same with 64-byte
+ * records and SHA-512(left || right) over exactly 128 bytes as the parent.
+ * 16-byte aligned blobs with up to about 131,000 chunks of 16 KiB or more (a
+ * multiple of 16 bytes) run through a kernel in the design of the SHA-256 path
+ * (tiled bulk copies, the compression split between two warps, chains migrating
+ * between workers); other shapes through a plain one-chain-per-lane kernel,
+ * which is the faster one when chains are plentiful.
  */
 int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint8_t *d_digests, uint64_t digests_cap, uint64_t *h_n_chunks,
@@ -336,7 +342,13 @@ int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint
 int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
                           void *cuda_stream);
 
-/* iv_verify_manifest for this variant: the same steps over 48-byte records.  The manifest holds the
+int iv_hash_chunks_sha512(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes,
+                          uint8_t *d_digests, uint64_t digests_cap, uint64_t *h_n_chunks,
+                          void *cuda_stream);
+int iv_merkle_root_sha512(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root,
+                          void *cuda_stream);
+
+/* iv_verify_manifest for the SHA-384 variant: the same steps over 48-byte records.  The manifest holds the
  * SHA-384 chunk digests (device) and the root of the SHA-384 tree; fields, index list, errors and
  * asynchrony as for iv_manifest / iv_verify_result / iv_verify_manifest. */
 typedef struct iv_manifest_sha384 {

@@ -32,6 +32,7 @@ EXPORTS = (
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
     "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update", "iv_verify_manifest_batch",
     "iv_hash_chunks_sha384", "iv_merkle_root_sha384", "iv_verify_manifest_sha384",
+    "iv_hash_chunks_sha512", "iv_merkle_root_sha512",
     "iv_hash_chunks_rfc6962", "iv_merkle_root_rfc6962", "iv_verify_manifest_rfc6962",
 )
 
@@ -118,6 +119,10 @@ def load_library() -> ctypes.CDLL:
     lib.iv_hash_chunks_sha384.restype = i32
     lib.iv_merkle_root_sha384.argtypes = [vp, vp, u64, vp, vp]
     lib.iv_merkle_root_sha384.restype = i32
+    lib.iv_hash_chunks_sha512.argtypes = [vp, vp, u64, u64, vp, u64, ctypes.POINTER(u64), vp]
+    lib.iv_hash_chunks_sha512.restype = i32
+    lib.iv_merkle_root_sha512.argtypes = [vp, vp, u64, vp, vp]
+    lib.iv_merkle_root_sha512.restype = i32
     lib.iv_verify_manifest_rfc6962.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest_rfc6962.restype = i32
     lib.iv_verify_manifest_sha384.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest384), vp, vp, u64, vp]
@@ -289,6 +294,28 @@ class Context:
             out = torch.empty(48, dtype=torch.uint8, device=leaves.device)
         rc = self._lib.iv_merkle_root_sha384(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
         self._check(rc, "iv_merkle_root_sha384")
+        return out
+
+    def hash_chunks_sha512(self, data: torch.Tensor, chunk_bytes: int, stream=None,
+                           out: torch.Tensor | None = None) -> torch.Tensor:
+        """iv_hash_chunks_sha512: (n, 64) uint8 SHA-512 digests of the chunks of `data`."""
+        nb = _nbytes(data)
+        n = n_chunks(nb, chunk_bytes) if chunk_bytes > 0 else 0
+        if out is None:
+            out = torch.empty((n, 64), dtype=torch.uint8, device=data.device)
+        got = ctypes.c_uint64(0)
+        rc = self._lib.iv_hash_chunks_sha512(self._h, _dev_ptr(data), nb, chunk_bytes, _dev_ptr(out), n,
+                                             ctypes.byref(got), _stream_ptr(stream))
+        self._check(rc, "iv_hash_chunks_sha512")
+        return out[:got.value]
+
+    def merkle_root_sha512(self, leaves: torch.Tensor, stream=None, out: torch.Tensor | None = None) -> torch.Tensor:
+        """iv_merkle_root_sha512: 64-byte root of (n, 64) leaf digests."""
+        n = leaves.numel() // 64
+        if out is None:
+            out = torch.empty(64, dtype=torch.uint8, device=leaves.device)
+        rc = self._lib.iv_merkle_root_sha512(self._h, _dev_ptr(leaves), n, _dev_ptr(out), _stream_ptr(stream))
+        self._check(rc, "iv_merkle_root_sha512")
         return out
 
     def verify_manifest_sha384(self, data: torch.Tensor, total_bytes: int, chunk_bytes: int, digests: torch.Tensor,

@@ -104,7 +104,8 @@ bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint6
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
                                const uint32_t *d_one, void *d_slice_scratch, cudaStream_t stream,
-                               uint64_t *launches, const char **kernel_used) {
+                               uint64_t *launches, const char **kernel_used, cudaStream_t tail_stream) {
+    if (!tail_stream) tail_stream = stream;
     const char *unused = nullptr;
     if (!kernel_used) kernel_used = &unused;
     if (n_chunks == 0) return cudaSuccess;
@@ -132,12 +133,13 @@ cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t 
                                                       d_slice_scratch, d_one, sm_count, stream, &covered);
             if (e != cudaSuccess || covered == n_chunks) return e;
             // what the tiled copies left out (a short last chunk; everything if the blob could not be described to
-            // the TMA unit): one chain per lane through the direct kernel
+            // the TMA unit): one chain per lane through the direct kernel, on tail_stream (beside the main kernel
+            // when the caller forked that stream off, after it otherwise)
             if (launches) ++*launches;
             const uint64_t off = covered * chunk_bytes, rest = n_chunks - covered;
             const uint64_t rest_blocks = (rest + 127) / 128;
             if (rest_blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
-            hash_chunks_kernel<true><<<(unsigned)rest_blocks, 128, 0, stream>>>(d_data + off, nbytes - off, chunk_bytes, rest,
+            hash_chunks_kernel<true><<<(unsigned)rest_blocks, 128, 0, tail_stream>>>(d_data + off, nbytes - off, chunk_bytes, rest,
                                                                               d_digests + 32 * covered);
             return cudaGetLastError();
         }

@@ -33,37 +33,10 @@
 #include "sha256_dev.cuh"
 #include "slice_queue_dev.cuh"
 #include "tma_dev.cuh"
+#include "chunk_tensor_map.h"
 
 namespace ivk {
 namespace {
-
-// A scheduler's second worker takes a task only when one lies in the FIFO unclaimed: the first
-// workers (one per scheduler) are served first, so no scheduler idles while another runs two
-// groups.  With nothing left over it polls; giving up (the return value total_tasks ends the
-// worker) is harmless, the first workers finish the launch.  Kept out of line so that the hashing
-// loop's register allocation does not depend on it.
-__device__ __noinline__ unsigned long long take_leftover_ticket(SliceQueue *q, unsigned long long total_tasks,
-                                                                bool first_take) {
-    if (first_take) __nanosleep(20000);      // at launch, let the first workers of every CTA claim their groups
-    const long long t0 = clock64();
-    for (;;) {
-        const unsigned long long h = *reinterpret_cast<volatile unsigned long long *>(&q->head);
-        if (h >= total_tasks) return total_tasks;
-        const unsigned long long tl = *reinterpret_cast<volatile unsigned long long *>(&q->tail);
-        if (tl > h) {
-            if (atomicCAS(&q->head, h, h + 1ull) == h) return h;
-            continue;
-        }
-        if (clock64() - t0 > 8000000000ll) return total_tasks;
-        __nanosleep(256);
-    }
-}
-
-__device__ __forceinline__ void tiled_g2s(uint32_t dst, const CUtensorMap *map, uint32_t x, uint32_t y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
 
 // FWF ("first workers first"): warps 4..7 take only left-over tasks, see the service order above.
 // PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash).  Message block j is then the
@@ -176,8 +149,8 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
                 const uint32_t boxes = (warp_bytes - off > 128) ? 2u : 1u;
                 tma::mbar_arrive_expect_tx(bar, boxes * 4096u);
                 const uint32_t x = (uint32_t)(lo + off), y = (uint32_t)(g * 32);
-                tiled_g2s(ring_warp + stg * kStageBytes, &tmap, x, y, bar);
-                if (boxes == 2) tiled_g2s(ring_warp + stg * kStageBytes + 4096u, &tmap, x + 128u, y, bar);
+                tma::tiled_g2s(ring_warp + stg * kStageBytes, &tmap, x, y, bar);
+                if (boxes == 2) tma::tiled_g2s(ring_warp + stg * kStageBytes + 4096u, &tmap, x + 128u, y, bar);
             }
         };
         auto fetch = [&](int stg, int blk_in_stage) {
@@ -331,6 +304,8 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+}  // namespace
+
 // The blob's whole chunks as a 2-D byte tensor [rows][chunk_bytes], box = 32 rows x 128 bytes, 128-byte swizzle.
 bool make_chunk_tensor_map(CUtensorMap *map, const uint8_t *d_data, uint64_t chunk_bytes, uint64_t rows) {
     EncodeTiledFn fn = encode_tiled_fn();
@@ -343,6 +318,8 @@ bool make_chunk_tensor_map(CUtensorMap *map, const uint8_t *d_data, uint64_t chu
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+namespace {
 
 thread_local const char *t_instance = "";
 

@@ -132,8 +132,9 @@ cudaError_t launch_direct(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk
 cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
                                        uint8_t *d_digests, int sm_count, uint32_t *d_status, const uint32_t *d_one,
                                        void *d_slice_scratch, cudaStream_t stream, uint64_t *launches,
-                                       const char **kernel_used) {
+                                       const char **kernel_used, cudaStream_t tail_stream) {
     if (n_chunks == 0) return cudaSuccess;
+    if (!tail_stream) tail_stream = stream;
     const bool aligned = ((reinterpret_cast<uintptr_t>(d_data) & 15u) == 0) && (chunk_bytes % 16u == 0);
     if (aligned && chunk_bytes >= 4096 && (n_chunks + 31) / 32 <= 2ull * (uint64_t)sm_count) {
         // few chains: the two-warp kernel, prefixed
@@ -157,7 +158,7 @@ cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, u
         if (launches) ++*launches;
         const uint64_t off = covered * chunk_bytes;
         return launch_direct(d_data + off, nbytes - off, chunk_bytes, n_chunks - covered, d_digests + 32 * covered,
-                             sm_count, stream);
+                             sm_count, tail_stream);
     }
     if (launches) ++*launches;
     if (kernel_used) *kernel_used = "hash_chunks_rfc6962_kernel";

@@ -31,7 +31,9 @@ struct iv_ctx {
     uint32_t *d_words = nullptr;
     uint64_t words_cap = 0;
     uint8_t *d_tree384[2] = {nullptr, nullptr};   // level ping-pong of the SHA-384 and RFC 6962 trees
-    uint64_t tree384_cap = 0;                 // in records of 48 bytes, each buffer
+    uint64_t tree384_cap = 0;                 // in records of 64 bytes, each buffer
+    uint8_t *d_pairs512 = nullptr;            // FIFO, slice counters and parked chaining values of the SHA-384/512 two-warp kernel
+    uint64_t pairs512_cap = 0;                // bytes
     uint8_t *d_batch = nullptr;               // offsets, lengths, roots, run roots, tickets of iv_verify_manifest_batch
     uint64_t batch_cap = 0;                   // bytes
     uint64_t batch_blobs = 0, batch_total = 0;   // shape of the last batch (the tickets' position depends on it)
@@ -52,6 +54,8 @@ struct iv_ctx {
     uint8_t *d_window[2] = {nullptr, nullptr};
     uint64_t window_cap = 0;
     cudaStream_t copy_stream = nullptr;
+    cudaStream_t tail_stream = nullptr;       // a blob's short last chunk is hashed here, beside the main leaf kernel
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaEvent_t ev_entry = nullptr, ev_copied[2] = {nullptr, nullptr}, ev_hashed[2] = {nullptr, nullptr};
 
     // phase timing: four events (start, hashed, reduced, compared) per recent call
@@ -119,15 +123,29 @@ int ensure_merkle_scratch(iv_ctx *ctx, uint64_t n_leaves) {
     return IV_OK;
 }
 
-// Level buffers of the variant trees: two buffers of at least `records` records of 48 bytes.
+// Level buffers of the variant trees: two buffers of at least `records` records of up to 64 bytes.
 int ensure_variant_tree_scratch(iv_ctx *ctx, uint64_t records) {
     if (records <= ctx->tree384_cap) return IV_OK;
     uint64_t cap_a = ctx->tree384_cap, cap_b = ctx->tree384_cap;
-    int rc = grow(ctx, &ctx->d_tree384[0], &cap_a, records, 48);
+    int rc = grow(ctx, &ctx->d_tree384[0], &cap_a, records, 64);
     if (rc != IV_OK) return rc;
-    rc = grow(ctx, &ctx->d_tree384[1], &cap_b, records, 48);
+    rc = grow(ctx, &ctx->d_tree384[1], &cap_b, records, 64);
     if (rc != IV_OK) return rc;
     ctx->tree384_cap = cap_a < cap_b ? cap_a : cap_b;
+    return IV_OK;
+}
+
+// The kernels with tiled copies hash a blob's whole chunks; a short last chunk is left to a direct kernel as one
+// serial chain, which for a large chunk can take as long as the whole main launch.  It therefore runs on the
+// context's second stream, forked off the caller's stream before the launches and joined after them.
+int fork_tail_stream(iv_ctx *ctx, cudaStream_t stream) {
+    IV_TRY(ctx, cudaEventRecord(ctx->ev_fork, stream));
+    IV_TRY(ctx, cudaStreamWaitEvent(ctx->tail_stream, ctx->ev_fork, 0));
+    return IV_OK;
+}
+int join_tail_stream(iv_ctx *ctx, cudaStream_t stream) {
+    IV_TRY(ctx, cudaEventRecord(ctx->ev_join, ctx->tail_stream));
+    IV_TRY(ctx, cudaStreamWaitEvent(stream, ctx->ev_join, 0));
     return IV_OK;
 }
 
@@ -146,8 +164,13 @@ int hash_leaves(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t ch
         if (rc != IV_OK) return rc;
         scratch = ctx->d_slices;
     }
+    const bool fork = scratch && nbytes % chunk_bytes != 0;
+    int rc = IV_OK;
+    if (fork && (rc = fork_tail_stream(ctx, stream)) != IV_OK) return rc;
     IV_TRY(ctx, ivk::launch_hash_chunks(d_data, nbytes, chunk_bytes, n, d_digests, ctx->sm_count, ctx->d_status,
-                                        ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel));
+                                        ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel,
+                                        fork ? ctx->tail_stream : nullptr));
+    if (fork && (rc = join_tail_stream(ctx, stream)) != IV_OK) return rc;
     note_leaf_instance(ctx);
     return IV_OK;
 }
@@ -162,9 +185,34 @@ int hash_leaves_rfc6962(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uin
         if (rc != IV_OK) return rc;
         scratch = ctx->d_slices;
     }
+    const bool fork = scratch && nbytes % chunk_bytes != 0;
+    int rc = IV_OK;
+    if (fork && (rc = fork_tail_stream(ctx, stream)) != IV_OK) return rc;
     IV_TRY(ctx, ivk::launch_hash_chunks_rfc6962(d_data, nbytes, chunk_bytes, n, d_digests, ctx->sm_count, ctx->d_status,
-                                                ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel));
+                                                ctx->d_one, scratch, stream, &ctx->launches, &ctx->leaf_kernel,
+                                                fork ? ctx->tail_stream : nullptr));
+    if (fork && (rc = join_tail_stream(ctx, stream)) != IV_OK) return rc;
     note_leaf_instance(ctx);
+    return IV_OK;
+}
+
+// SHA-384 (digest_words 6) or SHA-512 (8) leaf hashing with the scratch the launch shape needs.
+int hash_leaves_wide(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n,
+                     uint8_t *d_digests, int digest_words, cudaStream_t stream) {
+    void *scratch = nullptr;
+    if (ivk::sha512_wants_pairs(d_data, nbytes, chunk_bytes, ctx->sm_count)) {
+        int rc = grow(ctx, &ctx->d_pairs512, &ctx->pairs512_cap, ivk::sha512_pairs_scratch_bytes(nbytes, chunk_bytes), 1);
+        if (rc != IV_OK) return rc;
+        scratch = ctx->d_pairs512;
+    }
+    const bool fork = scratch && nbytes % chunk_bytes != 0;
+    int rc = IV_OK;
+    if (fork && (rc = fork_tail_stream(ctx, stream)) != IV_OK) return rc;
+    IV_TRY(ctx, ivk::launch_hash_chunks_sha384(d_data, nbytes, chunk_bytes, n, d_digests, digest_words, ctx->sm_count,
+                                               ctx->d_status, scratch, stream, &ctx->launches, &ctx->leaf_kernel,
+                                               fork ? ctx->tail_stream : nullptr));
+    if (fork && (rc = join_tail_stream(ctx, stream)) != IV_OK) return rc;
+    ctx->leaf_instance = "";
     return IV_OK;
 }
 
@@ -290,6 +338,9 @@ int iv_create(iv_ctx **out, int cuda_device) {
     cudaError_t e = cudaMalloc(&ctx->d_small, small_bytes);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_small, 0, small_bytes);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->tail_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming);
     for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
         e = cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming);
@@ -333,6 +384,7 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_dirty_scratch);
     cudaFree(ctx->d_columns);
     cudaFree(ctx->d_digests384);
+    cudaFree(ctx->d_pairs512);
     cudaFree(ctx->d_sub);
     cudaFree(ctx->d_batch);
     cudaFree(ctx->d_tree384[0]);
@@ -340,6 +392,9 @@ int iv_destroy(iv_ctx *ctx) {
     cudaFree(ctx->d_window[0]);
     cudaFree(ctx->d_window[1]);
     if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+    if (ctx->tail_stream) cudaStreamDestroy(ctx->tail_stream);
+    if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+    if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
     for (int i = 0; i < 2; ++i) {
         if (ctx->ev_copied[i]) cudaEventDestroy(ctx->ev_copied[i]);
@@ -770,8 +825,10 @@ int iv_hash_ragged_update(iv_ctx *ctx, const void *d_base, const uint64_t *d_off
     return IV_OK;
 }
 
-int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint8_t *d_digests,
-                          uint64_t digests_cap, uint64_t *h_n_chunks, void *cuda_stream) {
+namespace {
+
+int hash_chunks_wide(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint8_t *d_digests,
+                     uint64_t digests_cap, uint64_t *h_n_chunks, int digest_words, void *cuda_stream) {
     if (!ctx || chunk_bytes == 0) return IV_ERR_INVALID_ARG;
     const uint64_t n = chunk_count(nbytes, chunk_bytes);
     if (n > digests_cap) return IV_ERR_INVALID_ARG;
@@ -779,20 +836,39 @@ int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint
     if (h_n_chunks) *h_n_chunks = n;
     if (n == 0) return IV_OK;
     DeviceGuard guard(ctx->device);
-    IV_TRY(ctx, ivk::launch_hash_chunks_sha384(static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests,
-                                               ctx->sm_count, static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
-    ctx->leaf_kernel = "hash_chunks_sha384_kernel";
-    return IV_OK;
+    return hash_leaves_wide(ctx, static_cast<const uint8_t *>(d_data), nbytes, chunk_bytes, n, d_digests, digest_words,
+                            static_cast<cudaStream_t>(cuda_stream));
 }
 
-int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
+int merkle_root_wide(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, int digest_words,
+                     void *cuda_stream) {
     if (!ctx || !d_root || (n_leaves && !d_leaves)) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     int rc = ensure_variant_tree_scratch(ctx, (n_leaves + 1) / 2 + 1);
     if (rc != IV_OK) return rc;
-    IV_TRY(ctx, ivk::launch_merkle_root_sha384(d_leaves, n_leaves, d_root, ctx->d_tree384[0], ctx->d_tree384[1],
+    IV_TRY(ctx, ivk::launch_merkle_root_sha384(d_leaves, n_leaves, d_root, ctx->d_tree384[0], ctx->d_tree384[1], digest_words,
                                                static_cast<cudaStream_t>(cuda_stream), &ctx->launches));
     return IV_OK;
+}
+
+}  // namespace
+
+int iv_hash_chunks_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint8_t *d_digests,
+                          uint64_t digests_cap, uint64_t *h_n_chunks, void *cuda_stream) {
+    return hash_chunks_wide(ctx, d_data, nbytes, chunk_bytes, d_digests, digests_cap, h_n_chunks, 6, cuda_stream);
+}
+
+int iv_merkle_root_sha384(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
+    return merkle_root_wide(ctx, d_leaves, n_leaves, d_root, 6, cuda_stream);
+}
+
+int iv_hash_chunks_sha512(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint8_t *d_digests,
+                          uint64_t digests_cap, uint64_t *h_n_chunks, void *cuda_stream) {
+    return hash_chunks_wide(ctx, d_data, nbytes, chunk_bytes, d_digests, digests_cap, h_n_chunks, 8, cuda_stream);
+}
+
+int iv_merkle_root_sha512(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leaves, uint8_t *d_root, void *cuda_stream) {
+    return merkle_root_wide(ctx, d_leaves, n_leaves, d_root, 8, cuda_stream);
 }
 
 int iv_verify_manifest_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest_sha384 *m,
@@ -809,10 +885,10 @@ int iv_verify_manifest_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, 
     if ((rc = ensure_variant_tree_scratch(ctx, (n + 1) / 2 + 1)) != IV_OK) return rc;
     if ((rc = grow(ctx, &ctx->d_words, &ctx->words_cap, (n + 31) / 32 + 1, sizeof(uint32_t))) != IV_OK) return rc;
     uint8_t *d_root = ctx->d_digests384 + 48 * (n + 1);
-    IV_TRY(ctx, ivk::launch_hash_chunks_sha384(static_cast<const uint8_t *>(d_data), nbytes, m->chunk_bytes, n,
-                                               ctx->d_digests384, ctx->sm_count, stream, &ctx->launches));
-    ctx->leaf_kernel = "hash_chunks_sha384_kernel";
-    IV_TRY(ctx, ivk::launch_merkle_root_sha384(ctx->d_digests384, n, d_root, ctx->d_tree384[0], ctx->d_tree384[1], stream,
+    if (n && (rc = hash_leaves_wide(ctx, static_cast<const uint8_t *>(d_data), nbytes, m->chunk_bytes, n, ctx->d_digests384, 6,
+                                    stream)) != IV_OK)
+        return rc;
+    IV_TRY(ctx, ivk::launch_merkle_root_sha384(ctx->d_digests384, n, d_root, ctx->d_tree384[0], ctx->d_tree384[1], 6, stream,
                                                &ctx->launches));
     ivk::RootBytes384 expect;
     std::memcpy(expect.b, m->root, 48);

@@ -34,7 +34,10 @@ constexpr uint32_t kMerkleRun = 512;
 cudaError_t launch_hash_chunks(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                uint64_t n_chunks, uint8_t *d_digests, int sm_count, uint32_t *d_status,
                                const uint32_t *d_one, void *d_slice_scratch, cudaStream_t stream,
-                               uint64_t *launches, const char **kernel_used);
+                               uint64_t *launches, const char **kernel_used, cudaStream_t tail_stream = nullptr);
+// tail_stream (here and in the variants' launchers): where the kernel for what the tiled copies leave out -- a blob's
+// short last chunk, one long serial chain -- is launched; NULL = on `stream`, after the main kernel.  A caller that
+// has forked a second stream off `stream` passes it, and the chain runs beside the main kernel.
 // True when launch_hash_chunks would use the sliced kernel (and so needs its scratch).
 bool hash_chunks_wants_slices(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count);
 
@@ -147,11 +150,26 @@ cudaError_t launch_hash_chunks_pairs(const uint8_t *d_data, uint64_t nbytes, uin
                                      int sm_count, cudaStream_t stream, bool zero_prefix = false);
 
 // hash_sha384.cu -----------------------------------------------------------
-// SHA-384 variant: 48-byte chunk digests and the tree with SHA-384 parents.
+// SHA-384 / SHA-512 variants (digest_words = 6 / 8): chunk digests of 48 / 64 bytes and the tree whose parents
+// are the same hash.  With d_pairs_scratch (sha512_pairs_scratch_bytes(...) bytes, may be NULL) shapes that
+// sha512_wants_pairs go through the two-warp kernel of hash_sha512_pairs.cu.
 cudaError_t launch_hash_chunks_sha384(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
-                                      uint8_t *d_digests, int sm_count, cudaStream_t stream, uint64_t *launches);
+                                      uint8_t *d_digests, int digest_words, int sm_count, uint32_t *d_status,
+                                      void *d_pairs_scratch, cudaStream_t stream, uint64_t *launches,
+                                      const char **kernel_used, cudaStream_t tail_stream = nullptr);
 cudaError_t launch_merkle_root_sha384(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root, uint8_t *d_scratch_a,
-                                      uint8_t *d_scratch_b, cudaStream_t stream, uint64_t *launches);
+                                      uint8_t *d_scratch_b, int digest_words, cudaStream_t stream, uint64_t *launches);
+
+// hash_sha512_pairs.cu ------------------------------------------------------
+// 16-byte aligned blobs with at least one whole chunk of 16 KiB or more (a multiple of 16 bytes), at group counts
+// where the two-warp kernel is the faster one.
+bool sha512_wants_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, int sm_count);
+uint64_t sha512_pairs_scratch_bytes(uint64_t nbytes, uint64_t chunk_bytes);
+// Hashes the blob's whole chunks (*covered of them, from the front; 0 and nothing launched if the blob cannot be
+// described to the TMA unit); a short last chunk is left to the caller.
+cudaError_t launch_hash_sha512_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint8_t *d_digests,
+                                     int digest_words, uint32_t *d_status, void *d_scratch, int sm_count,
+                                     cudaStream_t stream, uint64_t *covered, uint64_t *launches);
 
 // hash_rfc6962.cu ----------------------------------------------------------
 // RFC 6962 section 2.1 mode: prefixed leaf hashes and the tree with prefixed nodes.
@@ -160,7 +178,7 @@ cudaError_t launch_merkle_root_sha384(const uint8_t *d_leaves, uint64_t n, uint8
 cudaError_t launch_hash_chunks_rfc6962(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
                                        uint8_t *d_digests, int sm_count, uint32_t *d_status, const uint32_t *d_one,
                                        void *d_slice_scratch, cudaStream_t stream, uint64_t *launches,
-                                       const char **kernel_used);
+                                       const char **kernel_used, cudaStream_t tail_stream = nullptr);
 cudaError_t launch_merkle_root_rfc6962(const uint8_t *d_leaves, uint64_t n, uint8_t *d_root, uint8_t *d_scratch_a,
                                        uint8_t *d_scratch_b, cudaStream_t stream, uint64_t *launches);
 

@@ -1,6 +1,7 @@
-// SHA-384 (FIPS 180-4 sections 4.1.3, 4.2.3, 5.3.4, 6.4.2, 6.5) for one compression chain per thread:
-// SHA-512's compression function on 64-bit words with SHA-384's initial value, digest = the first
-// six words.  64-bit rotates compile to pairs of funnel shifts, the boolean functions to pairs of LOP3.
+// SHA-384 and SHA-512 (FIPS 180-4 sections 4.1.3, 4.2.3, 5.3.4, 5.3.5, 6.4.2, 6.5) for one compression chain
+// per thread: one compression function on 64-bit words; SHA-384 starts from its own initial value and keeps
+// the first six words, SHA-512 keeps all eight.  64-bit rotates compile to pairs of funnel shifts, the boolean
+// functions to pairs of LOP3.
 #pragma once
 #include <cstdint>
 
@@ -30,19 +31,75 @@ static __constant__ uint64_t kSha512K[80] = {
     0x4cc5d4becb3e42b6ull, 0x597f299cfc657e2aull, 0x5fcb6fab3ad6faecull, 0x6c44198c4a475817ull,
 };
 
-__device__ __forceinline__ uint64_t rotr64(uint64_t x, int n) { return (x >> n) | (x << (64 - n)); }
-__device__ __forceinline__ uint64_t ch64(uint64_t x, uint64_t y, uint64_t z) { return (x & y) ^ (~x & z); }
-__device__ __forceinline__ uint64_t maj64(uint64_t x, uint64_t y, uint64_t z) { return (x & y) | (z & (x | y)); }
-__device__ __forceinline__ uint64_t big_s0_512(uint64_t x) { return rotr64(x, 28) ^ rotr64(x, 34) ^ rotr64(x, 39); }
-__device__ __forceinline__ uint64_t big_s1_512(uint64_t x) { return rotr64(x, 14) ^ rotr64(x, 18) ^ rotr64(x, 41); }
-__device__ __forceinline__ uint64_t small_s0_512(uint64_t x) { return rotr64(x, 1) ^ rotr64(x, 8) ^ (x >> 7); }
-__device__ __forceinline__ uint64_t small_s1_512(uint64_t x) { return rotr64(x, 19) ^ rotr64(x, 61) ^ (x >> 6); }
+// 64-bit words are handled as pairs of 32-bit registers, written out so that every rotation is two funnel
+// shifts and every three-input boolean function one LOP3 per half (left to itself the compiler splits the
+// 64-bit expressions but does not merge the two XORs of a Sigma into one three-input operation).
+__device__ __forceinline__ uint32_t lo32(uint64_t x) { return (uint32_t)x; }
+__device__ __forceinline__ uint32_t hi32(uint64_t x) { return (uint32_t)(x >> 32); }
+__device__ __forceinline__ uint64_t pack64(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+template <int LUT>
+__device__ __forceinline__ uint32_t lop3_512(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, %4;" : "=r"(r) : "r"(a), "r"(b), "r"(c), "n"(LUT));
+    return r;
+}
+// low and high half of rotr(x, N) and of x >> N
+template <int N>
+__device__ __forceinline__ uint32_t rotr64_lo(uint32_t lo, uint32_t hi) {
+    return N < 32 ? __funnelshift_r(lo, hi, N) : __funnelshift_r(hi, lo, N - 32);
+}
+template <int N>
+__device__ __forceinline__ uint32_t rotr64_hi(uint32_t lo, uint32_t hi) {
+    return N < 32 ? __funnelshift_r(hi, lo, N) : __funnelshift_r(lo, hi, N - 32);
+}
+// xor of three rotations (FIPS 180-4 equations 4.10, 4.11)
+template <int A, int B, int C>
+__device__ __forceinline__ uint64_t sigma_rrr(uint64_t x) {
+    const uint32_t l = lo32(x), h = hi32(x);
+    return pack64(lop3_512<0x96>(rotr64_lo<A>(l, h), rotr64_lo<B>(l, h), rotr64_lo<C>(l, h)),
+                  lop3_512<0x96>(rotr64_hi<A>(l, h), rotr64_hi<B>(l, h), rotr64_hi<C>(l, h)));
+}
+// xor of two rotations and a right shift by S < 32 (equations 4.12, 4.13)
+template <int A, int B, int S>
+__device__ __forceinline__ uint64_t sigma_rrs(uint64_t x) {
+    const uint32_t l = lo32(x), h = hi32(x);
+    return pack64(lop3_512<0x96>(rotr64_lo<A>(l, h), rotr64_lo<B>(l, h), __funnelshift_r(l, h, S)),
+                  lop3_512<0x96>(rotr64_hi<A>(l, h), rotr64_hi<B>(l, h), h >> S));
+}
+// FIPS 180-4 section 4.1.3, equations 4.8 - 4.13.
+__device__ __forceinline__ uint64_t ch64(uint64_t x, uint64_t y, uint64_t z) {
+    return pack64(lop3_512<0xCA>(lo32(x), lo32(y), lo32(z)), lop3_512<0xCA>(hi32(x), hi32(y), hi32(z)));
+}
+__device__ __forceinline__ uint64_t maj64(uint64_t x, uint64_t y, uint64_t z) {
+    return pack64(lop3_512<0xE8>(lo32(x), lo32(y), lo32(z)), lop3_512<0xE8>(hi32(x), hi32(y), hi32(z)));
+}
+__device__ __forceinline__ uint64_t big_s0_512(uint64_t x) { return sigma_rrr<28, 34, 39>(x); }
+__device__ __forceinline__ uint64_t big_s1_512(uint64_t x) { return sigma_rrr<14, 18, 41>(x); }
+__device__ __forceinline__ uint64_t small_s0_512(uint64_t x) { return sigma_rrs<1, 8, 7>(x); }
+__device__ __forceinline__ uint64_t small_s1_512(uint64_t x) { return sigma_rrs<19, 61, 6>(x); }
 
 // Initial hash value of SHA-384, FIPS 180-4 section 5.3.4.
 __device__ __forceinline__ void sha384_init(uint64_t (&st)[8]) {
     st[0] = 0xcbbb9d5dc1059ed8ull; st[1] = 0x629a292a367cd507ull; st[2] = 0x9159015a3070dd17ull;
     st[3] = 0x152fecd8f70e5939ull; st[4] = 0x67332667ffc00b31ull; st[5] = 0x8eb44a8768581511ull;
     st[6] = 0xdb0c2e0d64f98fa7ull; st[7] = 0x47b5481dbefa4fa4ull;
+}
+
+// Initial hash value of SHA-512, FIPS 180-4 section 5.3.5.
+__device__ __forceinline__ void sha512_init(uint64_t (&st)[8]) {
+    st[0] = 0x6a09e667f3bcc908ull; st[1] = 0xbb67ae8584caa73bull; st[2] = 0x3c6ef372fe94f82bull;
+    st[3] = 0xa54ff53a5f1d36f1ull; st[4] = 0x510e527fade682d1ull; st[5] = 0x9b05688c2b3e6c1full;
+    st[6] = 0x1f83d9abfb41bd6bull; st[7] = 0x5be0cd19137e2179ull;
+}
+template <int DIGEST_WORDS>
+__device__ __forceinline__ void sha512_family_init(uint64_t (&st)[8]) {
+    static_assert(DIGEST_WORDS == 6 || DIGEST_WORDS == 8, "SHA-384 keeps six words, SHA-512 eight");
+    if (DIGEST_WORDS == 6) sha384_init(st);
+    else sha512_init(st);
 }
 
 // st <- compress(st, block); w[0..15] holds the 128-byte block as big-endian 64-bit words and is
@@ -70,25 +127,25 @@ __device__ __forceinline__ void sha512_compress(uint64_t (&st)[8], uint64_t (&w)
 
 // big-endian 64-bit word from eight bytes in memory order held as two little-endian 32-bit words
 __device__ __forceinline__ uint64_t be64(uint32_t lo_addr_word, uint32_t hi_addr_word) {
-    return ((uint64_t)__byte_perm(lo_addr_word, 0, 0x0123) << 32) | (uint64_t)__byte_perm(hi_addr_word, 0, 0x0123);
+    return pack64(__byte_perm(hi_addr_word, 0, 0x0123), __byte_perm(lo_addr_word, 0, 0x0123));
 }
 
-// 48-byte digest record (six big-endian words) at a 16-byte aligned address.
-__device__ __forceinline__ void store_digest384(uint8_t *dst, const uint64_t (&st)[8]) {
-    uint32_t o[12];
+// Digest record: the first WORDS words, big-endian (48 bytes for SHA-384, 64 for SHA-512), at any alignment.
+template <int WORDS>
+__device__ __forceinline__ void store_digest512(uint8_t *dst, const uint64_t (&st)[8]) {
+    uint32_t o[2 * WORDS];
 #pragma unroll
-    for (int i = 0; i < 6; ++i) {
+    for (int i = 0; i < WORDS; ++i) {
         o[2 * i] = __byte_perm((uint32_t)(st[i] >> 32), 0, 0x0123);
         o[2 * i + 1] = __byte_perm((uint32_t)st[i], 0, 0x0123);
     }
     if ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
         uint4 *q = reinterpret_cast<uint4 *>(dst);
-        q[0] = make_uint4(o[0], o[1], o[2], o[3]);
-        q[1] = make_uint4(o[4], o[5], o[6], o[7]);
-        q[2] = make_uint4(o[8], o[9], o[10], o[11]);
+#pragma unroll
+        for (int i = 0; i < WORDS / 2; ++i) q[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
     } else {
 #pragma unroll
-        for (int i = 0; i < 12; ++i)
+        for (int i = 0; i < 2 * WORDS; ++i)
             for (int b = 0; b < 4; ++b) dst[4 * i + b] = (uint8_t)(o[i] >> (8 * b));
     }
 }

@@ -32,5 +32,27 @@ __device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
+// A scheduler's second worker takes a task only when one lies in the FIFO unclaimed: the first
+// workers (one per scheduler) are served first, so no scheduler idles while another runs two
+// groups.  With nothing left over it polls; giving up (the return value total_tasks ends the
+// worker) is harmless, the first workers finish the launch.  Kept out of line so that the hashing
+// loop's register allocation does not depend on it.
+__device__ __noinline__ unsigned long long take_leftover_ticket(SliceQueue *q, unsigned long long total_tasks,
+                                                                bool first_take) {
+    if (first_take) __nanosleep(20000);      // at launch, let the first workers of every CTA claim their groups
+    const long long t0 = clock64();
+    for (;;) {
+        const unsigned long long h = *reinterpret_cast<volatile unsigned long long *>(&q->head);
+        if (h >= total_tasks) return total_tasks;
+        const unsigned long long tl = *reinterpret_cast<volatile unsigned long long *>(&q->tail);
+        if (tl > h) {
+            if (atomicCAS(&q->head, h, h + 1ull) == h) return h;
+            continue;
+        }
+        if (clock64() - t0 > 8000000000ll) return total_tasks;
+        __nanosleep(256);
+    }
+}
+
 }  // namespace
 }  // namespace ivk

@@ -1,6 +1,6 @@
-"""GPU parity of the SHA-384 variant (FIPS 180-4 section 6.5; the digest of the paper's kernel
-listings): chunk digests and tree roots from the CUDA library equal the CPU oracle's bit for bit.
-All calls go through the C ABI via the ctypes binding."""
+"""GPU parity of the SHA-384 and SHA-512 variants (FIPS 180-4 sections 6.4 and 6.5; SHA-384 is the digest of
+the paper's kernel listings): chunk digests and tree roots from the CUDA library equal the CPU oracle's bit
+for bit.  All calls go through the C ABI via the ctypes binding."""
 import numpy as np
 import pytest
 import torch
@@ -24,6 +24,32 @@ def _host(t: torch.Tensor) -> np.ndarray:
     return t.cpu().numpy()
 
 
+class _Variant:
+    def __init__(self, name, rec):
+        self.name, self.rec = name, rec
+
+    def gpu_chunks(self, ctx, data, chunk):
+        return getattr(ctx, f"hash_chunks_{self.name}")(data, chunk)
+
+    def gpu_root(self, ctx, leaves):
+        return getattr(ctx, f"merkle_root_{self.name}")(leaves)
+
+    def cpu_chunks(self, host, chunk, nthreads=1):
+        return getattr(oracle, f"hash_chunks_{self.name}")(host, chunk, nthreads=nthreads)
+
+    def cpu_root(self, leaves):
+        return getattr(oracle, f"merkle_root_{self.name}")(leaves)
+
+    def cpu_hash(self, msg):
+        return getattr(oracle, self.name)(msg)
+
+    def __repr__(self):
+        return self.name
+
+
+VARIANTS = [_Variant("sha384", 48), _Variant("sha512", 64)]
+
+
 @pytest.mark.parametrize("nbytes,chunk", [
     (64 << 20, 64 << 10),                 # the small configuration
     (1 << 20, 4096), (1 << 20, 128), (1 << 20, 1 << 20), (1 << 20, 2 << 20),
@@ -36,56 +62,88 @@ def _host(t: torch.Tensor) -> np.ndarray:
     (19_000 * 4096, 4096),
     (9_600 * 65536, 65536),               # larger chunks, many chains
     (9_600 * 65536 + 127, 65536), (9_500 * (65536 + 16), 65536 + 16), (9_500 * (65536 + 112), 65536 + 112),
+    # the two-warp kernel: one group, one chunk, one group and a lane; more groups than worker pairs (888 on
+    # 148 SMs); many slices per chunk (1 MiB: 64, 4 MiB: 256); the last slice shorter than the others
+    (32 * 16384, 16384), (16384, 16384), (33 * 16384, 16384), (30_000 * 16384, 16384), (40 * (1 << 20), 1 << 20),
+    (36 * (4 << 20) + 4096, 4 << 20), (70 * (20480 + 48), 20480 + 48), (150 * (5 * 16384 - 128), 5 * 16384 - 128),
+    (500 * 32 * 16384, 16384), (4096 * 32 * 16384, 16384),       # group counts the plain kernel keeps
 ])
-def test_hash_chunks_sha384_equals_oracle(ctx, nbytes, chunk):
+@pytest.mark.parametrize("variant", VARIANTS, ids=repr)
+def test_hash_chunks_equals_oracle(ctx, variant, nbytes, chunk):
     data = inputs.uniform_bytes(nbytes, seed=384, device="cuda")
-    got = ctx.hash_chunks_sha384(data, chunk)
-    want = oracle.hash_chunks_sha384(_host(data), chunk, nthreads=oracle.host_threads())
+    got = variant.gpu_chunks(ctx, data, chunk)
+    groups = -(-(nbytes // chunk) // 32)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    if chunk >= 16384 and chunk % 16 == 0 and nbytes >= chunk and groups < 4096 and not (3 * sms <= groups <= 4 * sms):
+        assert ctx.last_leaf_kernel == "hash_sha512_pairs_kernel"
+    else:
+        assert ctx.last_leaf_kernel == "hash_chunks_sha384_kernel"
+    want = variant.cpu_chunks(_host(data), chunk, nthreads=oracle.host_threads())
     assert got.shape == want.shape
     assert np.array_equal(_host(got), want)
+    assert ctx.device_status() == 0
 
 
 @pytest.mark.parametrize("shift", [1, 3, 8, 13])
-@pytest.mark.parametrize("chunk", [256, 1000, 4096 + 3])
-def test_hash_chunks_sha384_any_base_alignment(ctx, shift, chunk):
+@pytest.mark.parametrize("chunk", [256, 1000, 4096 + 3, 16384])
+@pytest.mark.parametrize("variant", VARIANTS, ids=repr)
+def test_hash_chunks_any_base_alignment(ctx, variant, shift, chunk):
     buf = inputs.uniform_bytes(300_000 + 16, seed=385, device="cuda")
     data = buf[shift:shift + 300_000]
-    got = ctx.hash_chunks_sha384(data, chunk)
-    assert np.array_equal(_host(got), oracle.hash_chunks_sha384(_host(data), chunk))
+    got = variant.gpu_chunks(ctx, data, chunk)
+    assert ctx.last_leaf_kernel == "hash_chunks_sha384_kernel"
+    assert np.array_equal(_host(got), variant.cpu_chunks(_host(data), chunk))
 
 
-def test_hash_chunks_sha384_every_tail_length_of_two_blocks(ctx):
+@pytest.mark.parametrize("variant", VARIANTS, ids=repr)
+def test_hash_chunks_every_tail_length_of_two_blocks(ctx, variant):
     # one message per length 0..256 through the chunk entry point: the padding cases of section 5.1.2
     buf = inputs.uniform_bytes(257, seed=386, device="cuda")
     host = _host(buf)
     for n in range(1, 257):
-        got = ctx.hash_chunks_sha384(buf[:n], 512)
-        assert _host(got).tobytes() == oracle.sha384(host[:n]), n
+        got = variant.gpu_chunks(ctx, buf[:n], 512)
+        assert _host(got).tobytes() == variant.cpu_hash(host[:n]), n
 
 
-def test_hash_chunks_sha384_empty_and_argument_errors(ctx):
+@pytest.mark.parametrize("variant", VARIANTS, ids=repr)
+def test_two_warp_kernel_every_chunk_remainder(ctx, variant):
+    """Chunks of 16384 + r bytes for r = 0, 16, ..., 112 and beyond: the tail (remainder + padding) the producer
+    builds behind the tiled copies, on both sides of the one-block / two-block padding boundary."""
+    for r in range(0, 256, 16):
+        chunk = 16384 + r
+        data = inputs.uniform_bytes(45 * chunk, seed=390 + r, device="cuda")
+        got = variant.gpu_chunks(ctx, data, chunk)
+        assert ctx.last_leaf_kernel == "hash_sha512_pairs_kernel"
+        assert np.array_equal(_host(got), variant.cpu_chunks(_host(data), chunk)), r
+    assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("variant", VARIANTS, ids=repr)
+def test_hash_chunks_empty_and_argument_errors(ctx, variant):
     empty = torch.empty(0, dtype=torch.uint8, device="cuda")
-    assert ctx.hash_chunks_sha384(empty, 4096).shape == (0, 48)
+    assert variant.gpu_chunks(ctx, empty, 4096).shape == (0, variant.rec)
     with pytest.raises(binding.IvError):
-        ctx.hash_chunks_sha384(inputs.uniform_bytes(100, seed=1, device="cuda"), 0)
+        variant.gpu_chunks(ctx, inputs.uniform_bytes(100, seed=1, device="cuda"), 0)
 
 
 @pytest.mark.parametrize("n", [0, 1, 2, 3, 4, 5, 7, 8, 9, 127, 128, 129, 1000, 1023, 1024, 1025, 40_001])
-def test_merkle_root_sha384_equals_oracle(ctx, n):
-    leaves = inputs.uniform_bytes(48 * n, seed=387 + n, device="cuda").reshape(n, 48)
-    got = _host(ctx.merkle_root_sha384(leaves)).tobytes()
-    assert got == oracle.merkle_root_sha384(_host(leaves))
+@pytest.mark.parametrize("variant", VARIANTS, ids=repr)
+def test_merkle_root_equals_oracle(ctx, variant, n):
+    leaves = inputs.uniform_bytes(variant.rec * n, seed=387 + n, device="cuda").reshape(n, variant.rec)
+    got = _host(variant.gpu_root(ctx, leaves)).tobytes()
+    assert got == variant.cpu_root(_host(leaves))
 
 
-def test_sha384_chunks_then_root_repeated_calls(ctx):
+@pytest.mark.parametrize("variant", VARIANTS, ids=repr)
+def test_chunks_then_root_repeated_calls(ctx, variant):
     data = inputs.uniform_bytes((8 << 20) + 5, seed=388, device="cuda")
-    want_leaves = oracle.hash_chunks_sha384(_host(data), 4096, nthreads=oracle.host_threads())
-    want_root = oracle.merkle_root_sha384(want_leaves)
+    want_leaves = variant.cpu_chunks(_host(data), 4096, nthreads=oracle.host_threads())
+    want_root = variant.cpu_root(want_leaves)
     for _ in range(3):
-        leaves = ctx.hash_chunks_sha384(data, 4096)
-        assert _host(ctx.merkle_root_sha384(leaves)).tobytes() == want_root
+        leaves = variant.gpu_chunks(ctx, data, 4096)
+        assert _host(variant.gpu_root(ctx, leaves)).tobytes() == want_root
     # a smaller tree after a larger one reuses the level buffers
-    assert _host(ctx.merkle_root_sha384(leaves[:5])).tobytes() == oracle.merkle_root_sha384(want_leaves[:5])
+    assert _host(variant.gpu_root(ctx, leaves[:5].contiguous())).tobytes() == variant.cpu_root(want_leaves[:5])
     assert ctx.device_status() == 0
 
 
