@@ -368,6 +368,24 @@ int iv_verify_manifest_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
                               const iv_manifest_sha384 *h_manifest, iv_verify_result_sha384 *d_result,
                               uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream);
 
+/* The same for SHA-512: 64-byte records. */
+typedef struct iv_manifest_sha512 {
+    uint64_t total_bytes;
+    uint64_t chunk_bytes;
+    uint64_t n_chunks;
+    const uint8_t *d_digests; /* DEVICE: n_chunks * 64 bytes */
+    uint8_t root[64];
+} iv_manifest_sha512;
+typedef struct iv_verify_result_sha512 {
+    uint32_t status;
+    uint32_t root_ok;
+    uint64_t n_mismatch;
+    uint8_t root[64];
+} iv_verify_result_sha512;
+int iv_verify_manifest_sha512(iv_ctx *ctx, const void *d_data, uint64_t nbytes,
+                              const iv_manifest_sha512 *h_manifest, iv_verify_result_sha512 *d_result,
+                              uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------
  * RFC 6962 section 2.1 mode -- the Merkle Tree Hash the paper cites for its tree,
  * with that RFC's domain separation, over SHA-256 with the chunks as entries:

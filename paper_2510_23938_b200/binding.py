@@ -32,7 +32,7 @@ EXPORTS = (
     "iv_tree_records", "iv_tree_build", "iv_tree_update",
     "iv_hash_chunks_two_level", "iv_verify_manifest_two_level", "iv_hash_ragged_update", "iv_verify_manifest_batch",
     "iv_hash_chunks_sha384", "iv_merkle_root_sha384", "iv_verify_manifest_sha384",
-    "iv_hash_chunks_sha512", "iv_merkle_root_sha512",
+    "iv_hash_chunks_sha512", "iv_merkle_root_sha512", "iv_verify_manifest_sha512",
     "iv_hash_chunks_rfc6962", "iv_merkle_root_rfc6962", "iv_verify_manifest_rfc6962",
 )
 
@@ -63,6 +63,19 @@ class VerifyResult384(ctypes.Structure):
     """iv_verify_result_sha384 as laid out in device memory (64 bytes)."""
     _fields_ = [("status", ctypes.c_uint32), ("root_ok", ctypes.c_uint32),
                 ("n_mismatch", ctypes.c_uint64), ("root", ctypes.c_uint8 * 48)]
+
+
+class Manifest512(ctypes.Structure):
+    """iv_manifest_sha512: host struct, 64-byte digest records on the device."""
+    _fields_ = [("total_bytes", ctypes.c_uint64), ("chunk_bytes", ctypes.c_uint64),
+                ("n_chunks", ctypes.c_uint64), ("d_digests", ctypes.c_void_p),
+                ("root", ctypes.c_uint8 * 64)]
+
+
+class VerifyResult512(ctypes.Structure):
+    """iv_verify_result_sha512 as laid out in device memory (80 bytes)."""
+    _fields_ = [("status", ctypes.c_uint32), ("root_ok", ctypes.c_uint32),
+                ("n_mismatch", ctypes.c_uint64), ("root", ctypes.c_uint8 * 64)]
 
 
 class VerifyResult(ctypes.Structure):
@@ -123,6 +136,8 @@ def load_library() -> ctypes.CDLL:
     lib.iv_hash_chunks_sha512.restype = i32
     lib.iv_merkle_root_sha512.argtypes = [vp, vp, u64, vp, vp]
     lib.iv_merkle_root_sha512.restype = i32
+    lib.iv_verify_manifest_sha512.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest512), vp, vp, u64, vp]
+    lib.iv_verify_manifest_sha512.restype = i32
     lib.iv_verify_manifest_rfc6962.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest), vp, vp, u64, vp]
     lib.iv_verify_manifest_rfc6962.restype = i32
     lib.iv_verify_manifest_sha384.argtypes = [vp, vp, u64, ctypes.POINTER(Manifest384), vp, vp, u64, vp]
@@ -332,6 +347,21 @@ class Context:
                                                  _dev_ptr(mismatch_idx), cap, _stream_ptr(stream))
         self._check(rc, "iv_verify_manifest_sha384")
         r = VerifyResult384.from_buffer_copy(bytes(result.cpu().numpy().tobytes()))
+        return {"status": int(r.status), "root_ok": bool(r.root_ok), "n_mismatch": int(r.n_mismatch), "root": bytes(r.root)}
+
+    def verify_manifest_sha512(self, data: torch.Tensor, total_bytes: int, chunk_bytes: int, digests: torch.Tensor,
+                               root: bytes, mismatch_idx: torch.Tensor | None = None, stream=None) -> dict:
+        """iv_verify_manifest_sha512: as verify_manifest_sha384 with (n, 64) digests and a 64-byte root."""
+        m = Manifest512()
+        m.total_bytes, m.chunk_bytes, m.n_chunks = total_bytes, chunk_bytes, digests.numel() // 64
+        m.d_digests = _dev_ptr(digests)
+        m.root = (ctypes.c_uint8 * 64).from_buffer_copy(root)
+        result = torch.zeros(ctypes.sizeof(VerifyResult512), dtype=torch.uint8, device=data.device)
+        cap = 0 if mismatch_idx is None else mismatch_idx.numel()
+        rc = self._lib.iv_verify_manifest_sha512(self._h, _dev_ptr(data), _nbytes(data), ctypes.byref(m), _dev_ptr(result),
+                                                 _dev_ptr(mismatch_idx), cap, _stream_ptr(stream))
+        self._check(rc, "iv_verify_manifest_sha512")
+        r = VerifyResult512.from_buffer_copy(bytes(result.cpu().numpy().tobytes()))
         return {"status": int(r.status), "root_ok": bool(r.root_ok), "n_mismatch": int(r.n_mismatch), "root": bytes(r.root)}
 
     def hash_chunks_rfc6962(self, data: torch.Tensor, chunk_bytes: int, stream=None,

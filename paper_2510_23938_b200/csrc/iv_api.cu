@@ -47,8 +47,8 @@ struct iv_ctx {
     uint64_t slices_cap = 0;                  // bytes
 
     // streaming windows
-    uint8_t *d_digests384 = nullptr;          // chunk digests of iv_verify_manifest_sha384, then its 48-byte root
-    uint64_t digests384_cap = 0;              // records of 48 bytes
+    uint8_t *d_digests384 = nullptr;          // chunk digests of iv_verify_manifest_sha384 / _sha512, then the root
+    uint64_t digests384_cap = 0;              // records of 64 bytes
     uint8_t *d_columns = nullptr;             // offsets, lengths and chaining values of a window hashed in column parts
     uint64_t columns_cap = 0;                 // bytes
     uint8_t *d_window[2] = {nullptr, nullptr};
@@ -871,32 +871,55 @@ int iv_merkle_root_sha512(iv_ctx *ctx, const uint8_t *d_leaves, uint64_t n_leave
     return merkle_root_wide(ctx, d_leaves, n_leaves, d_root, 8, cuda_stream);
 }
 
-int iv_verify_manifest_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest_sha384 *m,
-                              iv_verify_result_sha384 *d_result, uint64_t *d_mismatch_idx, uint64_t idx_cap,
-                              void *cuda_stream) {
+extern "C++" {
+namespace {
+
+// iv_verify_manifest over SHA-384 (WORDS 6) or SHA-512 (8) records: hash, tree, compare.
+template <int WORDS, class Manifest, class Result, class Root>
+int verify_manifest_wide(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const Manifest *m, Result *d_result,
+                         uint64_t *d_mismatch_idx, uint64_t idx_cap, void *cuda_stream,
+                         cudaError_t (*compare)(const uint8_t *, const uint8_t *, uint64_t, const uint8_t *, Root, Result *,
+                                                uint64_t *, uint64_t, uint32_t *, uint32_t *, const uint32_t *, cudaStream_t,
+                                                uint64_t *)) {
+    constexpr uint64_t REC = 8 * WORDS;
     if (!ctx || !d_result || (idx_cap && !d_mismatch_idx)) return IV_ERR_INVALID_ARG;
     if (!m || m->chunk_bytes == 0 || m->total_bytes != nbytes) return IV_ERR_INVALID_ARG;
     const uint64_t n = chunk_count(nbytes, m->chunk_bytes);
     if (m->n_chunks != n || (n && !m->d_digests) || (nbytes && !d_data)) return IV_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    int rc = grow(ctx, &ctx->d_digests384, &ctx->digests384_cap, n + 2, 48);      // digests, then the root
+    int rc = grow(ctx, &ctx->d_digests384, &ctx->digests384_cap, n + 2, 64);      // digests, then the root
     if (rc != IV_OK) return rc;
     if ((rc = ensure_variant_tree_scratch(ctx, (n + 1) / 2 + 1)) != IV_OK) return rc;
     if ((rc = grow(ctx, &ctx->d_words, &ctx->words_cap, (n + 31) / 32 + 1, sizeof(uint32_t))) != IV_OK) return rc;
-    uint8_t *d_root = ctx->d_digests384 + 48 * (n + 1);
-    if (n && (rc = hash_leaves_wide(ctx, static_cast<const uint8_t *>(d_data), nbytes, m->chunk_bytes, n, ctx->d_digests384, 6,
-                                    stream)) != IV_OK)
+    uint8_t *d_root = ctx->d_digests384 + REC * (n + 1);
+    if (n && (rc = hash_leaves_wide(ctx, static_cast<const uint8_t *>(d_data), nbytes, m->chunk_bytes, n, ctx->d_digests384,
+                                    WORDS, stream)) != IV_OK)
         return rc;
-    IV_TRY(ctx, ivk::launch_merkle_root_sha384(ctx->d_digests384, n, d_root, ctx->d_tree384[0], ctx->d_tree384[1], 6, stream,
-                                               &ctx->launches));
-    ivk::RootBytes384 expect;
-    std::memcpy(expect.b, m->root, 48);
-    IV_TRY(ctx, ivk::launch_verify_compare_sha384(ctx->d_digests384, m->d_digests, n, d_root, expect, d_result,
-                                                  d_mismatch_idx, idx_cap, ctx->d_words,
-                                                  ctx->d_tickets + ivk::kMerkleMaxPasses, ctx->d_status, stream,
-                                                  &ctx->launches));
+    IV_TRY(ctx, ivk::launch_merkle_root_sha384(ctx->d_digests384, n, d_root, ctx->d_tree384[0], ctx->d_tree384[1], WORDS,
+                                               stream, &ctx->launches));
+    Root expect;
+    std::memcpy(expect.b, m->root, REC);
+    IV_TRY(ctx, compare(ctx->d_digests384, m->d_digests, n, d_root, expect, d_result, d_mismatch_idx, idx_cap, ctx->d_words,
+                        ctx->d_tickets + ivk::kMerkleMaxPasses, ctx->d_status, stream, &ctx->launches));
     return IV_OK;
+}
+
+}  // namespace
+}  // extern "C++"
+
+int iv_verify_manifest_sha384(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest_sha384 *m,
+                              iv_verify_result_sha384 *d_result, uint64_t *d_mismatch_idx, uint64_t idx_cap,
+                              void *cuda_stream) {
+    return verify_manifest_wide<6, iv_manifest_sha384, iv_verify_result_sha384, ivk::RootBytes384>(
+        ctx, d_data, nbytes, m, d_result, d_mismatch_idx, idx_cap, cuda_stream, ivk::launch_verify_compare_sha384);
+}
+
+int iv_verify_manifest_sha512(iv_ctx *ctx, const void *d_data, uint64_t nbytes, const iv_manifest_sha512 *m,
+                              iv_verify_result_sha512 *d_result, uint64_t *d_mismatch_idx, uint64_t idx_cap,
+                              void *cuda_stream) {
+    return verify_manifest_wide<8, iv_manifest_sha512, iv_verify_result_sha512, ivk::RootBytes512>(
+        ctx, d_data, nbytes, m, d_result, d_mismatch_idx, idx_cap, cuda_stream, ivk::launch_verify_compare_sha512);
 }
 
 int iv_hash_chunks_rfc6962(iv_ctx *ctx, const void *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint8_t *d_digests,

@@ -130,6 +130,12 @@ cudaError_t launch_tree_update(uint8_t *d_tree, uint64_t n_leaves, const uint8_t
 // uint32 mask words; d_ticket one zeroed uint32.
 struct RootBytes { uint8_t b[32]; };
 struct RootBytes384 { uint8_t b[48]; };
+struct RootBytes512 { uint8_t b[64]; };
+cudaError_t launch_verify_compare_sha512(const uint8_t *d_digests, const uint8_t *d_manifest_digests,
+                                         uint64_t n, const uint8_t *d_root, RootBytes512 manifest_root,
+                                         iv_verify_result_sha512 *d_result, uint64_t *d_mismatch_idx,
+                                         uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
+                                         const uint32_t *d_status, cudaStream_t stream, uint64_t *launches);
 cudaError_t launch_verify_compare_sha384(const uint8_t *d_digests, const uint8_t *d_manifest_digests,
                                          uint64_t n, const uint8_t *d_root, RootBytes384 manifest_root,
                                          iv_verify_result_sha384 *d_result, uint64_t *d_mismatch_idx,

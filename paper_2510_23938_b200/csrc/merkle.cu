@@ -288,7 +288,7 @@ __global__ void empty_root_kernel(uint8_t *d_root) {
 // words into the ascending index list with a block-wide exclusive scan.
 // ---------------------------------------------------------------------------
 
-// REC: bytes per digest record (32 for SHA-256, 48 for SHA-384).
+// REC: bytes per digest record (32 for SHA-256, 48 for SHA-384, 64 for SHA-512).
 template <int REC>
 __device__ __forceinline__ bool digest_differs(const uint8_t *a, const uint8_t *b, bool aligned) {
     uint32_t diff = 0;
@@ -550,6 +550,22 @@ cudaError_t launch_verify_compare_sha384(const uint8_t *d_digests, const uint8_t
     if (blocks == 0) blocks = 1;
     if (blocks > 1184) blocks = 1184;
     verify_compare_kernel<48, iv_verify_result_sha384, RootBytes384><<<(unsigned)blocks, kThreads, 0, stream>>>(
+        d_digests, d_manifest_digests, n, d_root, manifest_root, d_result, d_mismatch_idx, idx_cap,
+        d_words, d_ticket, d_status);
+    if (launches) ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_verify_compare_sha512(const uint8_t *d_digests, const uint8_t *d_manifest_digests,
+                                         uint64_t n, const uint8_t *d_root, RootBytes512 manifest_root,
+                                         iv_verify_result_sha512 *d_result, uint64_t *d_mismatch_idx,
+                                         uint64_t idx_cap, uint32_t *d_words, uint32_t *d_ticket,
+                                         const uint32_t *d_status, cudaStream_t stream, uint64_t *launches) {
+    const uint64_t n_words = (n + 31) / 32;
+    uint64_t blocks = (n_words + (kThreads / 32) - 1) / (kThreads / 32);
+    if (blocks == 0) blocks = 1;
+    if (blocks > 1184) blocks = 1184;
+    verify_compare_kernel<64, iv_verify_result_sha512, RootBytes512><<<(unsigned)blocks, kThreads, 0, stream>>>(
         d_digests, d_manifest_digests, n, d_root, manifest_root, d_result, d_mismatch_idx, idx_cap,
         d_words, d_ticket, d_status);
     if (launches) ++*launches;

@@ -148,31 +148,33 @@ def test_chunks_then_root_repeated_calls(ctx, variant):
 
 
 @pytest.mark.parametrize("nbytes,chunk", [((8 << 20) + 300, 4096), (64 << 20, 64 << 10), (100_003, 1001), (5000, 8192)])
-def test_verification_against_a_sha384_manifest_from_the_oracle(ctx, nbytes, chunk):
-    """Manifest = the oracle's SHA-384 chunk digests and root: clean data passes, flipped bits are located in
+@pytest.mark.parametrize("variant", VARIANTS, ids=repr)
+def test_verification_against_a_manifest_from_the_oracle(ctx, variant, nbytes, chunk):
+    """Manifest = the oracle's SHA-384 / SHA-512 chunk digests and root: clean data passes, flipped bits are located in
     ascending order with the exact count, the recomputed root is the oracle's root of the damaged blob."""
     data = inputs.uniform_bytes(nbytes, seed=3840, device="cuda")
-    digests = oracle.hash_chunks_sha384(_host(data), chunk, nthreads=oracle.host_threads())
-    root = oracle.merkle_root_sha384(digests)
+    digests = variant.cpu_chunks(_host(data), chunk, nthreads=oracle.host_threads())
+    root = variant.cpu_root(digests)
     d_digests = torch.from_numpy(digests).cuda()
+    verify = getattr(ctx, f"verify_manifest_{variant.name}")
     n = digests.shape[0]
     idx = torch.zeros(4, dtype=torch.int64, device="cuda")
-    r = ctx.verify_manifest_sha384(data, nbytes, chunk, d_digests, root, idx)
+    r = verify(data, nbytes, chunk, d_digests, root, idx)
     assert r == {"status": 0, "root_ok": True, "n_mismatch": 0, "root": root}
     bad = data.clone()
     hits = sorted({inputs.flip_position(s, nbytes) for s in range(11, 18)})
     for off, bit in hits:
         bad[off] ^= (1 << bit)
-    want = oracle.hash_chunks_sha384(_host(bad), chunk, nthreads=oracle.host_threads())
+    want = variant.cpu_chunks(_host(bad), chunk, nthreads=oracle.host_threads())
     want_idx = [i for i in range(n) if bytes(want[i]) != bytes(digests[i])]
     assert want_idx == sorted({off // chunk for off, _ in hits})
-    r = ctx.verify_manifest_sha384(bad, nbytes, chunk, d_digests, root, idx)
-    assert (not r["root_ok"]) and r["n_mismatch"] == len(want_idx) and r["root"] == oracle.merkle_root_sha384(want)
+    r = verify(bad, nbytes, chunk, d_digests, root, idx)
+    assert (not r["root_ok"]) and r["n_mismatch"] == len(want_idx) and r["root"] == variant.cpu_root(want)
     assert [int(v) for v in idx[:min(4, len(want_idx))].cpu()] == want_idx[:4]
     # manifest-side damage: one digest of the manifest changed, the data clean
     d_digests[n // 2, 7] ^= 1
-    r = ctx.verify_manifest_sha384(data, nbytes, chunk, d_digests, root, idx)
+    r = verify(data, nbytes, chunk, d_digests, root, idx)
     assert r["root_ok"] and r["n_mismatch"] == 1 and int(idx[0]) == n // 2
     with pytest.raises(binding.IvError):
-        ctx.verify_manifest_sha384(data, nbytes + 1, chunk, d_digests, root, idx)
+        verify(data, nbytes + 1, chunk, d_digests, root, idx)
     assert ctx.device_status() == 0

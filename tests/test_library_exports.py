@@ -39,6 +39,8 @@ def test_struct_layouts_match_the_header():
     assert binding.VerifyResult.root.offset == 16
     assert ctypes.sizeof(binding.Manifest) == 64
     assert binding.Manifest.root.offset == 32
+    assert ctypes.sizeof(binding.VerifyResult384) == 64 and ctypes.sizeof(binding.VerifyResult512) == 80
+    assert ctypes.sizeof(binding.Manifest384) == 80 and ctypes.sizeof(binding.Manifest512) == 96
 
 
 def test_create_fails_loudly_without_a_device():
