@@ -272,7 +272,9 @@ int iv_verify_streamed(iv_ctx *ctx, const void *const *h_windows, uint64_t n_win
  * switched on, iv_verify_manifest and iv_verify_streamed bracket their three
  * phases -- leaf hashing, tree reduction, comparison -- with CUDA events on
  * cuda_stream.  The context keeps the events of the most recent
- * IV_TIMING_RING verification calls.
+ * IV_TIMING_RING verification calls.  Independently of this switch the three
+ * phases are NVTX ranges ("iv: leaf hashing", "iv: Merkle reduction",
+ * "iv: manifest compare") around the launches of each phase, for profilers.
  *
  * iv_phase_times waits for the events of the call made `calls_back` calls ago
  * (0 = the most recent) and writes the three durations in milliseconds to

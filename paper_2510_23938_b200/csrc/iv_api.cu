@@ -4,6 +4,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "iv_internal.h"
 
 struct iv_ctx {
@@ -57,6 +59,10 @@ struct iv_ctx {
     cudaStream_t tail_stream = nullptr;       // a blob's short last chunk is hashed here, beside the main leaf kernel
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaEvent_t ev_entry = nullptr, ev_copied[2] = {nullptr, nullptr}, ev_hashed[2] = {nullptr, nullptr};
+
+    // NVTX range of the phase the current verification call is in (leaf hashing / Merkle reduction / compare)
+    nvtxRangeId_t nvtx_id = 0;
+    bool nvtx_open = false;
 
     // phase timing: four events (start, hashed, reduced, compared) per recent call
     bool timing = false;
@@ -259,8 +265,19 @@ int hash_window_in_columns(iv_ctx *ctx, const void *h_window, uint64_t bytes, ui
     return IV_OK;
 }
 
-// Records phase event `which` (0..3) of the current verification call when timing is on.
+// Phase boundary `which` (0 = leaf hashing begins, 1 = tree reduction begins, 2 = comparison begins, 3 = done) of
+// the current verification call: closes and opens the NVTX range of the phase (profilers show the launches of a
+// phase under its name; without a tool attached the calls do nothing) and, when timing is on, records the event.
 int mark_phase(iv_ctx *ctx, int which, cudaStream_t stream) {
+    static const char *const names[3] = {"iv: leaf hashing", "iv: Merkle reduction", "iv: manifest compare"};
+    if (ctx->nvtx_open) {
+        nvtxRangeEnd(ctx->nvtx_id);
+        ctx->nvtx_open = false;
+    }
+    if (which < 3) {
+        ctx->nvtx_id = nvtxRangeStartA(names[which]);
+        ctx->nvtx_open = true;
+    }
     if (!ctx->timing) return IV_OK;
     const uint32_t slot = (uint32_t)(ctx->timed_calls % IV_TIMING_RING);
     for (int k = 0; k < 4; ++k)
@@ -373,6 +390,7 @@ int iv_create(iv_ctx **out, int cuda_device) {
 int iv_destroy(iv_ctx *ctx) {
     if (!ctx) return IV_OK;
     DeviceGuard guard(ctx->device);
+    if (ctx->nvtx_open) nvtxRangeEnd(ctx->nvtx_id);
     cudaDeviceSynchronize();
     cudaFree(ctx->d_small);
     cudaFree(ctx->d_merkle_a);
