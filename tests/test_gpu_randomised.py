@@ -92,6 +92,31 @@ def test_migrating_kernel_on_random_large_shapes(ctx):
     assert ctx.device_status() == 0
 
 
+def test_sha384_and_sha512_two_warp_kernel_on_random_shapes(ctx):
+    """Random group counts from one warp's worth of chains to more groups than worker pairs, chunk sizes of 16 KiB
+    to 600 KiB that are multiples of 16 bytes (any remainder mod 128: every tail the producer builds; slice counts
+    from 1 to 37), a short last chunk: the shapes of the SHA-384 / SHA-512 kernel on the slice FIFO."""
+    rng = np.random.default_rng(512)
+    seen = set()
+    for k in range(10):
+        chunk = 16 * int(rng.integers(1024, 38_000)) if k % 3 else 16 * int(rng.integers(1024, 2_100))
+        budget = 700 << 20
+        n_chunks = int(rng.integers(1, max(2, min(40_000, budget // chunk))))
+        tail = int(rng.integers(1, chunk + 1))
+        nbytes = (n_chunks - 1) * chunk + tail
+        data = inputs.uniform_bytes(nbytes, seed=nbytes, device="cuda")
+        host = _host(data)
+        got = ctx.hash_chunks_sha384(data, chunk)
+        seen.add(ctx.last_leaf_kernel)
+        assert np.array_equal(_host(got), oracle.hash_chunks_sha384(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk)
+        got = ctx.hash_chunks_sha512(data, chunk)
+        assert np.array_equal(_host(got), oracle.hash_chunks_sha512(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk)
+        assert _host(ctx.merkle_root_sha512(got)).tobytes() == oracle.merkle_root_sha512(_host(got)), (nbytes, chunk)
+        del data
+    assert "hash_sha512_pairs_kernel" in seen
+    assert ctx.device_status() == 0
+
+
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_random_tensor_sets(ctx, seed):
     rng = np.random.default_rng(1000 + seed)
