@@ -47,10 +47,18 @@ SM_COUNT = 148
 SM_HZ = 1.965e9
 PEAK_GBS = SM_COUNT * INT_LANES_PER_SM * SM_HZ / INT_OPS_PER_BYTE / 1e9
 # Cycles ONE chain needs per 64-byte block when its warps have their SM schedulers to themselves: the
-# two-warp kernel as measured on the 16 GB configuration (leaf-kernel time x clock / blocks per chunk),
-# and the issue floor of the round function (10 SHF/LOP3 per round on a 16-lane pipe, two cycles each).
-SPLIT_CYCLES_PER_BLOCK = 1965.0
+# two-warp kernel as measured (leaf-kernel time x clock / blocks per chunk) in its instance for up to one
+# group of 32 chains per SM (the 16 GB configuration) and in the one for up to two, and the issue floor of
+# the round function (10 SHF/LOP3 per round on a 16-lane pipe, two cycles each).
+SPLIT_CYCLES_PER_BLOCK_ROOMY = 1877.0
+SPLIT_CYCLES_PER_BLOCK = 1916.0
 ISSUE_FLOOR_CYCLES_PER_BLOCK = 1280.0
+
+
+def split_cycles_per_block(chains: int) -> float:
+    return SPLIT_CYCLES_PER_BLOCK_ROOMY if -(-chains // 32) <= SM_COUNT else SPLIT_CYCLES_PER_BLOCK
+
+
 # DRAM read+write bytes per byte hashed, from the ncu captures summarised under profiles/.
 TRAFFIC_FACTOR = {"hash_chunks_sliced_kernel": 1.0034, "hash_chunks_split_kernel": 1.001}
 
@@ -240,7 +248,7 @@ def roofline_of(kernel_name: str, nbytes: int, hash_ms: float, chains: int, tree
     achieved = nbytes / (hash_ms * 1e-3) / 1e9
     factor = TRAFFIC_FACTOR.get(kernel_name.split(" ")[0])
     split = kernel_name.startswith("hash_chunks_split_kernel")
-    chain_bound = chains * 64 * SM_HZ / SPLIT_CYCLES_PER_BLOCK / 1e9
+    chain_bound = chains * 64 * SM_HZ / split_cycles_per_block(chains) / 1e9
     floor_bound = chains * 64 * SM_HZ / ISSUE_FLOOR_CYCLES_PER_BLOCK / 1e9
     return {
         "bound": "alu", "kernel": kernel_name,
@@ -253,7 +261,7 @@ def roofline_of(kernel_name: str, nbytes: int, hash_ms: float, chains: int, tree
         # what the chain count allows: chains x 64 B x f / (cycles one chain needs per block)
         "chain_count_bound_gbs": round(min(chain_bound, PEAK_GBS), 1),
         "chain_count_bound_at_issue_floor_gbs": round(min(floor_bound, PEAK_GBS), 1),
-        "cycles_per_block_assumed": SPLIT_CYCLES_PER_BLOCK if split else None,
+        "cycles_per_block_assumed": split_cycles_per_block(chains) if split else None,
         "peak_source": "derived: 148 SMs x 64 INT32 lanes x 1.965 GHz / 21.875 INT32 ops per byte",
         "hbm_peak_gbs_measured": _measured_peak("hbm_gbs"),
         "launch_ms": round(hash_ms, 4), "tree_ms": tree_ms, "compare_ms": cmp_ms,
@@ -670,7 +678,7 @@ def measure_secondary(ctx, device, gpu_index, args):
     seconds = e0.elapsed_time(e1) * 1e-3
     c3["per_tensor"] = {"seconds": round(seconds, 3), "n_tensors": len(table), "bytes": int(lens.sum().item()),
                         "longest_bytes": longest, "leaf_kernel": ctx.last_leaf_kernel,
-                        "bound_seconds": round(longest / 64 * SPLIT_CYCLES_PER_BLOCK / SM_HZ, 3),
+                        "bound_seconds": round(longest / 64 * split_cycles_per_block(len(table)) / SM_HZ, 3),
                         "bound": "longest_bytes / 64 x cycles per block of one chain / SM clock (one tensor is one serial chain)",
                         "device_status": ctx.device_status(), "clocks": clocks.summary()}
     out["config3"] = c3

@@ -61,7 +61,10 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     const uint32_t bar_full = bar_data + 8 * STAGES;
     const uint32_t bar_empty = bar_full + 8 * NSLOT;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES + 2 * NSLOT; ++s) tma::mbar_init(bar_data + 8 * s, 1);
+        // data stages: one arrival (lane 0 announces the bytes of all 32 copies); W+K slots: every lane of the
+        // producer (full) or consumer (empty) arrives for itself, which needs no warp barrier and no one-lane branch
+        for (int s = 0; s < STAGES; ++s) tma::mbar_init(bar_data + 8 * s, 1);
+        for (int s = STAGES; s < STAGES + 2 * NSLOT; ++s) tma::mbar_init(bar_data + 8 * s, 32);
         tma::fence_barrier_init();
     }
     __syncthreads();
@@ -195,8 +198,7 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
             }
             produce_wk(w, wk_base + slot * kWkSlot + in_slot * kWkBlock, one);
             if (in_slot == PAIR - 1 || blk + 1 == warp_total) {
-                __syncwarp();                          // all 32 lanes' stores are ordered before lane 0's arrival
-                if (lane == 0) tma::mbar_arrive(bar_full + 8 * slot);
+                tma::mbar_arrive(bar_full + 8 * slot);     // every lane arrives after its own stores (release)
                 if (++slot == NSLOT) { slot = 0; eparity ^= 1u; }
             }
         }
@@ -224,12 +226,9 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
             if (failed) break;
         }
         const uint32_t src = wk_base + slot * kWkSlot + in_slot * kWkBlock;
-        rounds64(v, src, one);
         const bool slot_done = in_slot == PAIR - 1 || blk + 1 == warp_total;
-        if (slot_done) {
-            __syncwarp();                              // all 32 lanes have their values in registers
-            if (lane == 0) tma::mbar_arrive(bar_empty + 8 * slot);
-        }
+        rounds64(v, src, one);
+        if (slot_done) tma::mbar_arrive(bar_empty + 8 * slot);   // every lane arrives once its own values are in registers
         // feed-forward; a lane whose message has ended keeps its state (multiplier 0 instead of 1)
         const uint32_t keep = (blk < my_total) ? one : 0u;
 #pragma unroll
@@ -253,38 +252,63 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
 
 }  // namespace
 
+namespace {
+
+// Two instances per mode.  Up to one group per SM a CTA may use most of an SM's shared memory: three W+K slots of
+// FOUR blocks each (156 KB; a hand-over every fourth block): 1,877 cycles per block.  Up to two groups per SM two
+// CTAs share an SM: three slots of two blocks (104 KB): 1,916 cycles per block.  (Fetching the next block's first
+// W+K values during the last rounds of the current one, within a slot, was measured and does not pay: 1,890.)
+template <bool RAGGED, bool PREFIX, int PAIR>
+cudaError_t launch_split_instance(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n, uint8_t *d_digests,
+                                  uint32_t *d_status, const uint32_t *d_one, const uint64_t *d_offsets, const uint64_t *d_lengths,
+                                  const uint32_t *d_order, iv_sha_state *d_states, int finish, cudaStream_t stream) {
+    constexpr int SEG = 512, STAGES = 3, NSLOT = 3;
+    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + (RAGGED ? 32 : 16)) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
+    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, RAGGED, PAIR, PREFIX>;
+    static bool configured[kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
+    const uint64_t blocks = (n + 31) / 32;
+    if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
+    kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_data, nbytes, chunk_bytes, n, d_digests, d_status, d_one, d_offsets,
+                                                   d_lengths, d_order, d_states, finish);
+    return cudaGetLastError();
+}
+
+int sm_count_of_current_device() {
+    static int cached[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    if (!cached[dev]) cudaDeviceGetAttribute(&cached[dev], cudaDevAttrMultiProcessorCount, dev);
+    return cached[dev];
+}
+
+}  // namespace
+
 cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                                      uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status,
                                      const uint32_t *d_one, cudaStream_t stream, bool zero_prefix) {
-    // 512-byte segments, three data stages, three W+K slots of two blocks each (two blocks per hand-over
-    // halve the barrier traffic: +1 % over four single-block slots; 104 KB per CTA, two CTAs per SM); the additions that close the two state
-    // recurrences stay three-input ALU adds, the others go to the FMA pipe (placement 3, the fastest measured).
-    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, PAIR = 2;
-    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
-    auto kernel = zero_prefix ? hash_chunks_split_kernel<SEG, STAGES, NSLOT, false, PAIR, true>
-                              : hash_chunks_split_kernel<SEG, STAGES, NSLOT, false, PAIR, false>;
-    static bool configured[2][kMaxDevices] = {};
-    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured[zero_prefix ? 1 : 0]); e0 != cudaSuccess) return e0;
-    const uint64_t blocks = (n_chunks + 31) / 32;
-    if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
-    kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
-                                                   nullptr, nullptr, nullptr, nullptr, 1);
-    return cudaGetLastError();
+    // 512-byte segments, three data stages; the additions that close the two state recurrences stay three-input
+    // ALU adds, the others go to the FMA pipe (the fastest placement measured).
+    const bool roomy = (n_chunks + 31) / 32 <= (uint64_t)sm_count_of_current_device();
+    if (zero_prefix)
+        return roomy ? launch_split_instance<false, true, 4>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
+                                                             nullptr, nullptr, nullptr, nullptr, 1, stream)
+                     : launch_split_instance<false, true, 2>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
+                                                             nullptr, nullptr, nullptr, nullptr, 1, stream);
+    return roomy ? launch_split_instance<false, false, 4>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
+                                                          nullptr, nullptr, nullptr, nullptr, 1, stream)
+                 : launch_split_instance<false, false, 2>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
+                                                          nullptr, nullptr, nullptr, nullptr, 1, stream);
 }
 
 cudaError_t launch_hash_ragged_split(const uint8_t *d_base, const uint64_t *d_offsets, const uint64_t *d_lengths,
                                      const uint32_t *d_order, uint64_t n, uint8_t *d_digests, uint32_t *d_status,
                                      const uint32_t *d_one, iv_sha_state *d_states, int finish, cudaStream_t stream) {
-    constexpr int SEG = 512, STAGES = 3, NSLOT = 3, PAIR = 2;
-    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 32) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
-    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, true, PAIR>;
-    static bool configured[kMaxDevices] = {};
-    if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
-    const uint64_t blocks = (n + 31) / 32;
-    if (blocks > 0x7fffffffull) return cudaErrorInvalidConfiguration;
-    kernel<<<(unsigned)blocks, 64, smem, stream>>>(d_base, 0, 0, n, d_digests, d_status, d_one, d_offsets, d_lengths,
-                                                   d_order, d_states, finish);
-    return cudaGetLastError();
+    const bool roomy = (n + 31) / 32 <= (uint64_t)sm_count_of_current_device();
+    return roomy ? launch_split_instance<true, false, 4>(d_base, 0, 0, n, d_digests, d_status, d_one, d_offsets, d_lengths,
+                                                         d_order, d_states, finish, stream)
+                 : launch_split_instance<true, false, 2>(d_base, 0, 0, n, d_digests, d_status, d_one, d_offsets, d_lengths,
+                                                         d_order, d_states, finish, stream);
 }
 
 }  // namespace ivk

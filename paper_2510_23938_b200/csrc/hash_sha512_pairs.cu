@@ -96,7 +96,10 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
     const uint32_t bar_full = bar_data + 8 * STAGES;
     const uint32_t bar_empty = bar_full + 8 * NSLOT;
     if (producer && lane == 0) {
-        for (int s = 0; s < STAGES + 2 * NSLOT; ++s) tma::mbar_init(bar_data + 8 * s, 1);
+        // data stages: one arrival (lane 0 announces the box); W+K units: every lane of the producer (full) or of
+        // the consumer (empty) arrives for itself, which needs no warp barrier and no one-lane branch
+        for (int s = 0; s < STAGES; ++s) tma::mbar_init(bar_data + 8 * s, 1);
+        for (int s = STAGES; s < STAGES + 2 * NSLOT; ++s) tma::mbar_init(bar_data + 8 * s, 32);
         for (int s = 0; s < kTaskRing; ++s) tma::mbar_init(tma::smem_u32(&task_bars[pair][s]), 1);
         s_failed[pair] = 0u;
         tma::fence_barrier_init();
@@ -223,8 +226,7 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
                     failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded_sleepy(bar_empty + 8 * wslot, eparity));
                     if (failed) break;
                     store_wk16_512(w, kSha512K + 16 * u, wk_ring + wslot * kUnitBytes);
-                    __syncwarp();                          // all 32 lanes' stores are ordered before lane 0's arrival
-                    if (lane == 0) tma::mbar_arrive(bar_full + 8 * wslot);
+                    tma::mbar_arrive(bar_full + 8 * wslot);    // every lane arrives after its own stores (release)
                     if (++wslot == NSLOT) { wslot = 0; eparity ^= 1u; }
                 }
             }
@@ -256,8 +258,7 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
                         kw[2 * j] = pack64(x, y);
                         kw[2 * j + 1] = pack64(z, t);
                     }
-                    __syncwarp();                          // all 32 lanes have their values in registers
-                    if (lane == 0) tma::mbar_arrive(bar_empty + 8 * wslot);
+                    tma::mbar_arrive(bar_empty + 8 * wslot);   // every lane arrives once its own values are in registers
                     if (++wslot == NSLOT) { wslot = 0; fparity ^= 1u; }
                     rounds16_512(v, kw);
                 }
