@@ -4,8 +4,8 @@ The blobs are built by bench.py's own workload builder and hashed through the sa
 benchmark calls.  Every configuration is checked completely: the blob goes to the host window by window through a
 pinned staging buffer, the oracle hashes every chunk (every tensor) on the host cores, and every digest,
 the root, and the count and indices of seeded bit flips are compared bit for bit.  Manifests are built
-from the ORACLE's digests and root, never from the library's own output.  The RFC 6962 and SHA-384
-variants at the largest size stay sampled."""
+from the ORACLE's digests and root, never from the library's own output.  At the largest size the RFC 6962
+and SHA-384 variants are checked completely too; SHA-512 (the same kernel as SHA-384) is sampled."""
 import numpy as np
 import pytest
 import torch
@@ -128,12 +128,19 @@ def test_largest_configuration_completely(ctx):
     assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel" and ctx.device_status() == 0
     host_got = _host(got)
 
-    # the oracle over the whole blob, one 4 GiB window at a time
+    # the oracle over the whole blob, one 4 GiB window at a time: SHA-256 chunk digests, and the RFC 6962 leaf hashes
+    # and SHA-384 digests of the same chunks for the variants' legs below
     window = 4 * GIB
     stage = _Stager(window)
     threads = oracle.host_threads()
-    want = np.concatenate([oracle.hash_chunks(stage(data[off:off + window]), chunk, nthreads=threads)
-                           for off in range(0, nbytes, window)])
+    parts, parts6962, parts384 = [], [], []
+    for off in range(0, nbytes, window):
+        host = stage(data[off:off + window])
+        parts.append(oracle.hash_chunks(host, chunk, nthreads=threads))
+        parts6962.append(oracle.hash_chunks_rfc6962(host, chunk, nthreads=threads))
+        parts384.append(oracle.hash_chunks_sha384(host, chunk, nthreads=threads))
+    want, want6962, want384 = np.concatenate(parts), np.concatenate(parts6962), np.concatenate(parts384)
+    del parts, parts6962, parts384
     assert want.shape == (n, 32)
     bad = np.nonzero((host_got != want).any(axis=1))[0]
     assert bad.size == 0, f"{bad.size} digests differ from the oracle, first at chunk {bad[:8]}"
@@ -168,21 +175,27 @@ def test_largest_configuration_completely(ctx):
     for off, bit in flips:
         data[off] ^= (1 << bit)
 
-    # the same launch shape in the RFC 6962 mode and with SHA-384 digests (sampled)
-    rng = np.random.default_rng(4)
-    sample = sorted(set([0, 1, 31, 32, 1023, 1024, 1025, 14_335, 14_336, n - 33, n - 32, n - 2, n - 1]
-                        + [int(v) for v in rng.integers(0, n, size=40)]))
-    got6962 = _host(ctx.hash_chunks_rfc6962(data, chunk))
+    # the same launch shape in the RFC 6962 mode (prefixed instance of the migrating kernel) and with SHA-384 and
+    # SHA-512 digests (the two-warp kernel on the slice FIFO, 256 slices per chunk): every digest; SHA-512 sampled
+    got6962 = ctx.hash_chunks_rfc6962(data, chunk)
     assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel" and ctx.device_status() == 0
-    for i in sample[::3]:
-        w = oracle.hash_chunks_rfc6962(stage(data[i * chunk:(i + 1) * chunk]), chunk)[0]
-        assert got6962[i].tobytes() == w.tobytes(), i
+    bad = np.nonzero((_host(got6962) != want6962).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} RFC 6962 leaf hashes differ from the oracle, first at chunk {bad[:8]}"
+    assert _host(ctx.merkle_root_rfc6962(got6962)).tobytes() == oracle.merkle_root_rfc6962(want6962)
     del got6962
-    got384 = _host(ctx.hash_chunks_sha384(data, chunk))
-    assert ctx.device_status() == 0
-    for i in sample[1::3]:
-        assert got384[i].tobytes() == oracle.sha384(stage(data[i * chunk:(i + 1) * chunk])), i
+    got384 = ctx.hash_chunks_sha384(data, chunk)
+    assert ctx.last_leaf_kernel == "hash_sha512_pairs_kernel" and ctx.device_status() == 0
+    bad = np.nonzero((_host(got384) != want384).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} SHA-384 digests differ from the oracle, first at chunk {bad[:8]}"
+    assert _host(ctx.merkle_root_sha384(got384)).tobytes() == oracle.merkle_root_sha384(want384)
     del got384
+    rng = np.random.default_rng(4)
+    sample = sorted(set([0, 1, 31, 32, 1023, 1024, n - 33, n - 32, n - 1] + [int(v) for v in rng.integers(0, n, size=12)]))
+    got512 = _host(ctx.hash_chunks_sha512(data, chunk))
+    assert ctx.device_status() == 0
+    for i in sample:
+        assert got512[i].tobytes() == oracle.sha512(stage(data[i * chunk:(i + 1) * chunk])), i
+    del got512
 
     # streamed from pinned host windows (a ring of two 4 GiB windows read as windows 0 and 1 of the blob),
     # against the oracle's digests of those windows
