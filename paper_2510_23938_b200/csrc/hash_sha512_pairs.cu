@@ -155,7 +155,7 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
             first_take = false;
             task = __shfl_sync(0xffffffffu, task, 0);
         } else {
-            if (!tma::mbar_wait_bounded(task_bar, (turn / kTaskRing) & 1u)) { failed = true; break; }
+            if (!tma::mbar_wait_bounded_sleepy(task_bar, (turn / kTaskRing) & 1u)) { failed = true; break; }
             task = *reinterpret_cast<volatile unsigned long long *>(&s_task[pair][turn % kTaskRing]);
         }
         if (task == kTaskDone) break;
@@ -244,11 +244,17 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
             }
 #pragma unroll
             for (int k = 0; k < 8; ++k) v[k] = st[k];
-            for (uint32_t blk = 0; blk < n_total && !failed; ++blk) {
+            // Five units of sixteen rounds per block.  A satisfied blocking wait in front of every unit costs about 130
+            // cycles (its result decides a branch); a non-blocking test for the NEXT unit, issued before the rounds of
+            // the current one, costs nothing when the producer is ahead, which it is after the slice's first units.
+            // The fast loop runs while that test succeeds; when it fails the blocking wait outside takes over.
+            uint32_t units_left = 5u * n_total;
+            int u5 = 0;
+            while (units_left != 0) {
+                if (!tma::mbar_wait_bounded_sleepy(bar_full + 8 * wslot, fparity)) { failed = true; break; }     // uniform: one barrier word
+                bool there;
 #pragma unroll 1
-                for (int u = 0; u < 5; ++u) {
-                    failed = !tma::mbar_wait_bounded_sleepy(bar_full + 8 * wslot, fparity);     // uniform: one barrier word
-                    if (failed) break;
+                do {
                     const uint32_t src = wk_ring + wslot * kUnitBytes;
                     uint64_t kw[16];
 #pragma unroll
@@ -260,13 +266,18 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
                     }
                     tma::mbar_arrive(bar_empty + 8 * wslot);   // every lane arrives once its own values are in registers
                     if (++wslot == NSLOT) { wslot = 0; fparity ^= 1u; }
+                    --units_left;
+                    there = units_left != 0 && tma::mbar_test_wait(bar_full + 8 * wslot, fparity);
                     rounds16_512(v, kw);
-                }
+                    if (++u5 == 5) {
+                        u5 = 0;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    st[k] += v[k];
-                    v[k] = st[k];
-                }
+                        for (int k = 0; k < 8; ++k) {
+                            st[k] += v[k];
+                            v[k] = st[k];
+                        }
+                    }
+                } while (there);
             }
             if (failed) {
                 if (lane == 0) atomicExch(&s_failed[pair], 1u);
@@ -290,9 +301,9 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
 }
 
 // Slices of at least 16 KiB, at most 256 per chunk, a multiple of 4 KiB, counted over the whole 128-byte blocks.
-void sha512_slices(uint64_t chunk_bytes, uint64_t *slice_bytes, uint64_t *per_group) {
+void sha512_slices(uint64_t chunk_bytes, uint64_t max_slices, uint64_t *slice_bytes, uint64_t *per_group) {
     uint64_t slices = chunk_bytes / 16384;
-    if (slices > 256) slices = 256;
+    if (slices > max_slices) slices = max_slices;
     if (slices < 1) slices = 1;
     uint64_t sb = (chunk_bytes + slices - 1) / slices;
     sb = (sb + 4095) & ~4095ull;
@@ -311,8 +322,10 @@ cudaError_t launch_pairs(const CUtensorMap &map, const uint8_t *d_data, uint64_t
     static bool configured[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, per_group = 0;
-    sha512_slices(chunk_bytes, &slice_bytes, &per_group);
-    const uint64_t groups = (whole + 31) / 32, total_tasks = groups * per_group;
+    const uint64_t groups = (whole + 31) / 32;
+    // a group per SM or fewer: every group keeps one pair for the whole launch, there is nothing to balance
+    sha512_slices(chunk_bytes, groups <= (uint64_t)sm_count ? 1 : 256, &slice_bytes, &per_group);
+    const uint64_t total_tasks = groups * per_group;
     uint8_t *base = static_cast<uint8_t *>(d_scratch);
     SliceQueue *q = reinterpret_cast<SliceQueue *>(base);
     uint64_t *mid = reinterpret_cast<uint64_t *>(base + 64);                       // 2 KiB per group
@@ -328,7 +341,7 @@ cudaError_t launch_pairs(const CUtensorMap &map, const uint8_t *d_data, uint64_t
 
 }  // namespace
 
-// Measured on 148 SMs (GB/s of SHA-384, G groups of 32 chains, chunks of 64 KiB to 4 MiB): the pairs give 1.36 per
+// Measured on 148 SMs (GB/s of SHA-384, G groups of 32 chains, chunks of 64 KiB to 4 MiB): the pairs give 1.5 per
 // group up to G = 148 and 600 to 614 from G = 896 on (91 % of the integer roofline); the plain kernel, one warp per
 // group, gives 0.9 per group up to G = 592 (every warp alone on its scheduler: ahead of the pairs between three and
 // four groups per SM, where the pairs already share schedulers), falls back behind 592 and reaches 650 to 660 from
@@ -345,7 +358,7 @@ bool sha512_wants_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_b
 
 uint64_t sha512_pairs_scratch_bytes(uint64_t nbytes, uint64_t chunk_bytes) {
     uint64_t slice_bytes = 0, per_group = 0;
-    sha512_slices(chunk_bytes, &slice_bytes, &per_group);
+    sha512_slices(chunk_bytes, 256, &slice_bytes, &per_group);
     const uint64_t groups = (nbytes / chunk_bytes + 31) / 32;
     return 64 + 2048 * groups + 4 * groups * per_group + 4 * groups + 256;
 }
