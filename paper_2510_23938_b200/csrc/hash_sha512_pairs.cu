@@ -86,7 +86,8 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u;
     const bool producer = warp < PAIRS;
-    const uint32_t pair = producer ? warp : warp - PAIRS;
+    // the two warps of a pair sit on different schedulers (warp w runs on scheduler w mod 4)
+    const uint32_t pair = producer ? warp : (PAIRS % 4 == 0 ? (warp - PAIRS + PAIRS - 1) % PAIRS : warp - PAIRS);
     // tiled boxes must start on a 1024-byte boundary (the swizzle pattern repeats every 8 rows)
     const uint32_t smem0 = (tma::smem_u32(smem) + 1023u) & ~1023u;
     const uint32_t data_ring = smem0 + pair * (STAGES * kBoxBytes);
@@ -313,10 +314,9 @@ void sha512_slices(uint64_t chunk_bytes, uint64_t max_slices, uint64_t *slice_by
     *per_group = pg;
 }
 
-template <int DIGEST_WORDS>
+template <int PAIRS, int STAGES, int NSLOT, int DIGEST_WORDS>
 cudaError_t launch_pairs(const CUtensorMap &map, const uint8_t *d_data, uint64_t chunk_bytes, uint64_t whole,
                          uint8_t *d_digests, uint32_t *d_status, void *d_scratch, int sm_count, cudaStream_t stream) {
-    constexpr int PAIRS = 6, STAGES = 3, NSLOT = 5;
     constexpr size_t smem = 1024 + (size_t)PAIRS * (STAGES * kBoxBytes + NSLOT * kUnitBytes);
     auto kernel = hash_sha512_pairs_kernel<PAIRS, STAGES, NSLOT, DIGEST_WORDS>;
     static bool configured[kMaxDevices] = {};
@@ -375,8 +375,16 @@ cudaError_t launch_hash_sha512_pairs(const uint8_t *d_data, uint64_t nbytes, uin
     if (whole == 0 || !make_chunk_tensor_map(&map, d_data, chunk_bytes, whole)) return cudaSuccess;
     *covered = whole;
     if (launches) *launches += 2;
-    return digest_words == 6 ? launch_pairs<6>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream)
-                             : launch_pairs<8>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream);
+    // Six pairs per SM (three warps per scheduler, two schedulers with two producers and a consumer, two with one
+    // and two) up to eight groups per SM; from there eight pairs with shorter rings (four warps per scheduler, two
+    // of each kind on every one: 624 to 638 GB/s of SHA-384 from 1,280 groups on against 597 to 610), which with
+    // fewer groups than pairs would leave the SMs unevenly filled.
+    const bool eight = (whole + 31) / 32 >= 8ull * (uint64_t)sm_count;
+    if (digest_words == 6)
+        return eight ? launch_pairs<8, 2, 4, 6>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream)
+                     : launch_pairs<6, 3, 5, 6>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream);
+    return eight ? launch_pairs<8, 2, 4, 8>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream)
+                 : launch_pairs<6, 3, 5, 8>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream);
 }
 
 }  // namespace ivk

@@ -67,6 +67,8 @@ VARIANTS = [_Variant("sha384", 48), _Variant("sha512", 64)]
     (32 * 16384, 16384), (16384, 16384), (33 * 16384, 16384), (30_000 * 16384, 16384), (40 * (1 << 20), 1 << 20),
     (36 * (4 << 20) + 4096, 4 << 20), (70 * (20480 + 48), 20480 + 48), (150 * (5 * 16384 - 128), 5 * 16384 - 128),
     (500 * 32 * 16384, 16384), (4096 * 32 * 16384, 16384),       # group counts the plain kernel keeps
+    # eight groups per SM and more: the instance with eight pairs per SM (1,250 / 1,300 / 2,000 groups on 148 SMs)
+    (40_000 * 16384 + 4096, 16384), (41_600 * 65536, 65536), (64_000 * (16384 + 48), 16384 + 48),
 ])
 @pytest.mark.parametrize("variant", VARIANTS, ids=repr)
 def test_hash_chunks_equals_oracle(ctx, variant, nbytes, chunk):
