@@ -314,6 +314,8 @@ void sha512_slices(uint64_t chunk_bytes, uint64_t max_slices, uint64_t *slice_by
     *per_group = pg;
 }
 
+thread_local const char *t_pairs_instance = "";     // which instance the calling thread's last launch used
+
 template <int PAIRS, int STAGES, int NSLOT, int DIGEST_WORDS>
 cudaError_t launch_pairs(const CUtensorMap &map, const uint8_t *d_data, uint64_t chunk_bytes, uint64_t whole,
                          uint8_t *d_digests, uint32_t *d_status, void *d_scratch, int sm_count, cudaStream_t stream) {
@@ -340,6 +342,8 @@ cudaError_t launch_pairs(const CUtensorMap &map, const uint8_t *d_data, uint64_t
 }
 
 }  // namespace
+
+const char *sha512_pairs_instance_name() { return t_pairs_instance; }
 
 // Measured on 148 SMs (GB/s of SHA-384, G groups of 32 chains, chunks of 64 KiB to 4 MiB): the pairs give 1.5 per
 // group up to G = 148 and 600 to 614 from G = 896 on (91 % of the integer roofline); the plain kernel, one warp per
@@ -380,6 +384,7 @@ cudaError_t launch_hash_sha512_pairs(const uint8_t *d_data, uint64_t nbytes, uin
     // of each kind on every one: 624 to 638 GB/s of SHA-384 from 1,280 groups on against 597 to 610), which with
     // fewer groups than pairs would leave the SMs unevenly filled.
     const bool eight = (whole + 31) / 32 >= 8ull * (uint64_t)sm_count;
+    t_pairs_instance = eight ? "8 pairs per SM" : ((whole + 31) / 32 <= (uint64_t)sm_count ? "6 pairs per SM, one slice per chunk" : "6 pairs per SM");
     if (digest_words == 6)
         return eight ? launch_pairs<8, 2, 4, 6>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream)
                      : launch_pairs<6, 3, 5, 6>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream);

@@ -218,7 +218,7 @@ int hash_leaves_wide(iv_ctx *ctx, const uint8_t *d_data, uint64_t nbytes, uint64
                                                ctx->d_status, scratch, stream, &ctx->launches, &ctx->leaf_kernel,
                                                fork ? ctx->tail_stream : nullptr));
     if (fork && (rc = join_tail_stream(ctx, stream)) != IV_OK) return rc;
-    ctx->leaf_instance = "";
+    ctx->leaf_instance = std::strcmp(ctx->leaf_kernel, "hash_sha512_pairs_kernel") == 0 ? ivk::sha512_pairs_instance_name() : "";
     return IV_OK;
 }
 

@@ -170,6 +170,7 @@ cudaError_t launch_merkle_root_sha384(const uint8_t *d_leaves, uint64_t n, uint8
 // 16-byte aligned blobs with at least one whole chunk of 16 KiB or more (a multiple of 16 bytes), at group counts
 // where the two-warp kernel is the faster one.
 bool sha512_wants_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, int sm_count);
+const char *sha512_pairs_instance_name();     // launch shape of the calling thread's last two-warp launch
 uint64_t sha512_pairs_scratch_bytes(uint64_t nbytes, uint64_t chunk_bytes);
 // Hashes the blob's whole chunks (*covered of them, from the front; 0 and nothing launched if the blob cannot be
 // described to the TMA unit); a short last chunk is left to the caller.

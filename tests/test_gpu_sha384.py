@@ -78,8 +78,11 @@ def test_hash_chunks_equals_oracle(ctx, variant, nbytes, chunk):
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     if chunk >= 16384 and chunk % 16 == 0 and nbytes >= chunk and groups < 4096 and not (3 * sms <= groups <= 4 * sms):
         assert ctx.last_leaf_kernel == "hash_sha512_pairs_kernel"
+        want_instance = "8 pairs per SM" if groups >= 8 * sms else ("6 pairs per SM, one slice per chunk" if groups <= sms else "6 pairs per SM")
+        assert ctx.last_leaf_instance == want_instance
     else:
         assert ctx.last_leaf_kernel == "hash_chunks_sha384_kernel"
+        assert ctx.last_leaf_instance == ""
     want = variant.cpu_chunks(_host(data), chunk, nthreads=oracle.host_threads())
     assert got.shape == want.shape
     assert np.array_equal(_host(got), want)
