@@ -20,10 +20,11 @@
 // over a block's five units stay rolled: the producers and consumers of twelve warps run different code at the
 // same time, and unrolled it no longer fits the instruction cache (218 GB/s against 521 at the time).
 //
-// A CTA holds PAIRS pairs (producer warps 0..PAIRS-1, consumer warps PAIRS..2 PAIRS-1; with six pairs every SM
-// scheduler hosts three warps, and producers and consumers are spread so that the schedulers' loads differ by
-// a twelfth).  One persistent CTA per SM; pair 0 of every CTA takes tickets as they come, the other pairs take a
-// task only when one lies in the FIFO unclaimed, so that few groups spread one per SM.  All waits are bounded.
+// A CTA holds PAIRS pairs (producer warps 0..PAIRS-1, consumer warps PAIRS..2 PAIRS-1, a pair's two warps on
+// different schedulers); the launch picks two, four, six or eight pairs by the groups per SM
+// (sha512_pairs_per_sm).  One persistent CTA per SM; pair 0 of every CTA takes tickets as they come, the other
+// pairs take a task only when one lies in the FIFO unclaimed, the later ones of a CTA later and less often, so
+// that few groups spread one per SM.  All waits are bounded.
 #include <cstring>
 
 #include "chunk_tensor_map.h"
@@ -129,7 +130,7 @@ hash_sha512_pairs_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t
                     task = kTaskFailed;
                 } else {
                     const unsigned long long t = pair == 0 ? atomicAdd(&q->head, 1ull)
-                                                           : take_leftover_ticket(q, total_tasks, first_take);
+                                                           : take_leftover_ticket(q, total_tasks, first_take, pair - 1u);
                     if (t < total_tasks) {
                         // With few groups a ticket can lie many slices ahead of the pushes; the wait gives up only
                         // when the FIFO has not moved for about four seconds.
@@ -345,18 +346,32 @@ cudaError_t launch_pairs(const CUtensorMap &map, const uint8_t *d_data, uint64_t
 
 const char *sha512_pairs_instance_name() { return t_pairs_instance; }
 
-// Measured on 148 SMs (GB/s of SHA-384, G groups of 32 chains, chunks of 64 KiB to 4 MiB): the pairs give 1.5 per
-// group up to G = 148 and 600 to 614 from G = 896 on (91 % of the integer roofline); the plain kernel, one warp per
-// group, gives 0.9 per group up to G = 592 (every warp alone on its scheduler: ahead of the pairs between three and
-// four groups per SM, where the pairs already share schedulers), falls back behind 592 and reaches 650 to 660 from
-// about 4,096 groups on (six and more warps per scheduler), where the pairs stay at 590.
+// Which launches the two-warp kernel takes and with how many pairs per SM.  Measured on 148 SMs (GB/s of SHA-384, G
+// groups of 32 chains, S SMs; "plain" is the one-chain-per-lane kernel of hash_sha384.cu):
+//   * pairs a CTA does not need cost the working ones a fifth of their speed (their warps poll and share schedulers
+//     in no fixed order), so the pair count follows the groups per SM: two pairs below 3 S groups (1.5 GB/s per
+//     group up to 2 S: 256 groups of 256 KiB chunks 375 against 273 with six pairs), four from there (each scheduler
+//     one producer and one consumer: 445 to 577 between 3 S and 4 S, where the plain kernel gives 399 to 533, and
+//     580 to 590 up to 6 S against 470 to 580 with six), six from 6 S for chunks of 1 MiB and more (612 against 604 on
+//     896 groups of 4 MiB), eight from 8 S (two producers and two consumers per scheduler: 620 to 646);
+//   * short chunks are short tasks: below 64 KiB the plain kernel is ahead from 3 S groups on (16 KiB chunks: 500
+//     against 359 at 592 groups, 548 against 496 at 2,048), below 256 KiB from 4,096 groups on (64 KiB chunks: 635
+//     against 610 at 4,000); from 256 KiB the pairs stay ahead at every count (641 against 598 at 4,800 groups).
+int sha512_pairs_per_sm(uint64_t groups, uint64_t chunk_bytes, int sm_count) {
+    const uint64_t s = (uint64_t)sm_count;
+    if (groups < 3 * s) return 2;
+    if (groups >= 8 * s && (chunk_bytes >= (128u << 10) || groups >= 14 * s)) return 8;
+    if (groups >= 6 * s && chunk_bytes >= (1u << 20)) return 6;
+    return 4;
+}
+
 bool sha512_wants_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, int sm_count) {
     if ((reinterpret_cast<uintptr_t>(d_data) & 15u) != 0 || chunk_bytes % 16u != 0 || chunk_bytes < 16384 ||
         chunk_bytes >= (1ull << 31) || nbytes < chunk_bytes)
         return false;
     const uint64_t groups = (nbytes / chunk_bytes + 31) / 32;
-    if (groups >= 4096) return false;
-    if (groups >= 3ull * (uint64_t)sm_count && groups <= 4ull * (uint64_t)sm_count) return false;
+    if (chunk_bytes < (64u << 10)) return groups < 3ull * (uint64_t)sm_count;
+    if (chunk_bytes < (256u << 10)) return groups < 4096;
     return true;
 }
 
@@ -379,17 +394,18 @@ cudaError_t launch_hash_sha512_pairs(const uint8_t *d_data, uint64_t nbytes, uin
     if (whole == 0 || !make_chunk_tensor_map(&map, d_data, chunk_bytes, whole)) return cudaSuccess;
     *covered = whole;
     if (launches) *launches += 2;
-    // Six pairs per SM (three warps per scheduler, two schedulers with two producers and a consumer, two with one
-    // and two) up to eight groups per SM; from there eight pairs with shorter rings (four warps per scheduler, two
-    // of each kind on every one: 624 to 638 GB/s of SHA-384 from 1,280 groups on against 597 to 610), which with
-    // fewer groups than pairs would leave the SMs unevenly filled.
-    const bool eight = (whole + 31) / 32 >= 8ull * (uint64_t)sm_count;
-    t_pairs_instance = eight ? "8 pairs per SM" : ((whole + 31) / 32 <= (uint64_t)sm_count ? "6 pairs per SM, one slice per chunk" : "6 pairs per SM");
-    if (digest_words == 6)
-        return eight ? launch_pairs<8, 2, 4, 6>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream)
-                     : launch_pairs<6, 3, 5, 6>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream);
-    return eight ? launch_pairs<8, 2, 4, 8>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream)
-                 : launch_pairs<6, 3, 5, 8>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream);
+    const int pairs = sha512_pairs_per_sm((whole + 31) / 32, chunk_bytes, sm_count);
+    t_pairs_instance = pairs == 8 ? "8 pairs per SM" : pairs == 6 ? "6 pairs per SM" : pairs == 4 ? "4 pairs per SM" : "2 pairs per SM";
+#define IV_GO(P, S, N)                                                                                                           \
+    (digest_words == 6 ? launch_pairs<P, S, N, 6>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream) \
+                       : launch_pairs<P, S, N, 8>(map, d_data, chunk_bytes, whole, d_digests, d_status, d_scratch, sm_count, stream))
+    switch (pairs) {
+        case 8: return IV_GO(8, 2, 4);
+        case 6: return IV_GO(6, 3, 5);
+        case 4: return IV_GO(4, 3, 5);
+        default: return IV_GO(2, 3, 5);
+    }
+#undef IV_GO
 }
 
 }  // namespace ivk

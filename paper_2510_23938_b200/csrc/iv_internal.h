@@ -168,8 +168,10 @@ cudaError_t launch_merkle_root_sha384(const uint8_t *d_leaves, uint64_t n, uint8
 
 // hash_sha512_pairs.cu ------------------------------------------------------
 // 16-byte aligned blobs with at least one whole chunk of 16 KiB or more (a multiple of 16 bytes), at group counts
-// where the two-warp kernel is the faster one.
+// where the two-warp kernel is the faster one; sha512_pairs_per_sm is the number of producer/consumer pairs per
+// SM it then runs with (2, 4, 6 or 8).
 bool sha512_wants_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, int sm_count);
+int sha512_pairs_per_sm(uint64_t groups, uint64_t chunk_bytes, int sm_count);
 const char *sha512_pairs_instance_name();     // launch shape of the calling thread's last two-warp launch
 uint64_t sha512_pairs_scratch_bytes(uint64_t nbytes, uint64_t chunk_bytes);
 // Hashes the blob's whole chunks (*covered of them, from the front; 0 and nothing launched if the blob cannot be

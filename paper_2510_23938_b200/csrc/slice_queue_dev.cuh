@@ -37,9 +37,12 @@ __device__ __forceinline__ void st_release_u32(uint32_t *p, uint32_t v) {
 // groups.  With nothing left over it polls; giving up (the return value total_tasks ends the
 // worker) is harmless, the first workers finish the launch.  Kept out of line so that the hashing
 // loop's register allocation does not depend on it.
+// `rank` orders the leftover workers of a CTA (0 = the first of them): a higher rank starts later and polls less
+// often, so that unclaimed work goes to the CTAs with the fewest busy workers first.
 __device__ __noinline__ unsigned long long take_leftover_ticket(SliceQueue *q, unsigned long long total_tasks,
-                                                                bool first_take) {
-    if (first_take) __nanosleep(20000);      // at launch, let the first workers of every CTA claim their groups
+                                                                bool first_take, unsigned rank = 0) {
+    if (first_take) __nanosleep(20000u + 5000u * rank);      // at launch, let the first workers of every CTA claim their groups
+    const unsigned poll_ns = 256u << (rank < 4u ? rank : 4u);
     const long long t0 = clock64();
     for (;;) {
         const unsigned long long h = *reinterpret_cast<volatile unsigned long long *>(&q->head);
@@ -50,7 +53,7 @@ __device__ __noinline__ unsigned long long take_leftover_ticket(SliceQueue *q, u
             continue;
         }
         if (clock64() - t0 > 8000000000ll) return total_tasks;
-        __nanosleep(256);
+        __nanosleep(poll_ns);
     }
 }
 

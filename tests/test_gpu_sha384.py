@@ -67,8 +67,11 @@ VARIANTS = [_Variant("sha384", 48), _Variant("sha512", 64)]
     (32 * 16384, 16384), (16384, 16384), (33 * 16384, 16384), (30_000 * 16384, 16384), (40 * (1 << 20), 1 << 20),
     (36 * (4 << 20) + 4096, 4 << 20), (70 * (20480 + 48), 20480 + 48), (150 * (5 * 16384 - 128), 5 * 16384 - 128),
     (500 * 32 * 16384, 16384), (4096 * 32 * 16384, 16384),       # group counts the plain kernel keeps
-    # eight groups per SM and more: the instance with eight pairs per SM (1,250 / 1,300 / 2,000 groups on 148 SMs)
-    (40_000 * 16384 + 4096, 16384), (41_600 * 65536, 65536), (64_000 * (16384 + 48), 16384 + 48),
+    # the launch shapes of the two-warp kernel on 148 SMs: eight pairs per SM (1,200 groups of 128 KiB chunks; 2,075
+    # groups of 64 KiB chunks), four (1,300 and 625 groups), two (below 444 groups: most shapes above); chunks
+    # below 64 KiB with many groups go to the plain kernel
+    (38_400 * 131072, 131072), (66_400 * 65536, 65536), (41_600 * 65536, 65536), (20_000 * (65536 + 48), 65536 + 48),
+    (64_000 * (16384 + 48), 16384 + 48),
 ])
 @pytest.mark.parametrize("variant", VARIANTS, ids=repr)
 def test_hash_chunks_equals_oracle(ctx, variant, nbytes, chunk):
@@ -76,10 +79,13 @@ def test_hash_chunks_equals_oracle(ctx, variant, nbytes, chunk):
     got = variant.gpu_chunks(ctx, data, chunk)
     groups = -(-(nbytes // chunk) // 32)
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    if chunk >= 16384 and chunk % 16 == 0 and nbytes >= chunk and groups < 4096 and not (3 * sms <= groups <= 4 * sms):
+    pairs_take_it = chunk >= 16384 and chunk % 16 == 0 and nbytes >= chunk and (
+        groups < 3 * sms if chunk < 65536 else groups < 4096 if chunk < 262144 else True)
+    if pairs_take_it:
         assert ctx.last_leaf_kernel == "hash_sha512_pairs_kernel"
-        want_instance = "8 pairs per SM" if groups >= 8 * sms else ("6 pairs per SM, one slice per chunk" if groups <= sms else "6 pairs per SM")
-        assert ctx.last_leaf_instance == want_instance
+        pairs = (2 if groups < 3 * sms else 8 if groups >= 8 * sms and (chunk >= 131072 or groups >= 14 * sms)
+                 else 6 if groups >= 6 * sms and chunk >= (1 << 20) else 4)
+        assert ctx.last_leaf_instance == f"{pairs} pairs per SM"
     else:
         assert ctx.last_leaf_kernel == "hash_chunks_sha384_kernel"
         assert ctx.last_leaf_instance == ""
