@@ -3,8 +3,8 @@
 //
 // One warp carries 32 chains (a "group"); a chunk is one serial chain of 128-byte blocks (FIPS 180-4
 // section 6.4).  The 64-bit additions and rotations are pairs of 32-bit instructions with carry and funnel
-// dependencies, so one warp alone leaves most issue slots of its SM scheduler empty, and with few groups
-// per scheduler the launch is bound by latency, not by the integer pipe.  As on the SHA-256 path the
+// dependencies, so one warp alone issues an instruction every 2.5 cycles, and with few groups the launch is
+// bound by what one warp can issue, not by the SM's integer pipes.  As on the SHA-256 path the
 // message schedule, the endian swap and the round-constant additions (44 % of the work) do not depend on
 // the chaining value, so a group is served by a PAIR of warps:
 //
@@ -17,7 +17,7 @@
 //
 // The three-input boolean functions and the rotations are written on 32-bit halves (sha512_dev.cuh); left to
 // the compiler's 64-bit code the same kernel ran at 78 % instead of 91 % of the integer roofline.  The loops
-// over a block's five units stay rolled: the producers and consumers of twelve warps run different code at the
+// over a block's five units stay rolled: the producers and consumers of up to sixteen warps run different code at the
 // same time, and unrolled it no longer fits the instruction cache (218 GB/s against 521 at the time).
 //
 // A CTA holds PAIRS pairs (producer warps 0..PAIRS-1, consumer warps PAIRS..2 PAIRS-1, a pair's two warps on
