@@ -117,6 +117,34 @@ def test_sha384_and_sha512_two_warp_kernel_on_random_shapes(ctx):
     assert ctx.device_status() == 0
 
 
+def test_sha384_and_sha512_two_warp_kernel_with_many_groups(ctx):
+    """Random shapes with three and more groups of 32 chains per SM, where the two-warp kernel runs four or eight
+    pairs per SM (or hands short chunks to the one-chain-per-lane kernel): chunks of 16 KiB to 192 KiB (multiples of
+    16 bytes), a ragged last group, a short last chunk half of the time, a base that is shifted by 16-byte steps."""
+    rng = np.random.default_rng(513)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    buf = inputs.uniform_bytes((2 << 30) + 1024, seed=513, device="cuda")
+    seen = set()
+    for k in range(8):
+        chunk = 16 * int(rng.integers(1024, 12_288))
+        groups = int(rng.integers(3 * sms + 1, 17 * sms))
+        n_chunks = groups * 32 - int(rng.integers(0, 32))
+        while chunk * n_chunks > (2 << 30):
+            n_chunks = n_chunks * 3 // 4
+        tail = int(rng.integers(1, chunk + 1)) if k % 2 else chunk
+        nbytes = (n_chunks - 1) * chunk + tail
+        shift = 16 * int(rng.integers(0, 64))
+        data = buf[shift:shift + nbytes]
+        host = _host(data)
+        got = ctx.hash_chunks_sha384(data, chunk)
+        seen.add(ctx.last_leaf_kernel + " " + ctx.last_leaf_instance)
+        assert np.array_equal(_host(got), oracle.hash_chunks_sha384(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk, shift)
+        got = ctx.hash_chunks_sha512(data, chunk)
+        assert np.array_equal(_host(got), oracle.hash_chunks_sha512(host, chunk, nthreads=oracle.host_threads())), (nbytes, chunk, shift)
+    assert "hash_sha512_pairs_kernel 4 pairs per SM" in seen, seen
+    assert ctx.device_status() == 0
+
+
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_random_tensor_sets(ctx, seed):
     rng = np.random.default_rng(1000 + seed)
