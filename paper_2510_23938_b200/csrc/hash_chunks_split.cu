@@ -6,7 +6,7 @@
 // chaining state.  Each CTA therefore runs two warps on two SM schedulers for its 32 chains:
 //
 //   producer warp: pulls the lanes' streams through a shared-memory ring with bulk copies
-//                  (as the staged kernel does), forms W[t] + K[t] for t = 0..63 of every block
+//                  (one per lane and segment), forms W[t] + K[t] for t = 0..63 of every block
 //                  and writes them to a second ring, lane-interleaved;
 //   consumer warp: runs only the 64 rounds, reading W[t] + K[t] with 128-bit shared loads.
 //

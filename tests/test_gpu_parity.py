@@ -37,7 +37,7 @@ def _root_bytes(t: torch.Tensor) -> bytes:
     (100_003, 1000), (100_003, 1001), (100_003, 7), (65, 64), (64, 64), (63, 64), (1, 1), (1, 4096),
     (5 * 4096 + 56, 4096), (5 * 4096 + 55, 4096), (5 * 4096 + 119, 4096), (5 * 4096 + 120, 4096),
     (37 * 48 + 16, 48),              # chunk size multiple of 16 but not 64
-    (50 * (4096 + 16) + 8, 4096 + 16),   # staged path with a 16-byte remainder in every chunk
+    (50 * (4096 + 16) + 8, 4096 + 16),   # bulk-copy path with a 16-byte remainder in every chunk
     (33 * 8192 + 4100, 8192), (3 * 65536 + 300, 65536 + 48),
     (20_000 * 4096 + 100, 4096),     # more than 592 warps: the many-chain launch shape, ragged last chunk
     (19_000 * 4096, 4096),    (60_000 * 4096 + 100, 4096), (57_000 * 16384, 16384),   # 12 or more groups per SM: the twelve-worker instance

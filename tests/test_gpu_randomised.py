@@ -35,7 +35,7 @@ def _cases(seed, count):
             chunk = 16 * int(rng.integers(1, 5_000))
         elif kind == 2:    # multiple of 64
             chunk = 64 * int(rng.integers(1, 2_000))
-        elif kind == 3:    # multiple of 4096 (the staged, two-warp and migrating kernels)
+        elif kind == 3:    # multiple of 4096 (the two-warp and migrating kernels)
             chunk = 4096 * int(rng.integers(1, 40))
         else:              # small chunks, many chains
             chunk = int(rng.integers(1, 300))
