@@ -12,6 +12,8 @@
 //
 // The two rings are handed over through mbarriers (full / empty per slot); all waits are bounded.
 // The chain's critical path per block drops from the whole compression to the rounds alone.
+#include <type_traits>
+
 #include "iv_internal.h"
 #include "rfc6962_dev.cuh"
 #include "sha256_dev.cuh"
@@ -34,18 +36,26 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
 // RAGGED = true:  message k of the CTA is tensor order[...] at data + offsets[.] with lengths[.] bytes,
 //                 any alignment: each bulk copy starts at the 16-byte boundary below the tensor and
 //                 carries 16 bytes more than a segment, so that every 64-byte block lies inside one
-//                 stage; the block is read as 17 aligned words and the byte shift is folded into the
-//                 endian-swap PRMT.
-// PAIR: blocks handed over per W+K slot (1 or 2); with 2 the barrier traffic per block halves.
+//                 stage.  A block is read as five aligned 16-byte pieces (conflict-free at this lane stride,
+//                 whatever the tensors' alignment; 17 scalar loads at the same stride collided up to
+//                 eight ways and cost the CHAIN up to 11 %, because the shared-memory pipe is the
+//                 consumer's too); the 0..3 whole words between the 16-byte boundary and the message are
+//                 skipped with two levels of selects, the last 0..3 bytes in the endian-swap PRMT.
+// PAIR: blocks handed over per W+K slot; the barrier traffic per block falls with it.
 // PREFIX (chunks only): message i is 0x00 || chunk i, the RFC 6962 leaf hash.
-template <int SEG, int STAGES, int NSLOT, bool RAGGED, int PAIR = 1, bool PREFIX = false>
-__global__ void __launch_bounds__(64)
+// MINB, NARROW: the second argument of __launch_bounds__ (0 = none) and 32-bit block counters in the
+//                 consumer.  Neither changes what is computed; they change the code the compiler makes of
+//                 the consumer's loop, which decides the chain's speed and came out 1,845 to 2,130 cycles
+//                 per block over the combinations tried.  The launcher passes the best one measured for
+//                 each mode (tensors: 1, true; chunks: 0, false).
+template <int SEG, int STAGES, int NSLOT, bool RAGGED, int PAIR = 1, bool PREFIX = false, int MINB = 0, bool NARROW = false>
+__global__ void __launch_bounds__(64, MINB)
 hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                          uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
                          const uint32_t *__restrict__ one_ptr, const uint64_t *__restrict__ offsets,
                          const uint64_t *__restrict__ lengths, const uint32_t *__restrict__ order,
                          iv_sha_state *__restrict__ states, int finish) {
-    constexpr uint32_t kLaneStride = SEG + (RAGGED ? 32 : 16);   // data ring: bytes per lane per stage
+    constexpr uint32_t kLaneStride = SEG + 16;            // data ring: bytes per lane per stage (33 or 65 x 16: conflict-free)
     constexpr uint32_t kStageBytes = 32 * kLaneStride;
     constexpr int kBlocksPerSeg = SEG / 64;
     constexpr uint32_t kWkLane = 64 * 4 + 16;             // W+K ring: bytes per lane per slot
@@ -105,6 +115,11 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     const uint64_t my_total = !valid ? 0 : (finishing ? ((len + (PREFIX ? 1 : 0) + 8) >> 6) + 1 : (len >> 6));
     const uint64_t warp_total = RAGGED ? warp_max_u64(my_total) : __shfl_sync(0xffffffffu, my_total, 0);
 
+    if (NARROW && warp_total > 0xffffffffull) {       // a message of 2^32 blocks (256 GiB) does not fit the device's memory
+        if (lane == 0) atomicExch(status, (uint32_t)IVK_DEV_BOUNDS);
+        return;                                        // both warps leave: nobody waits for the other
+    }
+
     if (warp == 1) {
         // ------------------------------------------------------------------ producer
         const uint8_t *p = data + begin;
@@ -117,7 +132,7 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
         const uint32_t mis = RAGGED ? (uint32_t)(reinterpret_cast<uintptr_t>(p) & 15u) : 0u;
         const uint8_t *p_al = p - mis;
         const uint64_t need = full_bytes ? ((mis + full_bytes + 15) & ~15ull) : 0;
-        const uint32_t word_off = mis & ~3u;                       // in-stage offset of the first aligned word
+        const bool skip1 = (mis & 4u) != 0, skip2 = (mis & 8u) != 0;   // whole words between the 16-byte boundary and the message
         const uint32_t sel = 0x0123u + 0x1111u * (mis & 3u);       // PRMT: byte shift + big-endian
         // One arrival per stage: lane 0 announces the bytes of all 32 copies, every lane issues its own.
         auto issue = [&](uint64_t seg, int stage) {
@@ -134,22 +149,16 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
         for (int s = 0; s < STAGES; ++s)
             if ((uint64_t)s < nseg) issue(s, s);
 
-        uint32_t w[16], raw[17], tw[32];
+        uint32_t w[16], raw[RAGGED ? 20 : 16], tw[32];
         uint32_t carry = 0u;                          // PREFIX: the data word before the block (byte 3 of 0 = the prefix)
         int stage = 0, in_stage = 0;
         uint32_t dparity = 0;
         bool failed = false, tail_built = false;
         auto fetch = [&](int blk_in_stage) {
             const uint32_t src = data_base + stage * kStageBytes + 64 * blk_in_stage;
-            if (RAGGED) {
 #pragma unroll
-                for (int q = 0; q < 17; ++q)
-                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(raw[q]) : "r"(src + word_off + 4 * q) : "memory");
-            } else {
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    tma::ld_shared_v4(src + 16 * q, raw[4 * q], raw[4 * q + 1], raw[4 * q + 2], raw[4 * q + 3]);
-            }
+            for (int q = 0; q < (RAGGED ? 5 : 4); ++q)
+                tma::ld_shared_v4(src + 16 * q, raw[4 * q], raw[4 * q + 1], raw[4 * q + 2], raw[4 * q + 3]);
         };
         if (warp_full) {
             failed = !__all_sync(0xffffffffu, tma::mbar_wait_bounded(bar_data, 0));
@@ -160,14 +169,22 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
         uint32_t eparity = 1;                         // first pass over the slots finds them empty
         for (uint64_t blk = 0; blk < warp_total && !failed; ++blk) {
             if (blk < my_full) {
-                if (PREFIX) {
+                if constexpr (PREFIX) {
                     w[0] = shifted_word(raw[0], carry);
 #pragma unroll
                     for (int k = 1; k < 16; ++k) w[k] = shifted_word(raw[k], raw[k - 1]);
                     carry = raw[15];
+                } else if constexpr (RAGGED) {
+                    uint32_t a[19], b[17];
+#pragma unroll
+                    for (int k = 0; k < 19; ++k) a[k] = skip1 ? raw[k + 1] : raw[k];
+#pragma unroll
+                    for (int k = 0; k < 17; ++k) b[k] = skip2 ? a[k + 2] : a[k];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) w[k] = __byte_perm(b[k], b[k + 1], sel);
                 } else {
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) w[k] = RAGGED ? __byte_perm(raw[k], raw[k + 1], sel) : bswap32(raw[k]);
+                    for (int k = 0; k < 16; ++k) w[k] = bswap32(raw[k]);
                 }
             } else if (blk < my_total) {
                 if (!tail_built) {
@@ -218,7 +235,10 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
     int slot = 0;
     uint32_t fparity = 0;
     bool failed = false;
-    for (uint64_t blk = 0; blk < warp_total; ++blk) {
+    // block counters of the loop: 64 bits, or 32 where the launcher asks (counts beyond 32 bits were refused above)
+    using Count = typename std::conditional<NARROW, uint32_t, uint64_t>::type;
+    const Count loop_total = (Count)warp_total, lane_total = (Count)my_total;
+    for (Count blk = 0; blk < loop_total; ++blk) {
         const uint32_t in_slot = (uint32_t)(blk % PAIR);
         if (in_slot == 0) {
             // every lane tests the same barrier word, so the outcome is uniform without a vote
@@ -226,11 +246,11 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
             if (failed) break;
         }
         const uint32_t src = wk_base + slot * kWkSlot + in_slot * kWkBlock;
-        const bool slot_done = in_slot == PAIR - 1 || blk + 1 == warp_total;
+        const bool slot_done = in_slot == PAIR - 1 || blk + 1 == loop_total;
         rounds64(v, src, one);
         if (slot_done) tma::mbar_arrive(bar_empty + 8 * slot);   // every lane arrives once its own values are in registers
         // feed-forward; a lane whose message has ended keeps its state (multiplier 0 instead of 1)
-        const uint32_t keep = (blk < my_total) ? one : 0u;
+        const uint32_t keep = (blk < lane_total) ? one : 0u;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             st[k] = padd<true>(v[k], st[k], keep);     // v * keep + st
@@ -255,16 +275,21 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
 namespace {
 
 // Two instances per mode.  Up to one group per SM a CTA may use most of an SM's shared memory: three W+K slots of
-// FOUR blocks each (156 KB; a hand-over every fourth block): 1,877 cycles per block.  Up to two groups per SM two
+// FOUR blocks each (a hand-over every fourth block): 1,877 cycles per block for chunks.  Up to two groups per SM two
 // CTAs share an SM: three slots of two blocks (104 KB): 1,916 cycles per block.  (Fetching the next block's first
 // W+K values during the last rounds of the current one, within a slot, was measured and does not pay: 1,890.)
+// The 32 bulk copies of a stage leave the producer one after the other and cost it about 2,000 cycles per stage.
+// With chunks the consumer is the slower warp either way; with tensors the producer has the selects on top and
+// was the slower one (1,970 cycles per block alone against 1,920 for the consumer), so where the CTA has an SM to
+// itself its stages are twice as long (two of 1,024 bytes per lane: 1,830 alone).
 template <bool RAGGED, bool PREFIX, int PAIR>
 cudaError_t launch_split_instance(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n, uint8_t *d_digests,
                                   uint32_t *d_status, const uint32_t *d_one, const uint64_t *d_offsets, const uint64_t *d_lengths,
                                   const uint32_t *d_order, iv_sha_state *d_states, int finish, cudaStream_t stream) {
-    constexpr int SEG = 512, STAGES = 3, NSLOT = 3;
-    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + (RAGGED ? 32 : 16)) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
-    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, RAGGED, PAIR, PREFIX>;
+    constexpr bool LONG_STAGES = RAGGED && PAIR == 4;
+    constexpr int SEG = LONG_STAGES ? 1024 : 512, STAGES = LONG_STAGES ? 2 : 3, NSLOT = 3;
+    constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
+    auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, RAGGED, PAIR, PREFIX, RAGGED ? 1 : 0, RAGGED>;
     static bool configured[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, smem, configured); e0 != cudaSuccess) return e0;
     const uint64_t blocks = (n + 31) / 32;
