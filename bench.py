@@ -52,11 +52,18 @@ PEAK_GBS = SM_COUNT * INT_LANES_PER_SM * SM_HZ / INT_OPS_PER_BYTE / 1e9
 # the round function (10 SHF/LOP3 per round on a 16-lane pipe, two cycles each).
 SPLIT_CYCLES_PER_BLOCK_ROOMY = 1877.0
 SPLIT_CYCLES_PER_BLOCK = 1916.0
+# the same kernel's instances for tensors (other launch-bounds hint, 32-bit block counters), as measured
+SPLIT_TENSOR_CYCLES_PER_BLOCK_ROOMY = 1845.0
+SPLIT_TENSOR_CYCLES_PER_BLOCK = 1910.0
 ISSUE_FLOOR_CYCLES_PER_BLOCK = 1280.0
 
 
 def split_cycles_per_block(chains: int) -> float:
     return SPLIT_CYCLES_PER_BLOCK_ROOMY if -(-chains // 32) <= SM_COUNT else SPLIT_CYCLES_PER_BLOCK
+
+
+def split_tensor_cycles_per_block(tensors: int) -> float:
+    return SPLIT_TENSOR_CYCLES_PER_BLOCK_ROOMY if -(-tensors // 32) <= SM_COUNT else SPLIT_TENSOR_CYCLES_PER_BLOCK
 
 
 # DRAM read+write bytes per byte hashed, from the ncu captures summarised under profiles/.
@@ -678,8 +685,10 @@ def measure_secondary(ctx, device, gpu_index, args):
     seconds = e0.elapsed_time(e1) * 1e-3
     c3["per_tensor"] = {"seconds": round(seconds, 3), "n_tensors": len(table), "bytes": int(lens.sum().item()),
                         "longest_bytes": longest, "leaf_kernel": ctx.last_leaf_kernel,
-                        "bound_seconds": round(longest / 64 * split_cycles_per_block(len(table)) / SM_HZ, 3),
+                        "cycles_per_block_measured": round(seconds * SM_HZ / (longest // 64 + 1), 1),
+                        "bound_seconds": round(longest / 64 * split_tensor_cycles_per_block(len(table)) / SM_HZ, 3),
                         "bound": "longest_bytes / 64 x cycles per block of one chain / SM clock (one tensor is one serial chain)",
+                        "floor_seconds": round(longest / 64 * ISSUE_FLOOR_CYCLES_PER_BLOCK / SM_HZ, 3),
                         "device_status": ctx.device_status(), "clocks": clocks.summary()}
     out["config3"] = c3
     del data, wl, m, tens
