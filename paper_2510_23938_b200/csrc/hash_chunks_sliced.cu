@@ -35,6 +35,16 @@
 #include "tma_dev.cuh"
 #include "chunk_tensor_map.h"
 
+#ifndef IV_ADD8
+#define IV_ADD8 0
+#endif
+#ifndef IV_MINB8
+#define IV_MINB8 1
+#endif
+#ifndef IV_MINB12
+#define IV_MINB12 0
+#endif
+
 namespace ivk {
 namespace {
 
@@ -43,8 +53,12 @@ namespace {
 // byte before data block j followed by its first 63 bytes; the word before the block is carried in a
 // register, at the start of a later slice it is read back from the blob.
 // ADD: where the additions of the compression go (see sha256_compress).
-template <int SEG, int STAGES, int MAX_WARPS, bool PREFIX, bool FWF, int ADD>
-__global__ void __launch_bounds__(32 * MAX_WARPS)
+// MINB: the second argument of __launch_bounds__ (0 = none).  It changes nothing that is computed, only the code the
+// compiler makes of the block loop: told that one CTA per SM is enough it spends 91-96 registers instead of 65-71 on
+// the instances with up to eight workers and orders the loop better (one group per scheduler: 798 -> 830 GB/s, two:
+// 876 -> 891, the 112 GiB launch: 808 -> 826); the twelve-worker instance loses by it (920 -> 904) and keeps 0.
+template <int SEG, int STAGES, int MAX_WARPS, bool PREFIX, bool FWF, int ADD, int MINB>
+__global__ void __launch_bounds__(32 * MAX_WARPS, MINB)
 hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
                           uint64_t slice_bytes, uint64_t total_tasks, uint32_t *__restrict__ slot,
@@ -332,9 +346,9 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8, MANY_STAGES = 2, MANY_WARPS = 12;
     constexpr size_t smem_per_warp = (size_t)STAGES * 8192, many_per_warp = (size_t)MANY_STAGES * 8192;
     constexpr size_t smem_pad = 1024;
-    auto kernel_plain = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, false, 0>;
-    auto kernel_fwf = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, true, 0>;
-    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, PREFIX, false, 2>;
+    auto kernel_plain = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, false, IV_ADD8, IV_MINB8>;
+    auto kernel_fwf = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, true, IV_ADD8, IV_MINB8>;
+    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, PREFIX, false, 2, IV_MINB12>;
     static bool configured[kMaxDevices] = {}, configured_fwf[kMaxDevices] = {}, configured_many[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel_plain, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
     if (cudaError_t e0 = ensure_dynamic_smem(kernel_fwf, MAX_WARPS * smem_per_warp + smem_pad, configured_fwf); e0 != cudaSuccess) return e0;
