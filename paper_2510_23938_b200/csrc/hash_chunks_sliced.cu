@@ -10,12 +10,9 @@
 // the FIFO at most once, its slices run in order; a warp never waits while it holds a task, so
 // the scheme needs no co-residency and cannot deadlock.  All waits are bounded.
 //
-// Service order.  A scheduler that runs two groups completes about 1.13 groups in the time a
-// scheduler with one group completes one, so between 592 and 1,184 groups the best fill has one
-// group on every scheduler and the surplus spread as second groups.  The launcher can therefore
-// ask for "first workers first": warps 0..3 of a CTA (one per scheduler) take tickets as they
-// come, warps 4..7 take a task only when one lies in the FIFO unclaimed.  The schedulers left
-// with one group finish early and then take over what remains of the others.
+// Worker count.  A scheduler that runs two groups completes about 1.07 groups in the time a
+// scheduler with one group completes one, so a second worker per scheduler pays only when most
+// schedulers get a second group: four workers per SM up to 6.45 groups per SM, eight from there.
 //
 // Data movement: the blob is described to the TMA unit as a 2-D tensor [chunk][byte] with the chunk
 // size as row pitch, and ONE tiled copy of a 32-row x 128-byte box brings the next two blocks of all
@@ -35,20 +32,9 @@
 #include "tma_dev.cuh"
 #include "chunk_tensor_map.h"
 
-#ifndef IV_ADD8
-#define IV_ADD8 0
-#endif
-#ifndef IV_MINB8
-#define IV_MINB8 1
-#endif
-#ifndef IV_MINB12
-#define IV_MINB12 0
-#endif
-
 namespace ivk {
 namespace {
 
-// FWF ("first workers first"): warps 4..7 take only left-over tasks, see the service order above.
 // PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash).  Message block j is then the
 // byte before data block j followed by its first 63 bytes; the word before the block is carried in a
 // register, at the start of a later slice it is read back from the blob.
@@ -57,7 +43,7 @@ namespace {
 // compiler makes of the block loop: told that one CTA per SM is enough it spends 91-96 registers instead of 65-71 on
 // the instances with up to eight workers and orders the loop better (one group per scheduler: 798 -> 830 GB/s, two:
 // 876 -> 891, the 112 GiB launch: 808 -> 826); the twelve-worker instance loses by it (920 -> 904) and keeps 0.
-template <int SEG, int STAGES, int MAX_WARPS, bool PREFIX, bool FWF, int ADD, int MINB>
+template <int SEG, int STAGES, int MAX_WARPS, bool PREFIX, int ADD, int MINB>
 __global__ void __launch_bounds__(32 * MAX_WARPS, MINB)
 hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
@@ -94,12 +80,10 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
     uint32_t parity = 0;
     bool failed = false;
 
-    bool first_take = true;
     for (;;) {
         // ---- take a ticket, wait for the group that is pushed under it
         unsigned long long t = 0;
-        if (lane == 0) t = (!FWF || warp < 4) ? atomicAdd(&q->head, 1ull) : take_leftover_ticket(q, total_tasks, first_take);
-        first_take = false;
+        if (lane == 0) t = atomicAdd(&q->head, 1ull);
         t = __shfl_sync(0xffffffffu, t, 0);
         if (t >= total_tasks) break;
         uint32_t entry = 0;
@@ -341,17 +325,15 @@ template <bool PREFIX>
 cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
                           const uint32_t *d_one, int sm_count, cudaStream_t stream) {
-    // Three instances: up to eight workers per SM with three stages each (arrival order or first workers
-    // first), and twelve workers with two stages each for launches that keep all of them busy.
+    // Two instances: up to eight workers per SM with three stages each, and twelve workers with two stages each
+    // for launches that keep all of them busy.
     constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8, MANY_STAGES = 2, MANY_WARPS = 12;
     constexpr size_t smem_per_warp = (size_t)STAGES * 8192, many_per_warp = (size_t)MANY_STAGES * 8192;
     constexpr size_t smem_pad = 1024;
-    auto kernel_plain = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, false, IV_ADD8, IV_MINB8>;
-    auto kernel_fwf = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, true, IV_ADD8, IV_MINB8>;
-    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, PREFIX, false, 2, IV_MINB12>;
-    static bool configured[kMaxDevices] = {}, configured_fwf[kMaxDevices] = {}, configured_many[kMaxDevices] = {};
-    if (cudaError_t e0 = ensure_dynamic_smem(kernel_plain, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
-    if (cudaError_t e0 = ensure_dynamic_smem(kernel_fwf, MAX_WARPS * smem_per_warp + smem_pad, configured_fwf); e0 != cudaSuccess) return e0;
+    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, 0, 1>;
+    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, PREFIX, 2, 0>;
+    static bool configured[kMaxDevices] = {}, configured_many[kMaxDevices] = {};
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
     if (cudaError_t e0 = ensure_dynamic_smem(kernel_many, MANY_WARPS * many_per_warp + smem_pad, configured_many); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, total_tasks = 0;
     (void)sliced_scratch_bytes(n_chunks, chunk_bytes, &slice_bytes, &total_tasks, nbytes);
@@ -364,22 +346,14 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     slice_queue_init<<<64, 256, 0, stream>>>(slot, total_tasks, groups, q, next_slice);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    // One persistent CTA per SM with four workers (one per scheduler) or eight (two per scheduler).  A
-    // scheduler with two groups finishes 1.11 groups in the time a scheduler with one finishes one, so
-    // eight workers pay once G is well above 592, but with G < 1184 not every scheduler gets two.  Measured
-    // (GB/s at G = 864 / 896 / 960 / 1024 / 1100 groups):
-    //  * four workers: 798 for every G >= 592;
-    //  * eight workers, FIFO served in arrival order: idle workers fall at random and groups that met
-    //    doubly loaded schedulers more often finish late (4 MiB chunks: 777 / 791 / 818 / 841 / 866);
-    //  * eight workers, first workers served first (a second worker takes only what is left over): the
-    //    schedulers with one group finish early and then take over the rest; needs fine slices (256
-    //    per chunk) to balance (4 MiB chunks: 801 / 806 / 825 / 842 / 865; 1 MiB chunks with 64 slices:
-    //    767 / 763 / 795 / 822 / 853 against 764 / 780 / 812 / 833 / 860 in arrival order).
-    const bool fine = ((chunk_bytes & ~63ull) + slice_bytes - 1) / slice_bytes >= 192;   // about 256 slices per chunk
-    uint64_t warps = 4;
-    bool first_workers_first = false;
-    if (fine && 20 * groups >= 117ull * (uint64_t)sm_count) { warps = MAX_WARPS; first_workers_first = groups < 8ull * sm_count; }
-    else if (!fine && 10 * groups >= 63ull * (uint64_t)sm_count) warps = MAX_WARPS;
+    // One persistent CTA per SM with four workers (one per scheduler) or eight (two per scheduler).  Measured
+    // (GB/s at G = 600 / 800 / 896 / 1000 / 1100 / 1184 groups of 4 MiB chunks; 1 MiB chunks within 1 %):
+    //  * four workers: 831 / 832 / 833 / 829 / 834 / 834, flat for every G >= 592;
+    //  * eight workers: 745 / 769 / 813 / 852 / 884 / 897 (idle second workers fall at random, and a scheduler
+    //    with two groups is only 7 % ahead of one with one);
+    //  * five, six or seven workers: 835 / 797 / 795 at 896, 834 / 849 / 847 at 1000; eight workers of which the second
+    //    four take only unclaimed tasks: 787 / 809 / 832 / 851 / 878 / 896 -- never ahead of the better of the two above.
+    const uint64_t warps = (100 * groups >= 645ull * (uint64_t)sm_count) ? MAX_WARPS : 4;
     // From twelve groups per SM on, three warps per scheduler hide the longer chains of multiply-add
     // additions, which take a tenth of the ALU pipe's load: 917 GB/s against 884 (32 GiB in 64 KiB chunks).
     if (groups >= (uint64_t)MANY_WARPS * (uint64_t)sm_count) {
@@ -389,9 +363,7 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
             next_slice, mid, d_one);
         return cudaGetLastError();
     }
-    auto kernel = first_workers_first ? kernel_fwf : kernel_plain;
-    t_instance = first_workers_first ? "8 workers per SM, first workers first"
-                                     : (warps == 4 ? "4 workers per SM" : "8 workers per SM, arrival order");
+    t_instance = warps == 4 ? "4 workers per SM" : "8 workers per SM";
     kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
         map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
         mid, d_one);

@@ -116,8 +116,8 @@ def test_weight_file_configurations_completely(ctx, cfg_id):
 
 
 def test_largest_configuration_completely(ctx):
-    """112 GiB, 4 MiB chunks: the launch the benchmark times (sliced kernel, tiled copies, first workers
-    first), every one of its 28,672 digests against the oracle."""
+    """112 GiB, 4 MiB chunks: the launch the benchmark times (migrating kernel, tiled copies, four workers
+    per SM), every one of its 28,672 digests against the oracle."""
     _need(125 * GIB)
     wl = bench.build_workload(4, torch.device("cuda", 0), seed=1000)
     data, chunk = wl["data"], wl["chunk"]
@@ -126,6 +126,7 @@ def test_largest_configuration_completely(ctx):
     assert n == 28_672
     got = ctx.hash_chunks(data, chunk)
     assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel" and ctx.device_status() == 0
+    assert ctx.last_leaf_instance == "4 workers per SM"
     host_got = _host(got)
 
     # the oracle over the whole blob, one 4 GiB window at a time: SHA-256 chunk digests, and the RFC 6962 leaf hashes

@@ -4,8 +4,7 @@ library writes, and the bounded-wait failure path run end to end.
 Guard bytes.  Every output of a call (digests, roots, result records, index lists, tree arrays, hashing
 states) lies inside a larger device buffer filled with a sentinel; after the call the margins on both sides
 must be untouched and the output must equal the oracle's.  The shapes walk through every leaf-hashing
-kernel and launch shape the dispatcher can pick below the full-size configurations (the remaining one,
-"first workers first", needs more than 83 GiB and is covered by the full-size test).
+kernel and launch shape the dispatcher can pick.
 
 Timeout.  A kernel whose wait runs out must return, set the device status to 1 and leave the context
 usable: `iv_selftest_wait_timeout` waits, with the library's own wait routine and a short limit, on a
@@ -63,7 +62,7 @@ LEAF_SHAPES = [
     (100 * (64 << 10) + 4097, 64 << 10, "hash_chunks_split_kernel", ""),    # few chains
     (9_600 * 4096 + 100, 4096, "hash_chunks_pairs_kernel", ""),             # 300 groups
     (16_000 * 4096 + 64, 4096, "hash_chunks_sliced_kernel", "4 workers per SM"),
-    (32_000 * 4096, 4096, "hash_chunks_sliced_kernel", "8 workers per SM, arrival order"),
+    (32_000 * 4096, 4096, "hash_chunks_sliced_kernel", "8 workers per SM"),
     (57_000 * 4096 + 5, 4096, "hash_chunks_sliced_kernel", "12 workers per SM"),
 ]
 
