@@ -29,7 +29,7 @@ constexpr unsigned long long kTaskDone = ~0ull, kTaskFailed = ~0ull - 1;
 
 // PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash), as in the migrating kernel.
 template <int SEG, int STAGES, int NSLOT, int PAIR, bool PREFIX>
-__global__ void __launch_bounds__(64)
+__global__ void __launch_bounds__(64, 1)   // the stated minimum of one CTA per SM changes only the compiler's code: 592 against 585 GB/s
 hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
                          uint8_t *__restrict__ digests, uint32_t *__restrict__ status, uint64_t slice_bytes,
                          uint64_t total_tasks, uint32_t *__restrict__ slot, SliceQueue *__restrict__ q,
@@ -276,10 +276,10 @@ hash_chunks_pairs_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
 }  // namespace
 
 bool hash_chunks_wants_pairs(const uint8_t *d_data, uint64_t chunk_bytes, uint64_t n_chunks, int sm_count) {
-    // 580 GB/s flat for the pairs against 1.345 GB/s per group for one whole-compression warp per group:
-    // measured crossover at 431 groups = 2.91 x SMs, for chunks of 64 KiB to 4 MiB
+    // 590 GB/s flat for the pairs against 1.40 GB/s per group for one whole-compression warp per group:
+    // measured crossover at 422 groups = 2.85 x SMs, for chunks of 1 MiB and 4 MiB
     return hash_chunks_wants_slices(d_data, chunk_bytes, n_chunks, sm_count) &&
-           ((n_chunks + 31) / 32) * 100ull < 291ull * (uint64_t)sm_count;
+           ((n_chunks + 31) / 32) * 100ull < 285ull * (uint64_t)sm_count;
 }
 
 cudaError_t launch_hash_chunks_pairs(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n_chunks,
