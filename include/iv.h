@@ -77,9 +77,8 @@ uint64_t iv_kernel_launches(const iv_ctx *ctx);
  * Static text, never freed. */
 const char *iv_last_leaf_kernel(const iv_ctx *ctx);
 
-/* Where that kernel has several launch shapes (the many-chain kernel: workers per SM and the order in
- * which they are served; the SHA-384/512 two-warp kernel: pairs per SM), the one the last call ran in;
- * "" otherwise.  Static text. */
+/* Where that kernel has several launch shapes (the many-chain kernel: workers per SM; the SHA-384/512
+ * two-warp kernel: pairs per SM), the one the last call ran in; "" otherwise.  Static text. */
 const char *iv_last_leaf_instance(const iv_ctx *ctx);
 
 /* Self-test of the bounded waits (a diagnostic; the paper has no counterpart).  Every wait inside the
