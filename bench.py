@@ -50,10 +50,10 @@ PEAK_GBS = SM_COUNT * INT_LANES_PER_SM * SM_HZ / INT_OPS_PER_BYTE / 1e9
 # two-warp kernel as measured (leaf-kernel time x clock / blocks per chunk) in its instance for up to one
 # group of 32 chains per SM (the 16 GB configuration) and in the one for up to two, and the issue floor of
 # the round function (10 SHF/LOP3 per round on a 16-lane pipe, two cycles each).
-SPLIT_CYCLES_PER_BLOCK_ROOMY = 1877.0
+SPLIT_CYCLES_PER_BLOCK_ROOMY = 1860.0
 SPLIT_CYCLES_PER_BLOCK = 1916.0
 # the same kernel's instances for tensors (other launch-bounds hint, 32-bit block counters), as measured
-SPLIT_TENSOR_CYCLES_PER_BLOCK_ROOMY = 1845.0
+SPLIT_TENSOR_CYCLES_PER_BLOCK_ROOMY = 1835.0
 SPLIT_TENSOR_CYCLES_PER_BLOCK = 1910.0
 ISSUE_FLOOR_CYCLES_PER_BLOCK = 1280.0
 

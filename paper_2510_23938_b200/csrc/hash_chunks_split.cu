@@ -274,9 +274,10 @@ hash_chunks_split_kernel(const uint8_t *__restrict__ data, uint64_t nbytes, uint
 
 namespace {
 
-// Two instances per mode.  Up to one group per SM a CTA may use most of an SM's shared memory: three W+K slots of
-// FOUR blocks each (a hand-over every fourth block): 1,877 cycles per block for chunks.  Up to two groups per SM two
-// CTAs share an SM: three slots of two blocks (104 KB): 1,916 cycles per block.  (Fetching the next block's first
+// Two instances per mode.  Up to one group per SM a CTA may use most of an SM's shared memory: two W+K slots of
+// EIGHT blocks each (190 KB; a hand-over every eighth block): 1,860 cycles per block for chunks (three slots of four:
+// 1,873, two of four: 1,890, four of four: 1,878).  Up to two groups per SM two CTAs share an SM: three slots of two
+// blocks (104 KB): 1,914 cycles per block.  (Fetching the next block's first
 // W+K values during the last rounds of the current one, within a slot, was measured and does not pay: 1,890.)
 // The 32 bulk copies of a stage leave the producer one after the other and cost it about 2,000 cycles per stage.
 // With chunks the consumer is the slower warp either way; with tensors the producer has the selects on top and
@@ -286,8 +287,8 @@ template <bool RAGGED, bool PREFIX, int PAIR>
 cudaError_t launch_split_instance(const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes, uint64_t n, uint8_t *d_digests,
                                   uint32_t *d_status, const uint32_t *d_one, const uint64_t *d_offsets, const uint64_t *d_lengths,
                                   const uint32_t *d_order, iv_sha_state *d_states, int finish, cudaStream_t stream) {
-    constexpr bool LONG_STAGES = RAGGED && PAIR == 4;
-    constexpr int SEG = LONG_STAGES ? 1024 : 512, STAGES = LONG_STAGES ? 2 : 3, NSLOT = 3;
+    constexpr bool ROOMY = PAIR == 8, LONG_STAGES = RAGGED && ROOMY;
+    constexpr int SEG = LONG_STAGES ? 1024 : 512, STAGES = LONG_STAGES ? 2 : 3, NSLOT = ROOMY ? 2 : 3;
     constexpr size_t smem = (size_t)STAGES * 32 * (SEG + 16) + (size_t)NSLOT * PAIR * 32 * (64 * 4 + 16);
     auto kernel = hash_chunks_split_kernel<SEG, STAGES, NSLOT, RAGGED, PAIR, PREFIX, RAGGED ? 1 : 0, RAGGED>;
     static bool configured[kMaxDevices] = {};
@@ -316,11 +317,11 @@ cudaError_t launch_hash_chunks_split(const uint8_t *d_data, uint64_t nbytes, uin
     // ALU adds, the others go to the FMA pipe (the fastest placement measured).
     const bool roomy = (n_chunks + 31) / 32 <= (uint64_t)sm_count_of_current_device();
     if (zero_prefix)
-        return roomy ? launch_split_instance<false, true, 4>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
+        return roomy ? launch_split_instance<false, true, 8>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
                                                              nullptr, nullptr, nullptr, nullptr, 1, stream)
                      : launch_split_instance<false, true, 2>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
                                                              nullptr, nullptr, nullptr, nullptr, 1, stream);
-    return roomy ? launch_split_instance<false, false, 4>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
+    return roomy ? launch_split_instance<false, false, 8>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
                                                           nullptr, nullptr, nullptr, nullptr, 1, stream)
                  : launch_split_instance<false, false, 2>(d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, d_one,
                                                           nullptr, nullptr, nullptr, nullptr, 1, stream);
@@ -330,7 +331,7 @@ cudaError_t launch_hash_ragged_split(const uint8_t *d_base, const uint64_t *d_of
                                      const uint32_t *d_order, uint64_t n, uint8_t *d_digests, uint32_t *d_status,
                                      const uint32_t *d_one, iv_sha_state *d_states, int finish, cudaStream_t stream) {
     const bool roomy = (n + 31) / 32 <= (uint64_t)sm_count_of_current_device();
-    return roomy ? launch_split_instance<true, false, 4>(d_base, 0, 0, n, d_digests, d_status, d_one, d_offsets, d_lengths,
+    return roomy ? launch_split_instance<true, false, 8>(d_base, 0, 0, n, d_digests, d_status, d_one, d_offsets, d_lengths,
                                                          d_order, d_states, finish, stream)
                  : launch_split_instance<true, false, 2>(d_base, 0, 0, n, d_digests, d_status, d_one, d_offsets, d_lengths,
                                                          d_order, d_states, finish, stream);
