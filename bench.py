@@ -67,7 +67,7 @@ def split_tensor_cycles_per_block(tensors: int) -> float:
 
 
 # DRAM read+write bytes per byte hashed, from the ncu captures summarised under profiles/.
-TRAFFIC_FACTOR = {"hash_chunks_sliced_kernel": 1.0038, "hash_chunks_split_kernel": 1.0026}
+TRAFFIC_FACTOR = {"hash_chunks_sliced_kernel": 1.0038, "hash_chunks_split_kernel": 1.0022}
 
 CONFIGS = {
     1: dict(name="config1: 64 MiB uniform random bytes, 64 KiB chunks, 1024 leaves", kind="uniform",
