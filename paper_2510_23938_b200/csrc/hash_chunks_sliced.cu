@@ -466,9 +466,6 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
         if (groups >= 6 * sms && groups < 7 * sms) warps = 6;
         else if (groups >= 7 * sms && 100 * groups < 725 * sms) warps = 7;
     }
-#ifdef IV_FORCE_WARPS
-    warps = IV_FORCE_WARPS;
-#endif
     // From twelve groups per SM on, three warps per scheduler hide the longer chains of multiply-add
     // additions, which take a tenth of the ALU pipe's load: 917 GB/s against 884 (32 GiB in 64 KiB chunks).
     if (groups >= (uint64_t)MANY_WARPS * (uint64_t)sm_count) {
