@@ -70,26 +70,42 @@ __global__ void lag_queues_init(uint32_t *__restrict__ slot0, uint32_t *__restri
 
 constexpr uint32_t kNoMoreTasks = 0u, kGaveUp = 0xffffffffu;
 
+// The four counters of the two queues as one lane saw them.
+struct QueueCounters {
+    unsigned long long head[2], tail[2];
+};
+__device__ __forceinline__ QueueCounters read_counters(const LagQueues *q) {
+    QueueCounters c;
+    c.head[0] = *reinterpret_cast<const volatile unsigned long long *>(&q->head[0]);
+    c.head[1] = *reinterpret_cast<const volatile unsigned long long *>(&q->head[1]);
+    c.tail[0] = *reinterpret_cast<const volatile unsigned long long *>(&q->tail[0]);
+    c.tail[1] = *reinterpret_cast<const volatile unsigned long long *>(&q->tail[1]);
+    return c;
+}
+
 // One lane's call: the next task for a worker that prefers queue `pref`.  Returns group + 1, kNoMoreTasks once every
 // slice of the launch is done, or kGaveUp after about four seconds without finding work (some other worker has
 // failed); *done_seen receives the number of slices completed when the task was taken (the push that follows the
-// task uses it as the average progress: a task's time out of date, which is exact enough).  The counters of both
-// queues are read together and the progress counter together with the entry, so that a take costs three trips to
-// memory.  Out of line so that the hashing loop's register allocation does not depend on it.
+// task uses it as the average progress: a task's time out of date, which is exact enough).  `seen` holds the
+// counters as the caller read them a little earlier (before it parked its finished slice, so that this read overlaps
+// that work); they only choose the queue and the position to try, the compare-and-swap decides.  A lost race tries
+// the position the swap returned before reading everything again.  Out of line so that the hashing loop's register
+// allocation does not depend on it.
 __device__ __noinline__ uint32_t take_task(LagQueues *q, const uint32_t *slot0, const uint32_t *slot1, uint32_t pref,
-                                           unsigned long long total_tasks, unsigned long long *done_seen) {
+                                           unsigned long long total_tasks, unsigned long long *done_seen, QueueCounters seen) {
     const long long t0 = clock64();
     unsigned ns = 64;
     for (;;) {
-        const unsigned long long h0 = *reinterpret_cast<volatile unsigned long long *>(&q->head[0]);
-        const unsigned long long h1 = *reinterpret_cast<volatile unsigned long long *>(&q->head[1]);
-        const unsigned long long t0q = *reinterpret_cast<volatile unsigned long long *>(&q->tail[0]);
-        const unsigned long long t1q = *reinterpret_cast<volatile unsigned long long *>(&q->tail[1]);
-        const bool have0 = t0q > h0, have1 = t1q > h1;
+        const bool have0 = seen.tail[0] > seen.head[0], have1 = seen.tail[1] > seen.head[1];
         if (have0 || have1) {
             const uint32_t which = (pref == 0u) ? (have0 ? 0u : 1u) : (have1 ? 1u : 0u);
-            const unsigned long long h = which ? h1 : h0;
-            if (atomicCAS(&q->head[which], h, h + 1ull) != h) continue;        // lost the race: look again
+            const unsigned long long h = seen.head[which];
+            const unsigned long long was = atomicCAS(&q->head[which], h, h + 1ull);
+            if (was != h) {                                    // lost the race (or the counters were stale): try again from
+                seen.head[which] = was;                        // where the head stands now, against the tail as last seen
+                if (seen.tail[which] <= was) seen = read_counters(q);
+                continue;
+            }
             // position h is this worker's; its entry may still be on its way (the pusher raises the tail first)
             const unsigned long long d = *reinterpret_cast<volatile unsigned long long *>(&q->done);
             const uint32_t *slot = (which ? slot1 : slot0) + h;
@@ -105,6 +121,7 @@ __device__ __noinline__ uint32_t take_task(LagQueues *q, const uint32_t *slot0, 
         if (clock64() - t0 > 8000000000ll) return kGaveUp;
         __nanosleep(ns);
         if (ns < 1024) ns *= 2;
+        seen = read_counters(q);
     }
 }
 
@@ -162,13 +179,15 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
     const uint32_t n_warps = blockDim.x >> 5;
     const bool mixed = n_warps > 4 && n_warps < 8;
     const uint32_t pref = (mixed && !(warp < 4 && warp + 4 >= n_warps)) ? 1u : 0u;
+    QueueCounters seen = {};
+    if (LAG && lane == 0) seen = read_counters(q);
 
     for (;;) {
         uint32_t entry = 0;
         unsigned long long done_seen = 0;
         if constexpr (LAG) {
             // ---- take a task: lagging groups first for a worker alone on its scheduler, leading ones first otherwise
-            if (lane == 0) entry = take_task(q, slot0, slot1, pref, total_tasks, &done_seen);
+            if (lane == 0) entry = take_task(q, slot0, slot1, pref, total_tasks, &done_seen, seen);
             entry = __shfl_sync(0xffffffffu, entry, 0);
             if (entry == kNoMoreTasks) break;
             if (entry == kGaveUp) { failed = true; break; }
@@ -304,6 +323,7 @@ hash_chunks_sliced_kernel(const __grid_constant__ CUtensorMap tmap, const uint8_
         }
         if (failed) break;
 
+        if (LAG && lane == 0) seen = read_counters(q);          // for the next take; on its way while the slice is parked
         if (!last_slice) {
             uint32_t *m = mid + g * 256 + lane;
 #pragma unroll
@@ -455,14 +475,15 @@ cudaError_t launch_sliced(const CUtensorMap &map, const uint8_t *d_data, uint64_
     //    at random, and a scheduler with two groups is only 8 % ahead of one with one);
     //  * as many workers as whole groups per SM, so that all are busy, on the single FIFO: five / six / seven workers
     //    835 / 797 / 795 at 896 and 834 / 849 / 847 at 1000 -- the groups' progress spreads and the launch ends on a
-    //    few stragglers; on the two progress-ordered queues: six workers 856 at 896 and 857 at 1000, seven 876 at
-    //    1,040 and 877 at 1,100, five 833 at 740 and 837 at 800.  The queues need slices to work with: with 64 per
-    //    chunk (1 MiB chunks) six and seven workers still win (839-844 and 861-864 against 825 and 858 for four or
-    //    eight), with 16 they lose.
+    //    few stragglers; on the two progress-ordered queues: five workers 836 / 843 / 844 at 740 / 800 / 887, six 862 /
+    //    863 at 896 / 1000, seven 881 at 1,040.  The queues need slices to work with: with 64 per chunk (1 MiB chunks)
+    //    six and seven workers still win (846-850 and 868 against 827 and 858 for four or eight) and five no longer do
+    //    (817-831 against 823-829), with 16 per chunk all of them lose.
     const uint64_t slices_per_chunk = ((chunk_bytes & ~63ull) + slice_bytes - 1) / slice_bytes;
     const uint64_t sms = (uint64_t)sm_count;
     uint64_t warps = (100 * groups >= 645 * sms) ? MAX_WARPS : 4;
     if (slices_per_chunk >= 64) {
+        if (slices_per_chunk >= 128 && groups >= 5 * sms && groups < 6 * sms) warps = 5;
         if (groups >= 6 * sms && groups < 7 * sms) warps = 6;
         else if (groups >= 7 * sms && 100 * groups < 725 * sms) warps = 7;
     }

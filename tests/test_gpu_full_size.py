@@ -213,12 +213,12 @@ def test_largest_configuration_completely(ctx):
     torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("groups,instance", [(900, "6 workers per SM"), (1_040, "7 workers per SM")])
-def test_progress_ordered_queues_with_one_mib_chunks(ctx, groups, instance):
+@pytest.mark.parametrize("groups,chunk,instance", [(750, 2 << 20, "5 workers per SM"), (900, 1 << 20, "6 workers per SM"),
+                                                   (1_040, 1 << 20, "7 workers per SM")])
+def test_progress_ordered_queues_with_64_and_128_slices_per_chunk(ctx, groups, chunk, instance):
     """The launch shapes whose workers differ in speed (six or seven per SM, tasks from the two progress-ordered
-    queues) with 64 slices per chunk: 28 to 33 GiB in 1 MiB chunks, every digest and the root against the oracle,
-    in the default and in the RFC 6962 mode."""
-    chunk = 1 << 20
+    queues) with 64 or 128 slices per chunk: 28 to 47 GiB in chunks of 1 or 2 MiB, every digest and the root against
+    the oracle, the last shape in the RFC 6962 mode as well."""
     n = groups * 32 - 5
     nbytes = n * chunk - 12_344                       # short last chunk beside the main launch
     torch.cuda.empty_cache()
@@ -232,7 +232,7 @@ def test_progress_ordered_queues_with_one_mib_chunks(ctx, groups, instance):
     assert ctx.device_status() == 0
     assert np.array_equal(_host(got), want)
     assert _host(ctx.merkle_root(got)).tobytes() == oracle.merkle_root(want)
-    if groups == 900:
+    if groups != 1_040:
         return                                        # the prefixed instance is held against the oracle on the other shape
     got6962 = ctx.hash_chunks_rfc6962(data, chunk)
     assert (ctx.last_leaf_kernel, ctx.last_leaf_instance) == ("hash_chunks_sliced_kernel", instance)
