@@ -668,6 +668,33 @@ def measure_secondary(ctx, device, gpu_index, args):
           "target_70pct_of_roofline": "not met and not reachable with leaf = SHA-256(4 MiB chunk): 3,830 serial chains bound "
                                       "the launch at 44 % of the roofline even at the issue floor of 1,280 cycles per block",
           "clocks": m["clocks"]}
+    # the same file in the separately named two-level mode (a chunk's digest is the root over the SHA-256 digests of
+    # its 64 KiB pieces: other digests than the default path's, 64 times as many chains)
+    sub = 64 << 10
+    d2 = ctx.hash_chunks_two_level(data, chunk, sub)
+    m2 = ctx.make_manifest(nbytes, chunk, d2, bytes(ctx.merkle_root(d2).cpu().numpy().tobytes()))
+    res2 = binding.new_result(device)
+    idx2 = torch.zeros(8, dtype=torch.int64, device=device)
+    for _ in range(3):
+        ctx.verify_manifest_two_level(data, m2, sub, res2, idx2)
+    n2 = steps_for(18.0, args.steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    with ClockSampler(gpu_index) as clocks2:
+        e0.record(stream)
+        for _ in range(n2):
+            ctx.verify_manifest_two_level(data, m2, sub, res2, idx2)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    r2 = binding.read_result(res2)
+    ok2 = bool(r2["root_ok"]) and r2["n_mismatch"] == 0 and r2["status"] == 0 and ctx.device_status() == 0
+    gbs2 = nbytes / (e0.elapsed_time(e1) / n2 * 1e-3) / 1e9
+    c3["two_level"] = {"value": round(gbs2, 3) if ok2 else None, "unit": "GB/s", "frac": round(gbs2 / PEAK_GBS, 4),
+                       "sub_bytes": sub, "chains": binding.n_chunks(nbytes, sub), "steps": n2, "verified_ok": ok2,
+                       "leaf_kernel": ctx.last_leaf_kernel + " (" + ctx.last_leaf_instance + ")",
+                       "note": "iv_verify_manifest_two_level: a separately named mode whose digests differ from the default path's",
+                       "clocks": clocks2.summary()}
+    del d2, m2
     e2e = measure_e2e(ctx, wl, device, 3)
     c3["streamed"] = {k: e2e.get(k) for k in ("value", "unit", "ms_per_step", "h2d_copy_alone_gbs", "verified_ok", "api")}
     # per-tensor digests of the same file: one iv_hash_ragged call over its 291 tensors
