@@ -642,8 +642,9 @@ def measure_cpu_baseline(ctx, wl, device, oracle, ragged, man_digests, ragged_st
 
 def measure_secondary(ctx, device, gpu_index, args):
     """The other named configurations, for the record beside the headline: the 16 GB weight file (device
-    resident, streamed from pinned host memory, and its per-tensor digests) and the 64 MiB blob (alone, and
-    with its three tampered copies verified as one batch).  Each timed region lasts at least a second so that
+    resident, in the two-level mode, streamed from pinned host memory, and its per-tensor digests), the 64 MiB blob
+    (alone, and with its three tampered copies verified as one batch), the 2.6 GB weight file and the ragged
+    tensor set.  Each timed region lasts at least a second so that
     the clock sampler sees it."""
     from paper_2510_23938_b200 import binding, inputs
     out = {}
@@ -752,6 +753,45 @@ def measure_secondary(ctx, device, gpu_index, args):
                         "mismatch_idx": got_idx, "api": "iv_verify_manifest_batch: the blob and its three tampered copies, "
                                                         "one hashing launch", "clocks": clocks}
     out["config1"] = c1
+    del data, wl, m, blobs, results, bidx
+    torch.cuda.empty_cache()
+
+    # ---- 2.6 GB weight file, 1 MiB chunks
+    wl = build_workload(2, device, seed=1000)
+    m = measure_verify(ctx, wl, device, steps_for(15.6, args.steps), 3, gpu_index)
+    rf = m["roofline"]
+    out["config2"] = {"workload": wl["name"], "bytes": wl["nbytes"], "chunk_bytes": wl["chunk"], "chains": m["n_units"],
+                      "value": round(m["gbs"], 3) if m["verified_ok"] else None, "unit": "GB/s",
+                      "verified_ok": m["verified_ok"], "ms_per_step": round(m["ms_per_step"], 4), "leaf_kernel": rf["kernel"],
+                      "leaf_kernel_ms": rf["launch_ms"], "frac": rf["frac"],
+                      "chain_count_bound_gbs": rf["chain_count_bound_gbs"], "clocks": m["clocks"]}
+    del wl, m
+    torch.cuda.empty_cache()
+
+    # ---- 10,000 ragged tensors: one SHA-256 each and the root over the digests
+    wl = build_workload(5, device, seed=1000)
+    data = wl["data"]
+    d_off = torch.from_numpy(wl["offsets"]).to(device)
+    d_len = torch.from_numpy(wl["lengths"]).to(device)
+    n_t = int(d_off.numel())
+    tens = torch.empty((n_t, 32), dtype=torch.uint8, device=device)
+    root = torch.empty(32, dtype=torch.uint8, device=device)
+
+    def ragged_step():
+        ctx.hash_ragged(data, d_off, d_len, out=tens)
+        ctx.merkle_root(tens, out=root)
+
+    n5 = max(2, min(args.steps, 3))
+    total_ms, clocks = time_steps(ragged_step, n5, 3, None, gpu_index)
+    longest = int(wl["lengths"].max())
+    ms5 = total_ms / n5
+    out["config5"] = {"workload": wl["name"], "bytes": wl["nbytes"], "n_tensors": n_t, "longest_bytes": longest,
+                      "value": round(wl["nbytes"] / (ms5 * 1e-3) / 1e9, 3), "unit": "GB/s", "ms_per_step": round(ms5, 3),
+                      "steps": n5, "frac": round(wl["nbytes"] / (ms5 * 1e-3) / 1e9 / PEAK_GBS, 4),
+                      "leaf_kernel": ctx.last_leaf_kernel,
+                      "cycles_per_block_of_the_longest_tensor": round(ms5 * 1e-3 * SM_HZ / (longest // 64 + 1), 1),
+                      "bound": "the longest tensor is one serial chain: its blocks x cycles per block / SM clock",
+                      "device_status": ctx.device_status(), "clocks": clocks}
     return out
 
 
